@@ -1,0 +1,144 @@
+"""Pins for the scheduler / block-allocator oracle: invariants, closed forms,
+brute-force re-simulation, legal slot transitions."""
+import numpy as np
+import pytest
+
+from oracle import scheduler as O1
+from synth import make_requests
+
+
+def _sim_reqs(reqs):
+    return [O1.SimRequest(r.ticket, r.n_prompt, r.max_new) for r in reqs]
+
+
+def _random_reqs(rng, n, pmax=70, nmax=20):
+    return [O1.SimRequest(t, int(rng.integers(1, pmax)), int(rng.integers(1, nmax))) for t in range(n)]
+
+
+def test_single_request_closed_form():
+    for P, N, chunk in [(1, 1, 64), (16, 1, 64), (17, 5, 8), (64, 32, 64), (65, 3, 16), (130, 7, 64)]:
+        tr, toks, sch = O1.simulate([O1.SimRequest(0, P, N)], 4, chunk, 64, 16, vocab=100)
+        n_prefill = O1.ceil_div(P, chunk)
+        assert len(tr) == n_prefill + N - 1
+        assert sum(len(r["allocated"]) for r in tr) == O1.ceil_div(P + N - 1, 16)
+        assert len(toks[0]) == N
+        # physical ids come off a fresh stack as 0, 1, 2, ...
+        assert [a[2] for r in tr for a in r["allocated"]] == list(range(O1.ceil_div(P + N - 1, 16)))
+        assert tr[-1]["free_count"] == 64 and tr[-1]["reserved"] == 0
+
+
+def test_max_batch_one_is_serial_in_ticket_order():
+    rng = np.random.default_rng(3)
+    reqs = _random_reqs(rng, 9)
+    tr, toks, _ = O1.simulate(reqs, 1, 32, 64, 16, vocab=50)
+    order = [t for r in tr for t in r["finished"]]
+    assert order == list(range(9))
+    for r in tr:
+        assert len({s[1] for s in r["scheduled"]}) == 1
+    assert len(tr) == sum(O1.ceil_div(q.P, 32) + q.N - 1 for q in reqs)
+
+
+def test_conservation_and_invariants_random():
+    rng = np.random.default_rng(5)
+    for trial in range(20):
+        reqs = _random_reqs(rng, int(rng.integers(1, 30)))
+        nb = int(rng.integers(8, 40))
+        reqs = [r for r in reqs if O1.blocks_needed(r.P, r.N, 16) <= nb]
+        for i, r in enumerate(reqs):
+            r.ticket = i
+        mb = int(rng.integers(1, 9))
+        chunk = int(rng.integers(1, 80))
+        tr, toks, sch = O1.simulate(reqs, mb, chunk, nb, 16, vocab=1000, check=O1.check_invariants)
+        assert sum(s[4] for r in tr for s in r["scheduled"] if s[2] == O1.PREFILL) == sum(q.P for q in reqs)
+        assert sum(len(r["sampled"]) for r in tr) == sum(q.N for q in reqs)
+        assert sorted(sch.stack) == list(range(nb)) and sch.reserved == 0
+        for r in tr:
+            assert sum(s[4] for s in r["scheduled"] if s[2] == O1.PREFILL) <= chunk
+            assert len(r["scheduled"]) <= mb
+            # token order inside a step: ascending batch slot
+            assert [s[0] for s in r["scheduled"]] == sorted(s[0] for s in r["scheduled"])
+        for (t, a, b) in sch.transitions:
+            assert (a, b) in O1.LEGAL_TRANSITIONS
+
+
+def test_fcfs_admission_order_and_head_of_line_blocking():
+    # pool fits the big head request only after the first ones drain; the small one behind must wait
+    reqs = [O1.SimRequest(0, 40, 8), O1.SimRequest(1, 100, 20), O1.SimRequest(2, 5, 2)]
+    nb = 8     # need: 3, 8, 1
+    tr, toks, _ = O1.simulate(reqs, 4, 64, nb, 16, vocab=10)
+    adm = [(r["iter"], t) for r in tr for (t, b) in r["admitted"]]
+    assert [t for _, t in adm] == [0, 1, 2]
+    it0, it1, it2 = (i for i, _ in adm)
+    fin0 = next(r["iter"] for r in tr if 0 in r["finished"])
+    assert it1 == fin0 + 1            # freed resources usable from the next iteration
+    assert it2 >= it1                 # never overtakes the blocked head
+    fin1 = next(r["iter"] for r in tr if 1 in r["finished"])
+    assert it2 == fin1 + 1            # pool is fully reserved by request 1 until it ends
+
+
+def test_watermark_gates_visibility():
+    reqs = [O1.SimRequest(t, 10, 3) for t in range(4)]
+    W = [0, 0, 1, 3, 3, 3, 3, 3, 3]
+    tr, _, _ = O1.simulate(reqs, 8, 64, 64, 16, watermarks=W, vocab=10)
+    adm = {t: r["iter"] for r in tr for (t, b) in r["admitted"]}
+    assert adm == {0: 0, 1: 2, 2: 3, 3: 3}
+
+
+def test_lowest_free_batch_slot_and_lifo_block_reuse():
+    reqs = [O1.SimRequest(0, 16, 2), O1.SimRequest(1, 16, 6), O1.SimRequest(2, 20, 2)]
+    W = [1, 1, 2, 2, 2, 2, 2]
+    tr, _, _ = O1.simulate(reqs, 4, 64, 16, 16, watermarks=W, vocab=10)
+    assert tr[0]["admitted"] == [(0, 0), (1, 1)]
+    assert tr[0]["allocated"] == [(0, 0, 0), (1, 0, 1)]
+    # iteration 1: both decode at position 16 -> second block each: ids 2, 3; request 0 ends, frees 0 then 2
+    assert tr[1]["allocated"] == [(0, 1, 2), (1, 1, 3)]
+    assert tr[1]["finished"] == [0] and tr[1]["freed"] == [0, 2]
+    # iteration 2: ticket 2 takes batch slot 0 again, pops the most recently pushed blocks first
+    assert tr[2]["admitted"] == [(2, 0)]
+    assert tr[2]["allocated"] == [(0, 0, 2), (0, 1, 0)]
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2, 3])
+def test_brute_force_resimulation_agrees(seed):
+    rng = np.random.default_rng(100 + seed)
+    reqs = _random_reqs(rng, 12, pmax=60, nmax=9)
+    nb, mb, chunk = 14, 3, int(rng.integers(5, 40))
+    reqs = [r for r in reqs if O1.blocks_needed(r.P, r.N, 16) <= nb]
+    for i, r in enumerate(reqs):
+        r.ticket = i
+    # a bursty visibility schedule
+    W = []
+    w = 0
+    for i in range(400):
+        if rng.random() < 0.3:
+            w = min(len(reqs) - 1, w + int(rng.integers(1, 4)))
+        W.append(w)
+    tr, toks, _ = O1.simulate(reqs, mb, chunk, nb, 16, watermarks=W, vocab=64)
+    bf = O1.brute_force(reqs, mb, chunk, nb, 16, W[:len(tr)], toks)
+    assert len(bf) == len(tr)
+    for a, b in zip(tr, bf):
+        assert a == b
+
+
+def test_eos_ends_a_request_early():
+    r = O1.SimRequest(0, 5, 10, eos_id=7)
+    seq = iter([1, 2, 7, 3, 4])
+    tr, toks, sch = O1.simulate([r], 2, 64, 8, 16, sample_fn=lambda items: [next(seq) for i in items if i.sample])
+    assert toks[0] == [1, 2, 7]
+    assert sch.reserved == 0 and len(sch.stack) == 8
+
+
+def test_config1_stream_shape_and_trace():
+    reqs = make_requests(1)
+    assert len(reqs) == 8 and all(16 <= r.n_prompt <= 64 and r.max_new == 32 for r in reqs)
+    tr, toks, sch = O1.simulate(_sim_reqs(reqs), 8, 64, 256, 16, vocab=4096, check=O1.check_invariants)
+    assert all(len(v) == 32 for v in toks.values())
+    assert tr[0]["W"] == 7 and len(tr[0]["admitted"]) == 8
+
+
+def test_config3_stream_trace_runs_at_full_scale():
+    reqs = make_requests(3, n_requests=64)
+    sim = _sim_reqs(reqs)
+    tr, toks, sch = O1.simulate(sim, 256, 512, 60000, 16, vocab=128256)
+    assert sum(len(v) for v in toks.values()) == sum(r.max_new for r in reqs)
+    assert sch.reserved == 0 and len(sch.stack) == 60000
