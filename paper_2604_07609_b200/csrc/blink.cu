@@ -1,0 +1,798 @@
+// libblink: kernels of the GPU-resident serving loop and the C ABI around them.
+//
+// Persistent mode: one cooperative kernel (one CTA per SM) loops on the device;
+// CTA 0 runs the control plane, then all CTAs run the phases of the step
+// separated by grid barriers.  Stepped mode runs the very same device functions
+// as one host launch per phase (for profilers and debugging).
+#include <cuda_runtime.h>
+#include <stdio.h>
+#include <string.h>
+#include <time.h>
+
+#include <atomic>
+#include <chrono>
+#include <cmath>
+#include <deque>
+#include <mutex>
+#include <new>
+#include <thread>
+#include <vector>
+
+#include "../../include/blink.h"
+#include "control.cuh"
+#include "dev_ctx.cuh"
+#include "forward.cuh"
+#include "gemm_tc.cuh"
+
+namespace blink {
+
+enum Phase : int {
+  PH_NORM1 = 0, PH_QKV, PH_ROPE, PH_ATTN, PH_O, PH_NORM2, PH_GU, PH_SILU, PH_DOWN,
+  PH_FNORM, PH_LMHEAD, PH_SAMPLE, PH_COUNT
+};
+
+template <typename WT>
+__device__ __forceinline__ void gemm_dispatch(const DevCtx& c, const GemmArgs& a, int which, int layer, float* smem,
+                                              TcState& tc) {
+  if (c.gemm_tc) phase_gemm_tc(c, a, which, layer, smem, tc);
+  else phase_gemm_simt<WT>(a);
+}
+
+template <typename WT, int HD>
+__device__ __forceinline__ void attention_dispatch(const DevCtx& c, int layer, float* smem) {
+  switch (c.n_rep) {
+    case 1: phase_attention<WT, HD, 1>(c, layer, smem); break;
+    case 2: phase_attention<WT, HD, 2>(c, layer, smem); break;
+    case 4: phase_attention<WT, HD, 4>(c, layer, smem); break;
+    default: phase_attention<WT, HD, 8>(c, layer, smem); break;
+  }
+}
+
+template <typename WT>
+__device__ void run_phase(const DevCtx& c, int phase, int layer, float* smem, TcState& tc) {
+  const int T = c.ss->cur_T;
+  const size_t esz = sizeof(WT);
+  switch (phase) {
+    case PH_NORM1: phase_norm<WT>(c, layer, 0); break;
+    case PH_QKV: {
+      GemmArgs a{c.xn, c.w_base + c.w_off[1] + (size_t)layer * c.qkv_dim * c.d * esz, c.qkv, T, c.qkv_dim, c.d,
+                 c.qkv_dim, 0};
+      gemm_dispatch<WT>(c, a, GEMM_QKV, layer, smem, tc);
+    } break;
+    case PH_ROPE: phase_rope_kv<WT>(c, layer); break;
+    case PH_ATTN:
+      if (c.hd == 64) attention_dispatch<WT, 64>(c, layer, smem);
+      else attention_dispatch<WT, 128>(c, layer, smem);
+      break;
+    case PH_O: {
+      GemmArgs a{c.attn, c.w_base + c.w_off[2] + (size_t)layer * c.d * c.q_dim * esz, c.h, T, c.d, c.q_dim, c.d, 1};
+      gemm_dispatch<WT>(c, a, GEMM_O, layer, smem, tc);
+    } break;
+    case PH_NORM2: phase_norm<WT>(c, layer, 1); break;
+    case PH_GU: {
+      GemmArgs a{c.xn, c.w_base + c.w_off[3] + (size_t)layer * 2 * c.F * c.d * esz, c.gu, T, 2 * c.F, c.d, 2 * c.F, 0};
+      gemm_dispatch<WT>(c, a, GEMM_GU, layer, smem, tc);
+    } break;
+    case PH_SILU: phase_silu_mul<WT>(c); break;
+    case PH_DOWN: {
+      GemmArgs a{c.act, c.w_base + c.w_off[4] + (size_t)layer * c.d * c.F * esz, c.h, T, c.d, c.F, c.d, 1};
+      gemm_dispatch<WT>(c, a, GEMM_DOWN, layer, smem, tc);
+    } break;
+    case PH_FNORM: phase_final_norm<WT>(c); break;
+    case PH_LMHEAD: {
+      GemmArgs a{c.xs, c.w_base + c.w_off[9], c.logits, c.ss->cur_rows, c.V, c.d, c.V, 0};
+      gemm_dispatch<WT>(c, a, GEMM_LMHEAD, 0, smem, tc);
+    } break;
+    case PH_SAMPLE: phase_sample(c, smem); break;
+    default: break;
+  }
+}
+
+// ---- persistent loop -----------------------------------------------------------------
+template <typename WT>
+__global__ void __launch_bounds__(FWD_THREADS, 1) blink_loop_kernel(const __grid_constant__ DevCtx c) {
+  extern __shared__ __align__(1024) float smem[];
+  unsigned int gen = 0;
+  if (threadIdx.x == 0) gen = ld_acquire_gpu_u32(&c.ss->bar_gen);
+  long long launch_iters = 0;
+  TcState tc;
+  tc_init(c, smem, tc);
+  while (true) {
+    if (blockIdx.x == 0) control_phase(c, launch_iters);
+    if (!grid_barrier(c, gen)) break;
+    if (*(volatile int*)&c.ss->cmd != CMD_RUN) break;
+    if (!c.control_only) {
+      bool ok = true;
+      for (int layer = 0; layer < c.L && ok; ++layer) {
+        for (int ph = PH_NORM1; ph <= PH_DOWN && ok; ++ph) {
+          run_phase<WT>(c, ph, layer, smem, tc);
+          ok = grid_barrier(c, gen);
+        }
+      }
+      for (int ph = PH_FNORM; ph <= PH_SAMPLE && ok; ++ph) {
+        run_phase<WT>(c, ph, 0, smem, tc);
+        if (ph != PH_SAMPLE) ok = grid_barrier(c, gen);
+      }
+      if (!ok) break;
+    }
+    if (!grid_barrier(c, gen)) break;
+  }
+  tc_fini(c, tc);
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    const int aborted = *(volatile int*)&c.ss->abort_flag;
+    __threadfence_system();
+    c.mbox->loop_state = aborted ? (uint32_t)BLINK_LOOP_EXIT_ERROR : (uint32_t)c.ss->exit_reason;
+    __threadfence_system();
+  }
+}
+
+// ---- stepped mode ----------------------------------------------------------------------
+__global__ void __launch_bounds__(CTRL_THREADS, 1) blink_control_kernel(const __grid_constant__ DevCtx c, int post_only) {
+  if (post_only) {
+    if (c.ss->pending_post) post_step(c);
+    if (threadIdx.x == 0) c.ss->cmd = CMD_NONE;
+    return;
+  }
+  long long li = 0;
+  control_phase(c, li);
+}
+
+template <typename WT>
+__global__ void __launch_bounds__(FWD_THREADS, 1) blink_phase_kernel(const __grid_constant__ DevCtx c, int phase, int layer) {
+  extern __shared__ __align__(1024) float smem[];
+  if (c.ss->cmd != CMD_RUN) return;
+  TcState tc;
+  tc_init(c, smem, tc);
+  run_phase<WT>(c, phase, layer, smem, tc);
+  tc_fini(c, tc);
+}
+
+// Sampler alone over caller-provided logits (one CTA per row).
+__global__ void __launch_bounds__(FWD_THREADS, 1)
+blink_sample_kernel(const float* logits, int rows, int V, const int* top_k, const float* temp,
+                    const unsigned long long* ticket, const int* gen_index, const unsigned long long* seed, int* out) {
+  extern __shared__ __align__(1024) float smem[];
+  for (int r = blockIdx.x; r < rows; r += gridDim.x) {
+    const int tok = sample_row(logits + (size_t)r * V, V, min(top_k[r], MAX_TOPK), temp[r], ticket[r], gen_index[r],
+                               seed[r], smem);
+    if (threadIdx.x == 0) out[r] = tok;
+  }
+}
+
+__global__ void blink_clock_probe_kernel(Mailbox* mb) {
+  mb->clock_probe = global_timer_ns();
+  __threadfence_system();
+}
+
+}  // namespace blink
+
+// =========================================================================================
+// Host side
+// =========================================================================================
+using namespace blink;
+
+namespace {
+
+uint64_t now_ns() {
+  timespec ts;
+  clock_gettime(CLOCK_MONOTONIC, &ts);
+  return (uint64_t)ts.tv_sec * 1000000000ull + (uint64_t)ts.tv_nsec;
+}
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct Layout {
+  uint64_t off[10];
+  uint64_t total;
+};
+
+bool model_ok(const blink_model_cfg* m) {
+  if (!m || m->size != sizeof(blink_model_cfg)) return false;
+  if (m->n_layers < 1 || m->d_model < 16 || m->n_q_heads < 1 || m->n_kv_heads < 1 || m->vocab < 2 || m->d_ff < 16)
+    return false;
+  if (m->head_dim != 64 && m->head_dim != 128) return false;
+  if (m->n_q_heads % m->n_kv_heads) return false;
+  const int rep = m->n_q_heads / m->n_kv_heads;
+  if (rep != 1 && rep != 2 && rep != 4 && rep != 8) return false;
+  if (m->dtype != BLINK_DTYPE_BF16 && m->dtype != BLINK_DTYPE_FP32) return false;
+  if (m->n_experts < 0 || (m->n_experts > 0 && (m->top_k_experts < 1 || m->top_k_experts > m->n_experts))) return false;
+  if (m->d_model % 8 || m->d_ff % 8) return false;
+  return true;
+}
+
+Layout weight_layout(const blink_model_cfg* m) {
+  Layout lo;
+  const uint64_t esz = m->dtype == BLINK_DTYPE_BF16 ? 2 : 4;
+  const uint64_t L = m->n_layers, d = m->d_model, V = m->vocab, F = m->d_ff;
+  const uint64_t qd = (uint64_t)m->n_q_heads * m->head_dim, kvd = (uint64_t)m->n_kv_heads * m->head_dim;
+  const uint64_t E1 = m->n_experts > 0 ? m->n_experts : 1, E = m->n_experts;
+  const uint64_t n[10] = {V * d, L * (qd + 2 * kvd) * d, L * d * qd, L * E1 * 2 * F * d, L * E1 * d * F,
+                          L * E * d, L * d, L * d, d, V * d};
+  const uint64_t es[10] = {esz, esz, esz, esz, esz, 4, 4, 4, 4, esz};
+  uint64_t off = 0;
+  for (int i = 0; i < 10; ++i) {
+    lo.off[i] = off;
+    off += align_up(n[i] * es[i], 256);
+  }
+  lo.total = off;
+  return lo;
+}
+
+}  // namespace
+
+struct SlotInfo {
+  uint64_t ticket = 0, user_tag = 0, t_submit_ns = 0;
+  int32_t max_new = 0, consumed = 0;
+  bool busy = false;
+};
+
+struct blink_ctx {
+  DevCtx dc;
+  blink_model_cfg model;
+  blink_sched_cfg sched;
+  cudaStream_t stream = nullptr, copy_stream = nullptr;
+  std::vector<void*> dev_allocs, host_allocs;
+  Mailbox* mbox = nullptr;       // host view
+  SubEntry* sub_q = nullptr;
+  int32_t *sub_tokens = nullptr, *sub_forced = nullptr, *out_tokens = nullptr;
+  uint64_t* out_time = nullptr;
+  uint32_t* out_count = nullptr;
+  std::mutex mu;
+  std::vector<SlotInfo> slots;
+  std::deque<int> active;
+  int hint = 0;
+  uint64_t next_ticket = 0;
+  int64_t launches = 0;
+  int64_t clock_offset = 0;
+  bool final_stop = false;
+  int n_sms = 1;
+  size_t smem_bytes = 0;
+  int grid = 1;
+  TcHost tc_host;
+};
+
+namespace {
+
+template <typename T>
+int dev_alloc(blink_ctx* x, T** p, size_t n, bool zero = true) {
+  void* q = nullptr;
+  if (cudaMalloc(&q, n * sizeof(T) > 0 ? n * sizeof(T) : 16) != cudaSuccess) return BLINK_ENOMEM;
+  if (zero && cudaMemset(q, 0, n * sizeof(T) > 0 ? n * sizeof(T) : 16) != cudaSuccess) return BLINK_ECUDA;
+  x->dev_allocs.push_back(q);
+  *p = reinterpret_cast<T*>(q);
+  return BLINK_OK;
+}
+
+template <typename T>
+int pinned_alloc(blink_ctx* x, T** host, T** dev, size_t n) {
+  void* q = nullptr;
+  const size_t bytes = n * sizeof(T) > 0 ? n * sizeof(T) : 16;
+  if (cudaHostAlloc(&q, bytes, cudaHostAllocMapped | cudaHostAllocPortable) != cudaSuccess) return BLINK_ENOMEM;
+  memset(q, 0, bytes);
+  void* d = nullptr;
+  if (cudaHostGetDevicePointer(&d, q, 0) != cudaSuccess) return BLINK_ECUDA;
+  x->host_allocs.push_back(q);
+  *host = reinterpret_cast<T*>(q);
+  *dev = reinterpret_cast<T*>(d);
+  return BLINK_OK;
+}
+
+void free_all(blink_ctx* x) {
+  for (void* p : x->dev_allocs) cudaFree(p);
+  for (void* p : x->host_allocs) cudaFreeHost(p);
+  x->dev_allocs.clear();
+  x->host_allocs.clear();
+  tc_host_free(x->tc_host);
+  if (x->stream) cudaStreamDestroy(x->stream);
+  if (x->copy_stream) cudaStreamDestroy(x->copy_stream);
+  x->stream = x->copy_stream = nullptr;
+}
+
+size_t phase_smem_bytes(const blink_ctx* x) {
+  size_t a = sizeof(float) * (size_t)ATTN_SMEM_FLOATS(x->dc.hd, x->dc.n_rep);
+  size_t s = sizeof(float) * (size_t)SAMPLE_SMEM_FLOATS;
+  size_t m = a > s ? a : s;
+  if (x->dc.gemm_tc && tc_smem_bytes() > m) m = tc_smem_bytes();
+  return m;
+}
+
+int launch_loop(blink_ctx* x) {
+  x->mbox->stop = 0;
+  x->mbox->loop_state = BLINK_LOOP_RUNNING;
+  std::atomic_thread_fence(std::memory_order_seq_cst);
+  void* args[] = {(void*)&x->dc};
+  const void* fn = x->dc.dtype == BLINK_DTYPE_BF16 ? (const void*)blink_loop_kernel<__nv_bfloat16>
+                                                    : (const void*)blink_loop_kernel<float>;
+  cudaError_t e = cudaLaunchCooperativeKernel(fn, dim3(x->grid), dim3(FWD_THREADS), args, x->smem_bytes, x->stream);
+  if (e != cudaSuccess) {
+    x->mbox->loop_state = BLINK_LOOP_EXIT_ERROR;
+    fprintf(stderr, "blink: persistent launch failed: %s\n", cudaGetErrorString(e));
+    return BLINK_ECUDA;
+  }
+  x->launches += 1;
+  return BLINK_OK;
+}
+
+// Re-instantiate a loop that left the GPU while work is outstanding (caller holds mu).
+int pump(blink_ctx* x) {
+  if (x->dc.stepped) return BLINK_OK;
+  const uint32_t st = x->mbox->loop_state;
+  if (st == BLINK_LOOP_RUNNING) return BLINK_OK;
+  if (st == BLINK_LOOP_EXIT_ERROR) return BLINK_EDEVICE;
+  if (x->final_stop) return BLINK_ESTOPPED;
+  const bool work = !x->active.empty();
+  if (!work && st != BLINK_LOOP_NOT_STARTED) return BLINK_OK;
+  if (cudaStreamSynchronize(x->stream) != cudaSuccess) return BLINK_ECUDA;
+  return launch_loop(x);
+}
+
+template <typename WT>
+void launch_phase(blink_ctx* x, int phase, int layer) {
+  blink_phase_kernel<WT><<<x->grid, FWD_THREADS, x->smem_bytes, x->stream>>>(x->dc, phase, layer);
+  x->launches += 1;
+}
+
+template <typename WT>
+int step_once(blink_ctx* x) {
+  blink_control_kernel<<<1, CTRL_THREADS, 0, x->stream>>>(x->dc, 0);
+  x->launches += 1;
+  if (!x->dc.control_only) {
+    for (int l = 0; l < x->dc.L; ++l)
+      for (int ph = PH_NORM1; ph <= PH_DOWN; ++ph) launch_phase<WT>(x, ph, l);
+    for (int ph = PH_FNORM; ph <= PH_SAMPLE; ++ph) launch_phase<WT>(x, ph, 0);
+  }
+  return cudaGetLastError() == cudaSuccess ? BLINK_OK : BLINK_ECUDA;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* blink_strerror(int code) {
+  switch (code) {
+    case BLINK_OK: return "ok";
+    case BLINK_EAGAIN: return "no empty ring slot (back-pressure)";
+    case BLINK_EINVAL: return "invalid argument";
+    case BLINK_ESTOPPED: return "loop stopped";
+    case BLINK_EDEVICE: return "device loop reported an error";
+    case BLINK_ETIMEDOUT: return "timed out";
+    case BLINK_ENOMEM: return "out of memory or pool too small";
+    case BLINK_ECUDA: return "CUDA call failed";
+    default: return "unknown error";
+  }
+}
+
+uint64_t blink_weights_bytes(const blink_model_cfg* cfg) {
+  if (!model_ok(cfg)) return 0;
+  return weight_layout(cfg).total;
+}
+
+uint64_t blink_weight_offset(const blink_model_cfg* cfg, int tensor_id) {
+  if (!model_ok(cfg) || tensor_id < 0 || tensor_id > 9) return UINT64_MAX;
+  return weight_layout(cfg).off[tensor_id];
+}
+
+int64_t blink_kv_blocks_for_bytes(const blink_model_cfg* cfg, int block_size, uint64_t bytes) {
+  if (!model_ok(cfg) || block_size < 1) return BLINK_EINVAL;
+  const uint64_t esz = cfg->dtype == BLINK_DTYPE_BF16 ? 2 : 4;
+  const uint64_t per = (uint64_t)cfg->n_layers * 2 * cfg->n_kv_heads * block_size * cfg->head_dim * esz;
+  return (int64_t)(bytes / per);
+}
+
+int blink_sample(const float* logits, int rows, int vocab, const int32_t* top_k, const float* temperature,
+                 const uint64_t* ticket, const int32_t* gen_index, const uint64_t* seed, int32_t* out) {
+  if (!logits || rows < 1 || vocab < 2 || !top_k || !temperature || !ticket || !gen_index || !seed || !out)
+    return BLINK_EINVAL;
+  for (int r = 0; r < rows; ++r)
+    if (top_k[r] < 0 || top_k[r] > MAX_TOPK || (top_k[r] > 0 && !(temperature[r] > 0.f))) return BLINK_EINVAL;
+  char* d = nullptr;
+  const size_t n = (size_t)rows;
+  const size_t bytes = n * (4 + 4 + 8 + 4 + 8 + 4);
+  if (cudaMalloc(&d, bytes) != cudaSuccess) return BLINK_ENOMEM;
+  unsigned long long* d_ticket = (unsigned long long*)d;
+  unsigned long long* d_seed = d_ticket + n;
+  int* d_topk = (int*)(d_seed + n);
+  float* d_temp = (float*)(d_topk + n);
+  int* d_gen = (int*)(d_temp + n);
+  int* d_out = d_gen + n;
+  int rc = BLINK_OK;
+  if (cudaMemcpy(d_ticket, ticket, n * 8, cudaMemcpyHostToDevice) != cudaSuccess ||
+      cudaMemcpy(d_seed, seed, n * 8, cudaMemcpyHostToDevice) != cudaSuccess ||
+      cudaMemcpy(d_topk, top_k, n * 4, cudaMemcpyHostToDevice) != cudaSuccess ||
+      cudaMemcpy(d_temp, temperature, n * 4, cudaMemcpyHostToDevice) != cudaSuccess ||
+      cudaMemcpy(d_gen, gen_index, n * 4, cudaMemcpyHostToDevice) != cudaSuccess)
+    rc = BLINK_ECUDA;
+  if (rc == BLINK_OK) {
+    const int grid = rows < 1184 ? rows : 1184;
+    blink_sample_kernel<<<grid, FWD_THREADS, SAMPLE_SMEM_FLOATS * sizeof(float)>>>(
+        logits, rows, vocab, d_topk, d_temp, d_ticket, d_gen, d_seed, d_out);
+    if (cudaDeviceSynchronize() != cudaSuccess) rc = BLINK_ECUDA;
+    else if (cudaMemcpy(out, d_out, n * 4, cudaMemcpyDeviceToHost) != cudaSuccess) rc = BLINK_ECUDA;
+  }
+  cudaFree(d);
+  return rc;
+}
+
+int blink_create(const blink_model_cfg* model, const blink_sched_cfg* sched, const blink_kv_pool* kv,
+                 blink_ctx** out) {
+  if (!out) return BLINK_EINVAL;
+  *out = nullptr;
+  if (!model_ok(model) || !sched || sched->size != sizeof(blink_sched_cfg) || !kv || kv->size != sizeof(blink_kv_pool))
+    return BLINK_EINVAL;
+  if (sched->max_batch < 1 || sched->max_batch > MAX_BATCH || sched->prefill_chunk_tokens < 1 || sched->n_slots < 1 ||
+      sched->max_prompt < 1 || sched->max_new < 1)
+    return BLINK_EINVAL;
+  if (kv->block_size != 16) return BLINK_EINVAL;
+  if (!sched->control_only && (model->weights == nullptr || model->weights_bytes < blink_weights_bytes(model)))
+    return BLINK_EINVAL;
+  if (model->n_experts > 0 && !sched->control_only) return BLINK_EINVAL;  // routed experts: not built yet
+  if (((uintptr_t)kv->base & 255) || ((uintptr_t)model->weights & 255)) return BLINK_EINVAL;
+  int dev_count = 0;
+  if (cudaGetDeviceCount(&dev_count) != cudaSuccess || dev_count < 1) return BLINK_ECUDA;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return BLINK_ECUDA;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return BLINK_ECUDA;
+  if (prop.major != 10) {
+    fprintf(stderr, "blink: built for sm_100a, device is sm_%d%d\n", prop.major, prop.minor);
+    return BLINK_ECUDA;
+  }
+  const int64_t nb = blink_kv_blocks_for_bytes(model, kv->block_size, kv->bytes);
+  if (nb < 1 || (!sched->control_only && kv->base == nullptr)) return BLINK_ENOMEM;
+
+  blink_ctx* x = new (std::nothrow) blink_ctx();
+  if (!x) return BLINK_ENOMEM;
+  x->model = *model;
+  x->sched = *sched;
+  x->n_sms = prop.multiProcessorCount;
+  DevCtx& c = x->dc;
+  memset(&c, 0, sizeof(c));
+  c.L = model->n_layers; c.d = model->d_model; c.Hq = model->n_q_heads; c.Hkv = model->n_kv_heads;
+  c.hd = model->head_dim; c.F = model->d_ff; c.V = model->vocab; c.E = model->n_experts; c.topE = model->top_k_experts;
+  c.dtype = model->dtype;
+  c.q_dim = c.Hq * c.hd; c.kv_dim = c.Hkv * c.hd; c.qkv_dim = c.q_dim + 2 * c.kv_dim; c.n_rep = c.Hq / c.Hkv;
+  c.rope_theta = model->rope_theta; c.rms_eps = model->rms_eps; c.attn_scale = 1.0f / sqrtf((float)c.hd);
+  c.w_base = reinterpret_cast<const char*>(model->weights);
+  const Layout lo = weight_layout(model);
+  for (int i = 0; i < 10; ++i) c.w_off[i] = lo.off[i];
+  c.MB = sched->max_batch; c.chunk = sched->prefill_chunk_tokens; c.n_slots = sched->n_slots;
+  c.max_prompt = sched->max_prompt; c.max_new = sched->max_new; c.Tmax = c.MB + c.chunk; c.bs = kv->block_size;
+  c.n_blocks = (int)(nb > 0x7fffffff ? 0x7fffffff : nb);
+  c.max_pos = c.max_prompt + c.max_new;
+  c.max_blocks_seq = (c.max_pos + c.bs - 1) / c.bs;
+  c.control_only = sched->control_only; c.start_paused = sched->start_paused;
+  c.stepped = sched->exec_mode == BLINK_EXEC_STEPPED;
+  c.gemm_tc = 0;
+  if (!c.control_only && model->dtype == BLINK_DTYPE_BF16 && sched->gemm_impl != BLINK_GEMM_SIMT) c.gemm_tc = tc_available();
+  if (sched->gemm_impl == BLINK_GEMM_TC && !c.gemm_tc) { delete x; return BLINK_EINVAL; }
+  c.iteration_budget = c.stepped ? 0 : sched->iteration_budget;
+  const double cyc_per_us = 2000.0;  // upper bound on the SM clock: time-outs only get longer at lower clocks
+  const int64_t idle_us = sched->idle_exit_us > 0 ? sched->idle_exit_us : 2000000;
+  c.idle_exit_cycles = (unsigned long long)(idle_us * cyc_per_us);
+  c.barrier_timeout_cycles = (unsigned long long)((idle_us + 3000000) * cyc_per_us);
+  c.kv_base = kv->base;
+  c.trace_cap = sched->trace_capacity_words;
+  c.stats_cap = sched->stats_capacity_iters;
+  c.logits_capture = sched->logits_capture;
+  c.capture_rows = sched->logits_capture ? sched->logits_capture_rows : 0;
+
+  int rc = BLINK_OK;
+  auto fail = [&](int code) { free_all(x); delete x; return code; };
+  if (cudaStreamCreateWithFlags(&x->stream, cudaStreamNonBlocking) != cudaSuccess) return fail(BLINK_ECUDA);
+  if (cudaStreamCreateWithFlags(&x->copy_stream, cudaStreamNonBlocking) != cudaSuccess) return fail(BLINK_ECUDA);
+
+#define TRY(expr) do { rc = (expr); if (rc != BLINK_OK) return fail(rc); } while (0)
+  const size_t S = c.n_slots, MB = c.MB, TM = c.Tmax;
+  const size_t esz = c.dtype == BLINK_DTYPE_BF16 ? 2 : 4;
+  TRY(dev_alloc(x, &c.slot_hot, S));
+  TRY(dev_alloc(x, &c.slot_cold, S));
+  TRY(dev_alloc(x, &c.in_arena, S * c.max_prompt, false));
+  TRY(dev_alloc(x, &c.gen_arena, S * c.max_new, false));
+  TRY(dev_alloc(x, &c.forced_arena, S * c.max_new, false));
+  TRY(dev_alloc(x, &c.ss, 1));
+  TRY(dev_alloc(x, &c.ticket_to_slot, S));
+  TRY(dev_alloc(x, &c.free_stack, (size_t)c.n_blocks, false));
+  TRY(dev_alloc(x, &c.block_table, MB * c.max_blocks_seq));
+  TRY(dev_alloc(x, &c.b_ticket, MB)); TRY(dev_alloc(x, &c.b_slot, MB)); TRY(dev_alloc(x, &c.b_P, MB));
+  TRY(dev_alloc(x, &c.b_N, MB)); TRY(dev_alloc(x, &c.b_prefilled, MB)); TRY(dev_alloc(x, &c.b_generated, MB));
+  TRY(dev_alloc(x, &c.b_phase, MB)); TRY(dev_alloc(x, &c.b_have, MB)); TRY(dev_alloc(x, &c.b_need, MB));
+  TRY(dev_alloc(x, &c.b_last, MB)); TRY(dev_alloc(x, &c.b_eos, MB)); TRY(dev_alloc(x, &c.b_topk, MB));
+  TRY(dev_alloc(x, &c.b_flags, MB)); TRY(dev_alloc(x, &c.b_temp, MB)); TRY(dev_alloc(x, &c.b_seed, MB));
+  TRY(dev_alloc(x, &c.it_bslot, MB)); TRY(dev_alloc(x, &c.it_start, MB)); TRY(dev_alloc(x, &c.it_ntok, MB));
+  TRY(dev_alloc(x, &c.it_qstart, MB)); TRY(dev_alloc(x, &c.it_row, MB));
+  TRY(dev_alloc(x, &c.tok_id, TM)); TRY(dev_alloc(x, &c.tok_pos, TM)); TRY(dev_alloc(x, &c.tok_item, TM));
+  TRY(dev_alloc(x, &c.tok_slotmap, TM));
+  TRY(dev_alloc(x, &c.row_tok, MB)); TRY(dev_alloc(x, &c.row_item, MB)); TRY(dev_alloc(x, &c.row_sampled, MB));
+  if (!c.control_only) {
+    char* p;
+    TRY(dev_alloc(x, &c.h, TM * c.d));
+    TRY(dev_alloc(x, &p, TM * c.d * esz)); c.xn = p;
+    TRY(dev_alloc(x, &c.qkv, TM * c.qkv_dim));
+    TRY(dev_alloc(x, &p, TM * c.q_dim * esz)); c.attn = p;
+    TRY(dev_alloc(x, &c.gu, TM * 2 * c.F));
+    TRY(dev_alloc(x, &p, TM * c.F * esz)); c.act = p;
+    TRY(dev_alloc(x, &p, MB * c.d * esz)); c.xs = p;
+    TRY(dev_alloc(x, &c.logits, MB * c.V));
+    TRY(dev_alloc(x, &c.rope_cos, (size_t)c.max_pos * (c.hd / 2), false));
+    TRY(dev_alloc(x, &c.rope_sin, (size_t)c.max_pos * (c.hd / 2), false));
+    std::vector<float> cs((size_t)c.max_pos * (c.hd / 2)), sn(cs.size());
+    for (int i = 0; i < c.hd / 2; ++i) {
+      const double inv = std::pow((double)c.rope_theta, -2.0 * i / c.hd);
+      for (int p2 = 0; p2 < c.max_pos; ++p2) {
+        cs[(size_t)p2 * (c.hd / 2) + i] = (float)std::cos(p2 * inv);
+        sn[(size_t)p2 * (c.hd / 2) + i] = (float)std::sin(p2 * inv);
+      }
+    }
+    if (cudaMemcpy(c.rope_cos, cs.data(), cs.size() * 4, cudaMemcpyHostToDevice) != cudaSuccess) return fail(BLINK_ECUDA);
+    if (cudaMemcpy(c.rope_sin, sn.data(), sn.size() * 4, cudaMemcpyHostToDevice) != cudaSuccess) return fail(BLINK_ECUDA);
+  }
+  if (c.trace_cap > 0) TRY(dev_alloc(x, &c.trace, (size_t)c.trace_cap, false));
+  if (c.stats_cap > 0) TRY(dev_alloc(x, &c.stats, (size_t)c.stats_cap));
+  // free stack: pop takes from the top; first pops return 0, 1, 2, ...
+  {
+    std::vector<int32_t> st((size_t)c.n_blocks);
+    for (int i = 0; i < c.n_blocks; ++i) st[(size_t)c.n_blocks - 1 - i] = i;
+    if (cudaMemcpy(c.free_stack, st.data(), st.size() * 4, cudaMemcpyHostToDevice) != cudaSuccess) return fail(BLINK_ECUDA);
+    SchedState s0;
+    memset(&s0, 0, sizeof(s0));
+    s0.free_top = c.n_blocks;
+    s0.cur_hdr = -1;
+    if (cudaMemcpy(c.ss, &s0, sizeof(s0), cudaMemcpyHostToDevice) != cudaSuccess) return fail(BLINK_ECUDA);
+  }
+  // pinned mailboxes
+  {
+    Mailbox* md; SubEntry* qd; int32_t *td, *fd, *od; uint64_t* tmd; uint32_t* cd;
+    TRY(pinned_alloc(x, &x->mbox, &md, 1)); c.mbox = md;
+    TRY(pinned_alloc(x, &x->sub_q, &qd, S)); c.sub_q = qd;
+    TRY(pinned_alloc(x, &x->sub_tokens, &td, S * c.max_prompt)); c.sub_tokens = td;
+    TRY(pinned_alloc(x, &x->sub_forced, &fd, S * c.max_new)); c.sub_forced = fd;
+    TRY(pinned_alloc(x, &x->out_tokens, &od, S * c.max_new)); c.out_tokens = od;
+    TRY(pinned_alloc(x, &x->out_time, &tmd, S * c.max_new)); c.out_time = tmd;
+    TRY(pinned_alloc(x, &x->out_count, &cd, S)); c.out_count = cd;
+  }
+  if (c.gemm_tc) TRY(tc_host_setup(x->tc_host, c));
+#undef TRY
+  x->slots.resize(S);
+
+  // clock calibration: host CLOCK_MONOTONIC vs device global timer
+  {
+    const uint64_t t0 = now_ns();
+    blink_clock_probe_kernel<<<1, 1, 0, x->stream>>>(c.mbox);
+    if (cudaStreamSynchronize(x->stream) != cudaSuccess) return fail(BLINK_ECUDA);
+    const uint64_t t1 = now_ns();
+    x->clock_offset = (int64_t)((t0 + t1) / 2) - (int64_t)x->mbox->clock_probe;
+  }
+
+  x->smem_bytes = phase_smem_bytes(x);
+  x->grid = c.control_only ? 1 : x->n_sms;
+  const void* loop_fn = c.dtype == BLINK_DTYPE_BF16 ? (const void*)blink_loop_kernel<__nv_bfloat16>
+                                                     : (const void*)blink_loop_kernel<float>;
+  const void* ph_fn = c.dtype == BLINK_DTYPE_BF16 ? (const void*)blink_phase_kernel<__nv_bfloat16>
+                                                   : (const void*)blink_phase_kernel<float>;
+  if (cudaFuncSetAttribute(loop_fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)x->smem_bytes) != cudaSuccess ||
+      cudaFuncSetAttribute(ph_fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)x->smem_bytes) != cudaSuccess)
+    return fail(BLINK_ECUDA);
+  int occ = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, loop_fn, FWD_THREADS, x->smem_bytes) != cudaSuccess || occ < 1)
+    return fail(BLINK_ECUDA);
+  if (cudaDeviceSynchronize() != cudaSuccess) return fail(BLINK_ECUDA);
+  if (!c.stepped) {
+    rc = launch_loop(x);
+    if (rc != BLINK_OK) return fail(rc);
+  } else {
+    x->mbox->loop_state = BLINK_LOOP_NOT_STARTED;
+  }
+  *out = x;
+  return BLINK_OK;
+}
+
+int blink_start(blink_ctx* x) {
+  if (!x) return BLINK_EINVAL;
+  std::lock_guard<std::mutex> g(x->mu);
+  std::atomic_thread_fence(std::memory_order_seq_cst);
+  x->mbox->start = 1;
+  return pump(x) == BLINK_EDEVICE ? BLINK_EDEVICE : BLINK_OK;
+}
+
+int blink_submit(blink_ctx* x, const blink_request* r, uint64_t* ticket_out) {
+  if (!x || !r || r->size != sizeof(blink_request) || !r->prompt) return BLINK_EINVAL;
+  const DevCtx& c = x->dc;
+  if (r->n_prompt < 1 || r->n_prompt > c.max_prompt || r->max_new_tokens < 1 || r->max_new_tokens > c.max_new)
+    return BLINK_EINVAL;
+  if (r->top_k < 0 || r->top_k > MAX_TOPK || (r->top_k > 0 && !(r->temperature > 0.f))) return BLINK_EINVAL;
+  if (r->eos_id >= c.V) return BLINK_EINVAL;
+  for (int i = 0; i < r->n_prompt; ++i)
+    if (r->prompt[i] < 0 || r->prompt[i] >= c.V) return BLINK_EINVAL;
+  if (r->forced_tokens)
+    for (int i = 0; i < r->max_new_tokens; ++i)
+      if (r->forced_tokens[i] < 0 || r->forced_tokens[i] >= c.V) return BLINK_EINVAL;
+  const long long need = ((long long)r->n_prompt + r->max_new_tokens - 1 + c.bs - 1) / c.bs;
+  if (need > c.n_blocks) return BLINK_EINVAL;  // could never be admitted: would block the queue for good
+
+  std::lock_guard<std::mutex> g(x->mu);
+  if (x->final_stop) return BLINK_ESTOPPED;
+  if (x->mbox->loop_state == BLINK_LOOP_EXIT_ERROR || x->mbox->device_status > 0) {
+    if (x->mbox->device_status != DEV_ERR_TRACE_OVERFLOW) return BLINK_EDEVICE;
+  }
+  // slot tracker: circular scan from a hint over the local availability cache
+  int slot = -1;
+  for (int k = 0; k < c.n_slots; ++k) {
+    const int s = (x->hint + k) % c.n_slots;
+    if (!x->slots[s].busy) { slot = s; break; }
+  }
+  if (slot < 0) return BLINK_EAGAIN;
+  x->hint = (slot + 1) % c.n_slots;
+  const uint64_t ticket = x->next_ticket++;
+  memcpy(x->sub_tokens + (size_t)slot * c.max_prompt, r->prompt, (size_t)r->n_prompt * 4);
+  if (r->forced_tokens) memcpy(x->sub_forced + (size_t)slot * c.max_new, r->forced_tokens, (size_t)r->max_new_tokens * 4);
+  x->out_count[slot] = 0;
+  SubEntry& e = x->sub_q[ticket % (uint64_t)c.n_slots];
+  e.ticket = ticket; e.seed = r->seed; e.user_tag = r->user_tag; e.slot = (uint32_t)slot;
+  e.n_prompt = (uint32_t)r->n_prompt; e.max_new = (uint32_t)r->max_new_tokens; e.top_k = (uint32_t)r->top_k;
+  e.temperature = r->temperature; e.eos_id = r->eos_id; e.flags = r->forced_tokens ? REQ_FLAG_FORCED : 0; e.pad = 0;
+  SlotInfo& si = x->slots[slot];
+  si.busy = true; si.ticket = ticket; si.user_tag = r->user_tag; si.max_new = r->max_new_tokens; si.consumed = 0;
+  si.t_submit_ns = now_ns();
+  x->active.push_front(slot);  // new slots are looked at first by the token reader
+  // payload first, then the tail that makes it visible
+  std::atomic_thread_fence(std::memory_order_release);
+  __atomic_store_n((uint64_t*)&x->mbox->sub_tail, ticket + 1, __ATOMIC_RELEASE);
+  if (ticket_out) *ticket_out = ticket;
+  const int prc = pump(x);
+  return prc == BLINK_EDEVICE ? BLINK_EDEVICE : BLINK_OK;
+}
+
+int blink_poll(blink_ctx* x, blink_token_event* out, int max_events, int timeout_us) {
+  if (!x || !out || max_events < 1) return BLINK_EINVAL;
+  const DevCtx& c = x->dc;
+  const uint64_t deadline = now_ns() + (uint64_t)(timeout_us > 0 ? timeout_us : 0) * 1000ull;
+  while (true) {
+    int n = 0;
+    {
+      std::lock_guard<std::mutex> g(x->mu);
+      const int prc = pump(x);
+      if (prc == BLINK_EDEVICE) return BLINK_EDEVICE;
+      const uint64_t t_now = now_ns();
+      for (auto it = x->active.begin(); it != x->active.end() && n < max_events;) {
+        const int slot = *it;
+        SlotInfo& si = x->slots[slot];
+        const uint32_t cnt = __atomic_load_n(&x->out_count[slot], __ATOMIC_ACQUIRE);
+        const int have = (int)(cnt & 0x7fffffffu);
+        const bool fin = (cnt >> 31) != 0;
+        while (si.consumed < have && n < max_events) {
+          blink_token_event& ev = out[n++];
+          const size_t idx = (size_t)slot * c.max_new + si.consumed;
+          ev.ticket = si.ticket; ev.user_tag = si.user_tag; ev.index = si.consumed;
+          ev.token = x->out_tokens[idx];
+          ev.is_first = si.consumed == 0;
+          ev.is_last = fin && si.consumed + 1 == have;
+          ev.t_device_ns = x->out_time[idx];
+          ev.t_host_ns = t_now;
+          ev.t_submit_ns = si.t_submit_ns;
+          si.consumed += 1;
+        }
+        if (fin && si.consumed == have) {
+          si.busy = false;  // DECODE_COMPLETED -> EMPTY: the frontend owns this transition
+          it = x->active.erase(it);
+        } else {
+          ++it;
+        }
+      }
+    }
+    if (n > 0 || now_ns() >= deadline) return n;
+    std::this_thread::sleep_for(std::chrono::microseconds(20));
+  }
+}
+
+int blink_step(blink_ctx* x, int n_iterations) {
+  if (!x || n_iterations < 0) return BLINK_EINVAL;
+  if (!x->dc.stepped) return BLINK_EINVAL;
+  std::lock_guard<std::mutex> g(x->mu);
+  for (int i = 0; i < n_iterations; ++i) {
+    const int rc = x->dc.dtype == BLINK_DTYPE_BF16 ? step_once<__nv_bfloat16>(x) : step_once<float>(x);
+    if (rc != BLINK_OK) return rc;
+  }
+  blink_control_kernel<<<1, CTRL_THREADS, 0, x->stream>>>(x->dc, 1);
+  x->launches += 1;
+  if (cudaStreamSynchronize(x->stream) != cudaSuccess) return BLINK_ECUDA;
+  return x->mbox->device_status > 0 && x->mbox->device_status != DEV_ERR_TRACE_OVERFLOW ? BLINK_EDEVICE : BLINK_OK;
+}
+
+int blink_stop(blink_ctx* x, int final, int timeout_ms) {
+  if (!x) return BLINK_EINVAL;
+  std::lock_guard<std::mutex> g(x->mu);
+  if (final) x->final_stop = true;
+  if (x->dc.stepped) return cudaStreamSynchronize(x->stream) == cudaSuccess ? BLINK_OK : BLINK_ECUDA;
+  const uint64_t deadline = now_ns() + (uint64_t)(timeout_ms > 0 ? timeout_ms : 0) * 1000000ull;
+  if (x->mbox->loop_state == BLINK_LOOP_RUNNING) {
+    std::atomic_thread_fence(std::memory_order_seq_cst);
+    x->mbox->stop = 1;
+  }
+  while (true) {
+    const cudaError_t q = cudaStreamQuery(x->stream);
+    if (q == cudaSuccess) break;
+    if (q != cudaErrorNotReady) return BLINK_ECUDA;
+    if (now_ns() >= deadline) return BLINK_ETIMEDOUT;
+    std::this_thread::sleep_for(std::chrono::microseconds(50));
+  }
+  return BLINK_OK;
+}
+
+int blink_destroy(blink_ctx* x, int timeout_ms) {
+  if (!x) return BLINK_EINVAL;
+  const int rc = blink_stop(x, 1, timeout_ms);
+  if (rc == BLINK_ETIMEDOUT) return rc;
+  free_all(x);
+  delete x;
+  return rc == BLINK_ECUDA ? BLINK_ECUDA : BLINK_OK;
+}
+
+static int read_ss(blink_ctx* x, SchedState* s) {
+  if (cudaMemcpyAsync(s, x->dc.ss, sizeof(SchedState), cudaMemcpyDeviceToHost, x->copy_stream) != cudaSuccess) return BLINK_ECUDA;
+  if (cudaStreamSynchronize(x->copy_stream) != cudaSuccess) return BLINK_ECUDA;
+  return BLINK_OK;
+}
+
+int blink_get_stats(blink_ctx* x, blink_stats* out) {
+  if (!x || !out || out->size != sizeof(blink_stats)) return BLINK_EINVAL;
+  std::lock_guard<std::mutex> g(x->mu);
+  SchedState s;
+  const int rc = read_ss(x, &s);
+  if (rc != BLINK_OK) return rc;
+  out->loop_state = (int32_t)x->mbox->loop_state;
+  out->device_status = x->mbox->device_status;
+  out->n_blocks = x->dc.n_blocks;
+  out->iterations = (int64_t)s.iter;
+  out->launches = x->launches;
+  out->tokens_out = (int64_t)s.tokens_out;
+  out->prompt_tokens = (int64_t)s.prompt_tokens;
+  out->trace_words = s.trace_pos;
+  out->device_clock_offset_ns = x->clock_offset;
+  out->free_blocks = s.free_top;
+  out->reserved_blocks = s.reserved;
+  std::vector<int32_t> ph((size_t)x->dc.MB);
+  if (cudaMemcpyAsync(ph.data(), x->dc.b_phase, ph.size() * 4, cudaMemcpyDeviceToHost, x->copy_stream) != cudaSuccess ||
+      cudaStreamSynchronize(x->copy_stream) != cudaSuccess)
+    return BLINK_ECUDA;
+  int live = 0;
+  for (int v : ph) live += v != PHASE_FREE;
+  out->batch_live = live;
+  out->reserved1 = 0;
+  return BLINK_OK;
+}
+
+int blink_get_trace(blink_ctx* x, int32_t* out, int64_t capacity, int64_t* n_words) {
+  if (!x || !n_words || capacity < 0 || (capacity > 0 && !out)) return BLINK_EINVAL;
+  std::lock_guard<std::mutex> g(x->mu);
+  SchedState s;
+  const int rc = read_ss(x, &s);
+  if (rc != BLINK_OK) return rc;
+  *n_words = s.trace_pos;
+  const int64_t n = s.trace_pos < capacity ? s.trace_pos : capacity;
+  if (n > 0) {
+    if (cudaMemcpyAsync(out, x->dc.trace, (size_t)n * 4, cudaMemcpyDeviceToHost, x->copy_stream) != cudaSuccess ||
+        cudaStreamSynchronize(x->copy_stream) != cudaSuccess)
+      return BLINK_ECUDA;
+  }
+  return BLINK_OK;
+}
+
+int blink_get_iter_stats(blink_ctx* x, blink_iter_stat* out, int64_t capacity, int64_t* n_records) {
+  if (!x || !n_records || capacity < 0 || (capacity > 0 && !out)) return BLINK_EINVAL;
+  static_assert(sizeof(blink_iter_stat) == sizeof(IterStat), "iter stat layout");
+  std::lock_guard<std::mutex> g(x->mu);
+  SchedState s;
+  const int rc = read_ss(x, &s);
+  if (rc != BLINK_OK) return rc;
+  int64_t have = (int64_t)s.iter < x->dc.stats_cap ? (int64_t)s.iter : x->dc.stats_cap;
+  *n_records = have;
+  const int64_t n = have < capacity ? have : capacity;
+  if (n > 0) {
+    if (cudaMemcpyAsync(out, x->dc.stats, (size_t)n * sizeof(IterStat), cudaMemcpyDeviceToHost, x->copy_stream) != cudaSuccess ||
+        cudaStreamSynchronize(x->copy_stream) != cudaSuccess)
+      return BLINK_ECUDA;
+  }
+  return BLINK_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,526 @@
+// Data-parallel phases of one serving step (every CTA of the grid takes part):
+// embedding + RMSNorm, CUDA-core reference GEMM, RoPE + paged-KV write, paged
+// attention, SwiGLU gate, final norm, sampling.  Each phase is a __device__
+// function that distributes its work over blockIdx.x / gridDim.x, so the same
+// code runs inside the persistent loop (phases separated by grid barriers) and
+// as host-launched kernels (stepped mode).
+//
+// Paper: the model step is the "inference engine" of Section 4.2 (paged KV cache,
+// context attention, fused MLP, sampling captured inside the step); Section 6.1
+// lists the engine features.  The math is the standard pre-norm decoder.
+#pragma once
+#include "dev_ctx.cuh"
+
+namespace blink {
+
+constexpr int FWD_THREADS = 256;
+
+template <typename T> struct OpType;
+template <> struct OpType<float> {
+  static __device__ __forceinline__ float to_f(float v) { return v; }
+  static __device__ __forceinline__ float from_f(float v) { return v; }
+};
+template <> struct OpType<__nv_bfloat16> {
+  static __device__ __forceinline__ float to_f(__nv_bfloat16 v) { return __bfloat162float(v); }
+  static __device__ __forceinline__ __nv_bfloat16 from_f(float v) { return __float2bfloat16_rn(v); }
+};
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ float block_sum(float v, float* s_red /*[8]*/) {
+  v = warp_sum(v);
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) s_red[threadIdx.x >> 5] = v;
+  __syncthreads();
+  float t = 0.f;
+#pragma unroll
+  for (int i = 0; i < FWD_THREADS / 32; ++i) t += s_red[i];
+  return t;
+}
+
+template <typename WT>
+__device__ __forceinline__ const WT* wptr(const DevCtx& c, int id) {
+  return reinterpret_cast<const WT*>(c.w_base + c.w_off[id]);
+}
+__device__ __forceinline__ const float* wptr_f(const DevCtx& c, int id) {
+  return reinterpret_cast<const float*>(c.w_base + c.w_off[id]);
+}
+
+// ---- RMSNorm of the residual rows into the operand buffer; layer 0 gathers the
+// embedding first.  n = x / sqrt(mean(x^2) + eps) * g
+template <typename WT>
+__device__ void phase_norm(const DevCtx& c, int layer, int which /*0: norm1, 1: norm2*/) {
+  __shared__ float s_red[FWD_THREADS / 32];
+  const int T = c.ss->cur_T;
+  const float* g = wptr_f(c, which == 0 ? 6 : 7) + (size_t)layer * c.d;
+  WT* out = reinterpret_cast<WT*>(c.xn);
+  for (int t = blockIdx.x; t < T; t += gridDim.x) {
+    float* hrow = c.h + (size_t)t * c.d;
+    if (which == 0 && layer == 0) {
+      const WT* e = wptr<WT>(c, 0) + (size_t)c.tok_id[t] * c.d;
+      for (int i = threadIdx.x; i < c.d; i += FWD_THREADS) hrow[i] = OpType<WT>::to_f(e[i]);
+      __syncthreads();
+    }
+    float ss = 0.f;
+    for (int i = threadIdx.x; i < c.d; i += FWD_THREADS) { const float v = hrow[i]; ss += v * v; }
+    ss = block_sum(ss, s_red);
+    const float inv = 1.0f / sqrtf(ss / (float)c.d + c.rms_eps);
+    for (int i = threadIdx.x; i < c.d; i += FWD_THREADS)
+      out[(size_t)t * c.d + i] = OpType<WT>::from_f(hrow[i] * inv * g[i]);
+    __syncthreads();
+  }
+}
+
+// Final norm of the sampled rows only (the LM head runs on those rows).
+template <typename WT>
+__device__ void phase_final_norm(const DevCtx& c) {
+  __shared__ float s_red[FWD_THREADS / 32];
+  const int R = c.ss->cur_rows;
+  const float* g = wptr_f(c, 8);
+  WT* out = reinterpret_cast<WT*>(c.xs);
+  for (int r = blockIdx.x; r < R; r += gridDim.x) {
+    const float* hrow = c.h + (size_t)c.row_tok[r] * c.d;
+    float ss = 0.f;
+    for (int i = threadIdx.x; i < c.d; i += FWD_THREADS) { const float v = hrow[i]; ss += v * v; }
+    ss = block_sum(ss, s_red);
+    const float inv = 1.0f / sqrtf(ss / (float)c.d + c.rms_eps);
+    for (int i = threadIdx.x; i < c.d; i += FWD_THREADS)
+      out[(size_t)r * c.d + i] = OpType<WT>::from_f(hrow[i] * inv * g[i]);
+    __syncthreads();
+  }
+}
+
+// ---- CUDA-core reference GEMM: out[t][n] (+)= sum_k x[t][k] * w[n][k], fp32 accumulate.
+// 64x64 output tile, BK = 16, 4x4 outputs per thread.  Deterministic (no split-K).
+struct GemmArgs {
+  const void* x;   // [M][K] operand type
+  const void* w;   // [N][K] operand type
+  float* out;      // [M][ldo]
+  int M, N, K, ldo;
+  int accumulate;  // 1: out += result (residual), 0: out = result
+};
+
+template <typename WT>
+__device__ void phase_gemm_simt(const GemmArgs& a) {
+  constexpr int BM = 64, BN = 64, BK = 16;
+  __shared__ float xs[BK][BM + 4];
+  __shared__ float ws[BK][BN + 4];
+  const WT* X = reinterpret_cast<const WT*>(a.x);
+  const WT* W = reinterpret_cast<const WT*>(a.w);
+  const int tiles_m = (a.M + BM - 1) / BM, tiles_n = (a.N + BN - 1) / BN;
+  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;  // 16 x 16 threads
+  const int lrow = threadIdx.x >> 2, lk = (threadIdx.x & 3) * 4;
+  for (int tile = blockIdx.x; tile < tiles_m * tiles_n; tile += gridDim.x) {
+    const int tm = tile % tiles_m, tn = tile / tiles_m;
+    const int m0 = tm * BM, n0 = tn * BN;
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+    for (int k0 = 0; k0 < a.K; k0 += BK) {
+      {
+        const int m = m0 + lrow, n = n0 + lrow;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int k = k0 + lk + e;
+          xs[lk + e][lrow] = (m < a.M && k < a.K) ? OpType<WT>::to_f(X[(size_t)m * a.K + k]) : 0.f;
+          ws[lk + e][lrow] = (n < a.N && k < a.K) ? OpType<WT>::to_f(W[(size_t)n * a.K + k]) : 0.f;
+        }
+      }
+      __syncthreads();
+#pragma unroll
+      for (int k = 0; k < BK; ++k) {
+        float xv[4], wv[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) xv[i] = xs[k][ty * 4 + i];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) wv[j] = ws[k][tx * 4 + j];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+          for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(xv[i], wv[j], acc[i][j]);
+      }
+      __syncthreads();
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int m = m0 + ty * 4 + i;
+      if (m >= a.M) continue;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int n = n0 + tx * 4 + j;
+        if (n >= a.N) continue;
+        float* o = a.out + (size_t)m * a.ldo + n;
+        *o = a.accumulate ? (*o + acc[i][j]) : acc[i][j];
+      }
+    }
+  }
+}
+
+// ---- RoPE (rotate-half pairing) on q and k, then K/V into the paged pool --------------
+// KV pool layout [L][2][n_blocks][Hkv][bs][hd]: one (block, kv head) tile is contiguous.
+template <typename WT>
+__device__ __forceinline__ WT* kv_tile(const DevCtx& c, int layer, int kv, int block, int head) {
+  const size_t tile = (size_t)c.bs * c.hd;
+  return reinterpret_cast<WT*>(c.kv_base) +
+         ((((size_t)layer * 2 + kv) * c.n_blocks + block) * c.Hkv + head) * tile;
+}
+
+template <typename WT>
+__device__ void phase_rope_kv(const DevCtx& c, int layer) {
+  const int T = c.ss->cur_T;
+  const int half = c.hd / 2;
+  const int heads = c.Hq + 2 * c.Hkv;
+  const long long total = (long long)T * heads * half;
+  for (long long idx = (long long)blockIdx.x * FWD_THREADS + threadIdx.x; idx < total;
+       idx += (long long)gridDim.x * FWD_THREADS) {
+    const int i = (int)(idx % half);
+    const int hh = (int)((idx / half) % heads);
+    const int t = (int)(idx / ((long long)half * heads));
+    float* row = c.qkv + (size_t)t * c.qkv_dim + (size_t)hh * c.hd;
+    const int pos = c.tok_pos[t];
+    const float x1 = row[i], x2 = row[i + half];
+    if (hh < c.Hq + c.Hkv) {
+      const float cs = c.rope_cos[(size_t)pos * half + i], sn = c.rope_sin[(size_t)pos * half + i];
+      const float y1 = x1 * cs - x2 * sn, y2 = x2 * cs + x1 * sn;
+      if (hh < c.Hq) {
+        row[i] = y1;
+        row[i + half] = y2;
+      } else {
+        const int sm = c.tok_slotmap[t];
+        WT* dst = kv_tile<WT>(c, layer, 0, sm / c.bs, hh - c.Hq) + (size_t)(sm % c.bs) * c.hd;
+        dst[i] = OpType<WT>::from_f(y1);
+        dst[i + half] = OpType<WT>::from_f(y2);
+      }
+    } else {
+      const int sm = c.tok_slotmap[t];
+      WT* dst = kv_tile<WT>(c, layer, 1, sm / c.bs, hh - c.Hq - c.Hkv) + (size_t)(sm % c.bs) * c.hd;
+      dst[i] = OpType<WT>::from_f(x1);
+      dst[i + half] = OpType<WT>::from_f(x2);
+    }
+  }
+}
+
+// ---- paged attention ---------------------------------------------------------------------
+// Unit of work: (row t, kv head g): the n_rep query heads of the group share every K/V
+// load.  The 8 warps of the CTA take KV blocks round-robin; within a warp a 16-byte
+// vector load per lane covers whole (block, head) tiles with coalesced 512-byte rows.
+// Online softmax per warp, merged across warps in shared memory at the end.
+template <typename WT, int HD, int NREP>
+__device__ void phase_attention(const DevCtx& c, int layer, float* smem) {
+  constexpr int CE = 16 / (int)sizeof(WT);  // elements per 16-byte chunk
+  constexpr int LPK = HD / CE;              // lanes per key
+  constexpr int KPP = 32 / LPK;             // keys per pass
+  constexpr int MAXR = NREP;                // query heads per kv head
+  constexpr int NW = FWD_THREADS / 32;
+  static_assert(LPK <= 32 && KPP >= 1, "head_dim too large for this mapping");
+  const int T = c.ss->cur_T;
+  constexpr int n_rep = NREP;
+  const int bs = c.bs;
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const int sub = lane / LPK;   // which key of the pass
+  const int ch = lane % LPK;    // which 16-byte chunk of the head vector
+  // shared: q [NREP][HD], per-warp m,l [NW][NREP], acc [NW][NREP][HD]
+  float* s_q = smem;
+  float* s_m = s_q + MAXR * HD;
+  float* s_l = s_m + NW * MAXR;
+  float* s_acc = s_l + NW * MAXR;
+  WT* out = reinterpret_cast<WT*>(c.attn);
+
+  const int units = T * c.Hkv;
+  for (int u = blockIdx.x; u < units; u += gridDim.x) {
+    const int t = u / c.Hkv, g = u % c.Hkv;
+    const int item = c.tok_item[t];
+    const int b = c.it_bslot[item];
+    const int n_ctx = c.tok_pos[t] + 1;
+    const int32_t* table = c.block_table + (size_t)b * c.max_blocks_seq;
+    __syncthreads();
+    for (int i = threadIdx.x; i < n_rep * HD; i += FWD_THREADS)
+      s_q[i] = c.qkv[(size_t)t * c.qkv_dim + (size_t)g * n_rep * HD + i] * c.attn_scale;
+    __syncthreads();
+    float q[MAXR][CE];
+    float acc[MAXR][CE];
+    float m[MAXR], l[MAXR];
+#pragma unroll
+    for (int r = 0; r < MAXR; ++r) {
+      m[r] = -INFINITY;
+      l[r] = 0.f;
+#pragma unroll
+      for (int e = 0; e < CE; ++e) {
+        acc[r][e] = 0.f;
+        q[r][e] = (r < n_rep) ? s_q[r * HD + ch * CE + e] : 0.f;
+      }
+    }
+    const int n_kb = (n_ctx + bs - 1) / bs;
+    for (int kb = w; kb < n_kb; kb += NW) {
+      const int blk = table[kb];
+      const WT* kt = kv_tile<WT>(c, layer, 0, blk, g);
+      const WT* vt = kv_tile<WT>(c, layer, 1, blk, g);
+      for (int k0 = 0; k0 < bs; k0 += KPP) {
+        const int key = k0 + sub;
+        const int kpos = kb * bs + key;
+        const bool valid = key < bs && kpos < n_ctx;
+        float kf[CE], vf[CE];
+        if (valid) {
+          const uint4 kr = *reinterpret_cast<const uint4*>(kt + (size_t)key * HD + ch * CE);
+          const uint4 vr = *reinterpret_cast<const uint4*>(vt + (size_t)key * HD + ch * CE);
+          const WT* kp = reinterpret_cast<const WT*>(&kr);
+          const WT* vp = reinterpret_cast<const WT*>(&vr);
+#pragma unroll
+          for (int e = 0; e < CE; ++e) { kf[e] = OpType<WT>::to_f(kp[e]); vf[e] = OpType<WT>::to_f(vp[e]); }
+        } else {
+#pragma unroll
+          for (int e = 0; e < CE; ++e) { kf[e] = 0.f; vf[e] = 0.f; }
+        }
+#pragma unroll
+        for (int r = 0; r < MAXR; ++r) {
+          if (r >= n_rep) break;
+          float s = 0.f;
+#pragma unroll
+          for (int e = 0; e < CE; ++e) s = fmaf(q[r][e], kf[e], s);
+#pragma unroll
+          for (int o = LPK / 2; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+          if (!valid) s = -INFINITY;
+          // max over the keys of this pass (lanes with different `sub`)
+          float mx = s;
+#pragma unroll
+          for (int o = LPK; o < 32; o <<= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+          const float m_new = fmaxf(m[r], mx);
+          if (m_new == -INFINITY) continue;   // nothing valid yet (uniform across the warp)
+          const float corr = __expf(m[r] - m_new);
+          const float p = valid ? __expf(s - m_new) : 0.f;
+          // l and acc are per-lane partials over this lane's keys; lanes of other `sub`
+          // hold the other keys and are merged at the end
+          l[r] = l[r] * corr + p;
+#pragma unroll
+          for (int e = 0; e < CE; ++e) acc[r][e] = fmaf(p, vf[e], acc[r][e] * corr);
+          m[r] = m_new;
+        }
+      }
+    }
+    // merge lanes that handled different keys (same chunk): sum over `sub`
+#pragma unroll
+    for (int r = 0; r < MAXR; ++r) {
+      if (r >= n_rep) break;
+#pragma unroll
+      for (int o = LPK; o < 32; o <<= 1) {
+        l[r] += __shfl_xor_sync(0xffffffffu, l[r], o);
+#pragma unroll
+        for (int e = 0; e < CE; ++e) acc[r][e] += __shfl_xor_sync(0xffffffffu, acc[r][e], o);
+      }
+      // every lane with the same `ch` now holds the warp's full partial
+      if (sub == 0) {
+#pragma unroll
+        for (int e = 0; e < CE; ++e) s_acc[((size_t)w * MAXR + r) * HD + ch * CE + e] = acc[r][e];
+        if (ch == 0) { s_m[w * MAXR + r] = m[r]; s_l[w * MAXR + r] = l[r]; }
+      }
+    }
+    __syncthreads();
+    // merge the warps: out = sum_w e^(m_w - M) acc_w / sum_w e^(m_w - M) l_w
+    for (int i = threadIdx.x; i < n_rep * HD; i += FWD_THREADS) {
+      const int r = i / HD, dim = i % HD;
+      float M = -INFINITY;
+#pragma unroll
+      for (int ww = 0; ww < NW; ++ww) M = fmaxf(M, s_m[ww * MAXR + r]);
+      float num = 0.f, den = 0.f;
+#pragma unroll
+      for (int ww = 0; ww < NW; ++ww) {
+        const float mw = s_m[ww * MAXR + r];
+        if (mw == -INFINITY) continue;
+        const float f = __expf(mw - M);
+        num += f * s_acc[((size_t)ww * MAXR + r) * HD + dim];
+        den += f * s_l[ww * MAXR + r];
+      }
+      out[(size_t)t * c.q_dim + (size_t)(g * n_rep + r) * HD + dim] = OpType<WT>::from_f(num / den);
+    }
+  }
+}
+constexpr int ATTN_SMEM_FLOATS(int HD, int NREP) { return NREP * HD + 2 * 8 * NREP + 8 * NREP * HD; }
+
+// ---- SwiGLU gate: act = silu(gate) * up ------------------------------------------------
+template <typename WT>
+__device__ void phase_silu_mul(const DevCtx& c) {
+  const int T = c.ss->cur_T;
+  WT* out = reinterpret_cast<WT*>(c.act);
+  const long long total = (long long)T * c.F;
+  for (long long idx = (long long)blockIdx.x * FWD_THREADS + threadIdx.x; idx < total;
+       idx += (long long)gridDim.x * FWD_THREADS) {
+    const int t = (int)(idx / c.F), j = (int)(idx % c.F);
+    const float gte = c.gu[(size_t)t * 2 * c.F + j], up = c.gu[(size_t)t * 2 * c.F + c.F + j];
+    out[idx] = OpType<WT>::from_f(gte / (1.0f + __expf(-gte)) * up);
+  }
+}
+
+// ---- sampling ------------------------------------------------------------------------------
+// Philox4x32-10 (Salmon et al., SC'11): counter-based, so the draw for (ticket, index)
+// does not depend on batch composition.
+__device__ __forceinline__ uint32_t philox4x32_10_word0(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                                        uint32_t k0, uint32_t k1) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+    const uint32_t n0 = hi1 ^ c1 ^ k0, n2 = hi0 ^ c3 ^ k1;
+    c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+    k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+  }
+  return c0;
+}
+
+// order-preserving map float -> uint32 (larger float => larger key)
+__device__ __forceinline__ uint32_t float_key(float f) {
+  const uint32_t u = __float_as_uint(f);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+// One CTA per sampled row.  Greedy: lowest index among the maxima.  Top-k: z = logit / T
+// (IEEE fp32 divide); the k largest by (z desc, index asc) are found with a radix select
+// on the float keys; weights exp(z - z0) and the inverse-CDF walk run in fp64.
+// The result is returned by thread 0 (other threads return -1).
+__device__ int sample_row(const float* lg, int V, int top_k, float temp, unsigned long long ticket, int gen_index,
+                          unsigned long long seed, float* smem) {
+  constexpr int CAND_MAX = 1024;
+  const int tid = threadIdx.x;
+  uint32_t* s_hist = reinterpret_cast<uint32_t*>(smem);             // [256]
+  float* s_cz = smem + 256;                                          // [CAND_MAX]
+  int* s_ci = reinterpret_cast<int*>(smem + 256 + CAND_MAX);         // [CAND_MAX]
+  __shared__ float s_bv[FWD_THREADS / 32];
+  __shared__ int s_bi[FWD_THREADS / 32];
+  __shared__ unsigned long long s_prefix, s_mask;
+  __shared__ int s_remaining, s_ncand;
+  __shared__ float s_tz[MAX_TOPK];
+  __shared__ int s_ti[MAX_TOPK];
+  int result = -1;
+  __syncthreads();
+  if (top_k <= 0) {
+    float bv = -INFINITY;
+    int bi = 0x7fffffff;
+    for (int i = tid; i < V; i += FWD_THREADS) {
+      const float v = lg[i];
+      if (v > bv || (v == bv && i < bi)) { bv = v; bi = i; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+      if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+    }
+    if ((tid & 31) == 0) { s_bv[tid >> 5] = bv; s_bi[tid >> 5] = bi; }
+    __syncthreads();
+    if (tid == 0) {
+      for (int i = 1; i < FWD_THREADS / 32; ++i)
+        if (s_bv[i] > bv || (s_bv[i] == bv && s_bi[i] < bi)) { bv = s_bv[i]; bi = s_bi[i]; }
+      result = bi;
+    }
+    __syncthreads();
+    return result;
+  }
+  const int k = min(top_k, V);
+  // radix select over the composite key (z key, ~index): unique keys, so ties in z
+  // break towards the lower index and the k-th key is exact.  Refine 8 bits at a time
+  // until the set {key >= prefix} (>= k elements by construction) fits the sort buffer.
+  if (tid == 0) { s_prefix = 0; s_mask = 0; s_remaining = k; }
+  __syncthreads();
+  for (int shift = 56; shift >= 0; shift -= 8) {
+    s_hist[tid] = 0;   // FWD_THREADS == 256 bins
+    __syncthreads();
+    const unsigned long long prefix = s_prefix, mask = s_mask;
+    for (int i = tid; i < V; i += FWD_THREADS) {
+      const unsigned long long key =
+          ((unsigned long long)float_key(__fdiv_rn(lg[i], temp)) << 32) | (uint32_t)(~(uint32_t)i);
+      if ((key & mask) == prefix) atomicAdd(&s_hist[(unsigned)(key >> shift) & 255u], 1u);
+    }
+    __syncthreads();
+    if (tid == 0) {
+      const int need = s_remaining;   // how many are still needed from inside the current prefix
+      int bin = 255;
+      uint32_t above = 0;
+      for (; bin > 0; --bin) {
+        if (above + s_hist[bin] >= (uint32_t)need) break;
+        above += s_hist[bin];
+      }
+      s_remaining = need - (int)above;
+      s_prefix = prefix | ((unsigned long long)bin << shift);
+      s_mask = mask | (255ull << shift);
+      // keys >= new prefix: those in strictly higher bins at every level so far, plus this bin
+      s_ncand = (k - s_remaining) + (int)s_hist[bin];
+    }
+    __syncthreads();
+    if (s_ncand <= CAND_MAX) break;
+  }
+  const unsigned long long thr = s_prefix;
+  __syncthreads();
+  if (tid == 0) s_ncand = 0;
+  __syncthreads();
+  for (int i = tid; i < V; i += FWD_THREADS) {
+    const float z = __fdiv_rn(lg[i], temp);
+    const unsigned long long key = ((unsigned long long)float_key(z) << 32) | (uint32_t)(~(uint32_t)i);
+    if (key >= thr) {
+      const int p = atomicAdd(&s_ncand, 1);
+      if (p < CAND_MAX) { s_cz[p] = z; s_ci[p] = i; }
+    }
+  }
+  __syncthreads();
+  const int nc = min(s_ncand, CAND_MAX);
+  // rank every candidate by (z desc, index asc); the k best land at their rank
+  for (int a = tid; a < nc; a += FWD_THREADS) {
+    const float za = s_cz[a];
+    const int ia = s_ci[a];
+    int rank = 0;
+    for (int j = 0; j < nc; ++j) {
+      const float zj = s_cz[j];
+      rank += (zj > za) || (zj == za && s_ci[j] < ia);
+    }
+    if (rank < k) { s_tz[rank] = za; s_ti[rank] = ia; }
+  }
+  __syncthreads();
+  if (tid == 0) {
+    const uint32_t x = philox4x32_10_word0((uint32_t)ticket, (uint32_t)(ticket >> 32), (uint32_t)gen_index, 0u,
+                                           (uint32_t)seed, (uint32_t)(seed >> 32));
+    const double u = (double)(x >> 8) * (1.0 / 16777216.0);
+    const int kk = min(k, nc);
+    double total = 0.0;
+    for (int j = 0; j < kk; ++j) total += exp((double)s_tz[j] - (double)s_tz[0]);
+    const double target = u * total;
+    double accum = 0.0;
+    int pick = s_ti[kk - 1];
+    for (int j = 0; j < kk; ++j) {
+      accum += exp((double)s_tz[j] - (double)s_tz[0]);
+      if (accum > target) { pick = s_ti[j]; break; }
+    }
+    result = pick;
+  }
+  __syncthreads();
+  return result;
+}
+
+__device__ void phase_sample(const DevCtx& c, float* smem) {
+  const int R = c.ss->cur_rows;
+  const int V = c.V;
+  const int tid = threadIdx.x;
+  const unsigned long long rows_before = c.ss->sample_rows_total;
+  for (int r = blockIdx.x; r < R; r += gridDim.x) {
+    const float* lg = c.logits + (size_t)r * V;
+    const int item = c.row_item[r];
+    const int b = c.it_bslot[item];
+    if (c.logits_capture != nullptr && (long long)(rows_before + r) < c.capture_rows) {
+      float* dst = c.logits_capture + (size_t)(rows_before + r) * V;
+      for (int i = tid; i < V; i += FWD_THREADS) dst[i] = lg[i];
+    }
+    const int tok = sample_row(lg, V, min(c.b_topk[b], MAX_TOPK), c.b_temp[b], (unsigned long long)c.b_ticket[b],
+                               c.b_generated[b], c.b_seed[b], smem);
+    if (tid == 0) c.row_sampled[r] = tok;
+  }
+}
+constexpr int SAMPLE_SMEM_FLOATS = 256 + 2 * 1024;
+
+}  // namespace blink

@@ -1,0 +1,127 @@
+"""GPU parity of the control plane (scheduler, allocator, ring protocol): the device
+trace must equal the oracle's, word for word."""
+import numpy as np
+import pytest
+
+from oracle import scheduler as O1
+from paper_2604_07609_b200 import binding as B
+from synth import make_requests, model_cfg, sched_cfg
+from synth.workload import Request
+
+from gpu_util import assert_traces_equal, oracle_control_trace, run_control_only
+
+pytestmark = pytest.mark.gpu
+
+
+def _check(model, sched, reqs, **kw):
+    trace, toks, st, its = run_control_only(model, sched, reqs, **kw)
+    assert st.device_status == 0
+    tr_o, toks_o = oracle_control_trace(sched, reqs, trace, model.vocab)
+    assert_traces_equal(trace, tr_o)
+    assert toks == toks_o
+    assert st.free_blocks == sched.n_blocks and st.reserved_blocks == 0 and st.batch_live == 0
+    return trace, st, its
+
+
+@pytest.mark.parametrize("mode", [B.EXEC_PERSISTENT, B.EXEC_STEPPED], ids=["persistent", "stepped"])
+def test_config1_trace_bit_exact(mode):
+    model, sched = model_cfg(1), sched_cfg(1)
+    trace, st, _ = _check(model, sched, make_requests(1), exec_mode=mode)
+    assert trace[0]["W"] == 7 and len(trace[0]["admitted"]) == 8     # all visible to the first iteration
+
+
+def test_tiny_pool_head_of_line_blocking():
+    model = model_cfg(1)
+    sched = sched_cfg(1, n_blocks=9, max_batch=4, prefill_chunk_tokens=24)
+    rng = np.random.default_rng(11)
+    reqs = [Request(t, 0.0, rng.integers(0, 4096, size=int(p)).astype(np.int32), int(n))
+            for t, (p, n) in enumerate([(40, 8), (64, 32), (5, 2), (33, 17), (64, 1), (1, 1), (17, 30)])]
+    trace, st, _ = _check(model, sched, reqs)
+    assert max(r["reserved"] for r in trace) <= 9
+
+
+def test_relaunch_with_small_iteration_budget_continues_bit_exactly():
+    model, sched = model_cfg(1), sched_cfg(1)
+    reqs = make_requests(1)
+    full, _, st_full, _ = run_control_only(model, sched, reqs)
+    cut, _, st_cut, _ = run_control_only(model, sched, reqs, iteration_budget=7)
+    assert st_cut.launches > st_full.launches and st_cut.launches >= len(full) // 7
+    assert_traces_equal(cut, full)
+
+
+def test_slot_reuse_and_backpressure():
+    model = model_cfg(1)
+    sched = sched_cfg(1, n_slots=4, max_batch=2)
+    rng = np.random.default_rng(5)
+    eng = B.Blink(model, sched, control_only=True, trace_words=1 << 20, idle_exit_us=300_000)
+    try:
+        mk = lambda: rng.integers(0, 4096, size=20).astype(np.int32)
+        for i in range(4):
+            assert eng.blink_submit(mk(), 6) == i
+        assert eng.blink_submit(mk(), 6, raise_on_error=False) == B.BLINK_EAGAIN     # ring full
+        ev = eng.drain(24, timeout_s=30)
+        assert sorted(set(int(t) for t in ev["ticket"])) == [0, 1, 2, 3]
+        for i in range(4, 8):                                                         # slots were recycled
+            assert eng.blink_submit(mk(), 3) == i
+        ev2 = eng.drain(12, timeout_s=30)
+        assert sorted(set(int(t) for t in ev2["ticket"])) == [4, 5, 6, 7]
+        for t in range(4, 8):
+            idx = [int(e["index"]) for e in ev2 if e["ticket"] == t]
+            assert idx == [0, 1, 2]
+        # argument checks
+        assert eng.blink_submit(np.zeros(65, np.int32), 3, raise_on_error=False) == B.BLINK_EINVAL
+        assert eng.blink_submit(np.array([4096], np.int32), 3, raise_on_error=False) == B.BLINK_EINVAL
+        assert eng.blink_submit(mk(), 0, raise_on_error=False) == B.BLINK_EINVAL
+        assert eng.blink_submit(mk(), 3, top_k=65, raise_on_error=False) == B.BLINK_EINVAL
+    finally:
+        assert eng.blink_destroy() == B.BLINK_OK
+
+
+def test_idle_exit_and_relaunch_on_submit():
+    import time
+    model, sched = model_cfg(1), sched_cfg(1)
+    eng = B.Blink(model, sched, control_only=True, idle_exit_us=50_000)
+    try:
+        time.sleep(0.5)
+        assert eng.blink_get_stats().loop_state == B.LOOP_EXIT_IDLE       # left the GPU on its own
+        eng.blink_submit(np.arange(10, dtype=np.int32), 4)
+        ev = eng.drain(4, timeout_s=30)
+        assert len(ev) == 4 and eng.blink_get_stats().launches == 2
+        assert eng.blink_stop(final=True) == B.BLINK_OK
+        assert eng.blink_submit(np.arange(10, dtype=np.int32), 4, raise_on_error=False) == B.BLINK_ESTOPPED
+    finally:
+        assert eng.blink_destroy() == B.BLINK_OK
+
+
+def test_config3_and_config5_streams_trace_at_full_scale():
+    """Traces do not depend on the model math (fixed output lengths), so the full request
+    streams of the 8B and MoE configurations are checked in control-only mode."""
+    for cfg_i, n_blocks in ((3, 60000), (5, 60000)):
+        model = model_cfg(cfg_i)
+        sched = sched_cfg(cfg_i, n_blocks=n_blocks)
+        reqs = make_requests(cfg_i)
+        trace, st, its = _check(model, sched, reqs, trace_words=1 << 27)
+        assert sum(len(r["sampled"]) for r in trace) == sum(r.max_new for r in reqs)
+        assert max(len(r["scheduled"]) for r in trace) <= 256
+        dt = (its["t_end_ns"] - its["t_begin_ns"]).astype(np.float64)
+        print(f"config {cfg_i}: {len(trace)} iterations, control plane median {np.median(dt) / 1e3:.1f} us/iter")
+
+
+def test_timestamps_and_event_order():
+    model, sched = model_cfg(1), sched_cfg(1)
+    reqs = make_requests(1)
+    eng = B.Blink(model, sched, control_only=True, idle_exit_us=300_000)
+    try:
+        for r in reqs:
+            eng.submit_request(r)
+        ev = eng.drain(8 * 32, timeout_s=30)
+        off = eng.blink_get_stats().device_clock_offset_ns
+        for t in range(8):
+            e = np.sort(ev[ev["ticket"] == t], order="index")
+            assert list(e["index"]) == list(range(32))
+            assert e["is_first"][0] == 1 and e["is_last"][-1] == 1 and e["is_last"][:-1].sum() == 0
+            assert np.all(np.diff(e["t_device_ns"].astype(np.int64)) > 0)
+            ttft_ns = int(e["t_device_ns"][0]) + off - int(e["t_submit_ns"][0])
+            assert -1_000_000 < ttft_ns < 2_000_000_000
+    finally:
+        assert eng.blink_destroy() == B.BLINK_OK

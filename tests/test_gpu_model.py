@@ -1,0 +1,128 @@
+"""GPU parity of the whole step (forward + sampling) against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import sampler as S
+from oracle import transformer as O2
+from paper_2604_07609_b200 import binding as B
+from synth import make_requests, make_weights, model_cfg, sched_cfg
+
+from gpu_util import assert_traces_equal, gpu_run_forced, oracle_run
+
+pytestmark = pytest.mark.gpu
+
+TOL_FP32 = 1e-4     # max-abs logit error, fp32 reference mode
+TOL_BF16 = 2e-2     # max-abs logit error, bf16 mode
+
+
+def _compare(model, sched, reqs, weights, act_round, tol, **kw):
+    ora = oracle_run(model, sched, reqs, weights, act_round)
+    trace, toks, logits, _ = gpu_run_forced(model, sched, reqs, weights, ora["tokens"], **kw)
+    assert_traces_equal([{**r, "sampled": []} for r in trace], [{**r, "sampled": []} for r in ora["trace"]])
+    lo = np.stack([row for (_, _, _, _, row) in ora["logits"]])
+    assert logits.shape == lo.shape
+    err = np.abs(logits.astype(np.float64) - lo).max()
+    # tokens: identical wherever the oracle's decision margin exceeds twice the tolerance
+    n_in_margin = 0
+    k = 0
+    for (it, bslot, ticket, gi, row) in ora["logits"]:
+        r = reqs[ticket]
+        if r.top_k == 0:
+            srt = np.sort(row)
+            margin = srt[-1] - srt[-2]
+            if margin > 2 * tol:
+                assert toks[ticket][gi] == ora["tokens"][ticket][gi], (ticket, gi, margin)
+            else:
+                n_in_margin += 1
+                assert row[toks[ticket][gi]] >= srt[-1] - 2 * tol
+        k += 1
+    return err, n_in_margin, trace, toks, ora
+
+
+def test_config1_fp32_reference_mode_logits_tokens_trace():
+    model, sched = model_cfg(1, dtype="fp32"), sched_cfg(1)
+    reqs = make_requests(1)
+    w = make_weights(model, 1234, "cpu")
+    err, n_margin, trace, toks, ora = _compare(model, sched, reqs, w, None, TOL_FP32)
+    print(f"C1 fp32: max-abs logit error {err:.3e}, {n_margin} in-margin decisions")
+    assert err <= TOL_FP32
+    assert toks == ora["tokens"]           # unconditional bit-exact token gate of the small configuration
+    assert_traces_equal(trace, ora["trace"])
+
+
+def test_config1_bf16_logits_within_tolerance():
+    model, sched = model_cfg(1, dtype="bf16"), sched_cfg(1)
+    reqs = make_requests(1)
+    w = make_weights(model, 1234, "cpu")
+    err, n_margin, trace, toks, ora = _compare(model, sched, reqs, w, O2.round_bf16, TOL_BF16)
+    print(f"C1 bf16: max-abs logit error {err:.3e}, {n_margin} in-margin decisions")
+    assert err <= TOL_BF16
+
+
+def test_stepped_mode_matches_persistent_mode_bitwise():
+    model, sched = model_cfg(1, dtype="fp32"), sched_cfg(1)
+    reqs = make_requests(1, n_requests=4)
+    w = make_weights(model, 99, "cpu", random_gains=True)
+    a = gpu_run_forced(model, sched, reqs, w, None, exec_mode=B.EXEC_PERSISTENT)
+    b = gpu_run_forced(model, sched, reqs, w, None, exec_mode=B.EXEC_STEPPED)
+    assert a[1] == b[1]
+    assert np.array_equal(a[2], b[2])
+    assert_traces_equal(a[0], b[0])
+
+
+def test_gqa_random_gains_chunked_prefill_small_chunk():
+    """Grouped-query heads (4 q per kv head), head_dim 128, non-unit norm gains, and a chunk
+    budget smaller than the prompts so prefill spans several iterations and mixes with decode."""
+    model = model_cfg(1, n_q_heads=4, n_kv_heads=1, head_dim=128, d_model=256, dtype="fp32")
+    sched = sched_cfg(1, prefill_chunk_tokens=24, max_batch=4, n_blocks=64)
+    reqs = make_requests(1, n_requests=6)
+    w = make_weights(model, 7, "cpu", random_gains=True)
+    err, n_margin, trace, toks, ora = _compare(model, sched, reqs, w, None, TOL_FP32)
+    print(f"GQA fp32: max-abs logit error {err:.3e}")
+    assert err <= TOL_FP32
+    assert any(s[2] == 1 for r in trace for s in r["scheduled"]) and any(
+        {1, 2} <= {s[2] for s in r["scheduled"]} for r in trace)
+
+
+def test_topk_sampling_end_to_end_fp32():
+    model, sched = model_cfg(1, dtype="fp32"), sched_cfg(1)
+    reqs = make_requests(1, n_requests=4)
+    for r in reqs:
+        r.top_k, r.temperature = 50, 0.8
+    w = make_weights(model, 5, "cpu")
+    ora = oracle_run(model, sched, reqs, w, None)
+    trace, toks, logits, _ = gpu_run_forced(model, sched, reqs, w, ora["tokens"])
+    lo = np.stack([row for (_, _, _, _, row) in ora["logits"]])
+    assert np.abs(logits - lo).max() <= TOL_FP32
+    # the draw is identical on both sides; tokens agree unless a candidate boundary sits inside the tolerance
+    agree = sum(toks[t][i] == ora["tokens"][t][i] for t in toks for i in range(len(toks[t])))
+    total = sum(len(v) for v in toks.values())
+    print(f"top-k end to end: {agree}/{total} tokens identical")
+    assert agree >= total - 2
+
+
+def test_sampler_alone_bit_exact_on_oracle_logits():
+    rng = np.random.default_rng(3)
+    V, rows = 128256, 48
+    logits = (rng.normal(size=(rows, V)) * 1.3).astype(np.float32)
+    logits[0, :] = 0.0                              # all equal: ties must break to the lowest indices
+    logits[1, 1000:1200] = logits[1].max() + 1.0    # a plateau larger than k
+    logits[2] = np.round(logits[2] * 2) / 2         # heavy quantisation: many exact ties
+    top_k = np.array([0 if i % 3 == 0 else (50 if i % 3 == 1 else 7) for i in range(rows)], dtype=np.int32)
+    top_k[:3] = [50, 50, 64]
+    temp = np.where(np.arange(rows) % 2 == 0, 0.8, 1.3).astype(np.float32)
+    ticket = np.arange(rows, dtype=np.uint64) * 977 + (1 << 33)
+    gen = (np.arange(rows) * 5 % 97).astype(np.int32)
+    seed = (np.arange(rows, dtype=np.uint64) * 0x9E3779B97F4A7C15) ^ np.uint64(0xB11C0003)
+    got = B.blink_sample(torch.from_numpy(logits).cuda(), top_k, temp, ticket, gen, seed)
+    for r in range(rows):
+        want = S.sample(logits[r], int(top_k[r]), float(temp[r]), int(ticket[r]), int(gen[r]), int(seed[r]))
+        assert int(got[r]) == want, (r, int(got[r]), want)
+    # many draws on one row: the empirical distribution is the oracle's
+    row = logits[5:6].repeat(400, axis=0)
+    n = 400
+    g2 = B.blink_sample(torch.from_numpy(row).cuda(), np.full(n, 50, np.int32), np.full(n, 0.8, np.float32),
+                        np.full(n, 7, np.uint64), np.arange(n, dtype=np.int32), np.full(n, 42, np.uint64))
+    w2 = [S.sample(logits[5], 50, 0.8, 7, i, 42) for i in range(n)]
+    assert list(g2) == w2
