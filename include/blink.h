@@ -54,7 +54,8 @@ enum { BLINK_DTYPE_BF16 = 0, BLINK_DTYPE_FP32 = 1 };
 /* how the iteration is executed */
 enum {
   BLINK_EXEC_PERSISTENT = 0, /* one cooperative kernel loops on the device (product mode)           */
-  BLINK_EXEC_STEPPED = 1     /* same device code, one host launch per phase (profiling, debugging)  */
+  BLINK_EXEC_STEPPED = 1,    /* same device code, one host launch per phase (profiling, debugging)  */
+  BLINK_EXEC_MANUAL = 2      /* the cooperative loop kernel, launched only by blink_run (measurement) */
 };
 
 /* which kernels run the dense contractions */
@@ -169,7 +170,9 @@ typedef struct blink_iter_stat {
   int32_t n_decode;       /* decode rows                                       */
   int32_t n_sample_rows;  /* rows that went through LM head + sampler          */
   int32_t n_items;        /* requests in the step                              */
-  int64_t ctx_tokens;     /* sum over rows of keys attended (KV tokens read)   */
+  int64_t ctx_tokens;     /* sum over rows of keys attended (attention flops)  */
+  int64_t kv_tokens;      /* sum over requests in the step of their context length after the
+                             step: KV tokens an ideal kernel reads once per step              */
 } blink_iter_stat;
 
 /* Bytes of the flat weight buffer for a model shape (dtype taken from cfg). */
@@ -210,6 +213,12 @@ int blink_poll(blink_ctx* ctx, blink_token_event* out, int max_events, int timeo
 /* Stepped mode only: run `n_iterations` iterations, one host launch per phase,
  * and wait for them. */
 int blink_step(blink_ctx* ctx, int n_iterations);
+
+/* Manual mode only: launch the loop kernel once with an iteration budget of
+ * `n_iterations`, wait until it has left the GPU (budget used up, or nothing left to do
+ * for idle_exit_us) and report the launch's duration measured with CUDA events on the
+ * library's stream.  One launch = up to n_iterations whole steps of the hot path. */
+int blink_run(blink_ctx* ctx, int64_t n_iterations, float* elapsed_ms);
 
 /* Ask the loop to leave the GPU and wait (bounded) until it has. State stays
  * intact; blink_poll / blink_submit / blink_start re-launch it when needed

@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libblink.so")
 BLINK_OK, BLINK_EAGAIN, BLINK_EINVAL, BLINK_ESTOPPED, BLINK_EDEVICE = 0, -1, -2, -3, -4
 BLINK_ETIMEDOUT, BLINK_ENOMEM, BLINK_ECUDA = -5, -6, -7
 DTYPE_BF16, DTYPE_FP32 = 0, 1
-EXEC_PERSISTENT, EXEC_STEPPED = 0, 1
+EXEC_PERSISTENT, EXEC_STEPPED, EXEC_MANUAL = 0, 1, 2
 GEMM_AUTO, GEMM_SIMT, GEMM_TC = 0, 1, 2
 LOOP_NOT_STARTED, LOOP_RUNNING, LOOP_EXIT_STOP, LOOP_EXIT_BUDGET, LOOP_EXIT_IDLE, LOOP_EXIT_ERROR = range(6)
 TRACE_MAGIC = 0x424C4B31
@@ -69,18 +69,18 @@ class blink_stats(C.Structure):
 class blink_iter_stat(C.Structure):
     _fields_ = [("t_begin_ns", C.c_uint64), ("t_forward_ns", C.c_uint64), ("t_end_ns", C.c_uint64),
                 ("n_tokens", C.c_int32), ("n_decode", C.c_int32), ("n_sample_rows", C.c_int32),
-                ("n_items", C.c_int32), ("ctx_tokens", C.c_int64)]
+                ("n_items", C.c_int32), ("ctx_tokens", C.c_int64), ("kv_tokens", C.c_int64)]
 
 
 ITER_STAT_DTYPE = np.dtype([("t_begin_ns", "<u8"), ("t_forward_ns", "<u8"), ("t_end_ns", "<u8"),
                             ("n_tokens", "<i4"), ("n_decode", "<i4"), ("n_sample_rows", "<i4"),
-                            ("n_items", "<i4"), ("ctx_tokens", "<i8")])
+                            ("n_items", "<i4"), ("ctx_tokens", "<i8"), ("kv_tokens", "<i8")])
 EVENT_DTYPE = np.dtype([("ticket", "<u8"), ("user_tag", "<u8"), ("index", "<i4"), ("token", "<i4"),
                         ("is_first", "<i4"), ("is_last", "<i4"), ("t_device_ns", "<u8"), ("t_host_ns", "<u8"),
                         ("t_submit_ns", "<u8")])
 
 EXPORTS = ["blink_weights_bytes", "blink_weight_offset", "blink_kv_blocks_for_bytes", "blink_create",
-           "blink_start", "blink_submit", "blink_poll", "blink_step", "blink_stop", "blink_destroy",
+           "blink_start", "blink_submit", "blink_poll", "blink_step", "blink_run", "blink_stop", "blink_destroy",
            "blink_get_stats", "blink_get_trace", "blink_get_iter_stats", "blink_sample", "blink_strerror"]
 
 _lib = None
@@ -112,6 +112,8 @@ def lib():
     L.blink_poll.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int]
     L.blink_step.restype = C.c_int
     L.blink_step.argtypes = [C.c_void_p, C.c_int]
+    L.blink_run.restype = C.c_int
+    L.blink_run.argtypes = [C.c_void_p, C.c_int64, P(C.c_float)]
     L.blink_stop.restype = C.c_int
     L.blink_stop.argtypes = [C.c_void_p, C.c_int, C.c_int]
     L.blink_destroy.restype = C.c_int
@@ -288,6 +290,15 @@ class Blink:
         rc = lib().blink_step(self._h, n)
         if rc != BLINK_OK:
             raise BlinkError(rc, "blink_step")
+
+    def blink_run(self, n_iterations: int) -> float:
+        """Manual mode: one launch of the loop kernel for up to n_iterations steps; returns its
+        duration in ms (CUDA events on the library's stream)."""
+        ms = C.c_float()
+        rc = lib().blink_run(self._h, n_iterations, C.byref(ms))
+        if rc != BLINK_OK:
+            raise BlinkError(rc, "blink_run")
+        return float(ms.value)
 
     def blink_stop(self, final=False, timeout_ms=10000):
         return lib().blink_stop(self._h, int(final), timeout_ms)

@@ -249,6 +249,8 @@ struct blink_ctx {
   size_t smem_bytes = 0;
   int grid = 1;
   TcHost tc_host;
+  bool manual = false;
+  cudaEvent_t ev0 = nullptr, ev1 = nullptr;
 };
 
 namespace {
@@ -283,6 +285,9 @@ void free_all(blink_ctx* x) {
   x->dev_allocs.clear();
   x->host_allocs.clear();
   tc_host_free(x->tc_host);
+  if (x->ev0) cudaEventDestroy(x->ev0);
+  if (x->ev1) cudaEventDestroy(x->ev1);
+  x->ev0 = x->ev1 = nullptr;
   if (x->stream) cudaStreamDestroy(x->stream);
   if (x->copy_stream) cudaStreamDestroy(x->copy_stream);
   x->stream = x->copy_stream = nullptr;
@@ -315,7 +320,7 @@ int launch_loop(blink_ctx* x) {
 
 // Re-instantiate a loop that left the GPU while work is outstanding (caller holds mu).
 int pump(blink_ctx* x) {
-  if (x->dc.stepped) return BLINK_OK;
+  if (x->dc.stepped || x->manual) return BLINK_OK;
   const uint32_t st = x->mbox->loop_state;
   if (st == BLINK_LOOP_RUNNING) return BLINK_OK;
   if (st == BLINK_LOOP_EXIT_ERROR) return BLINK_EDEVICE;
@@ -462,6 +467,7 @@ int blink_create(const blink_model_cfg* model, const blink_sched_cfg* sched, con
   c.max_blocks_seq = (c.max_pos + c.bs - 1) / c.bs;
   c.control_only = sched->control_only; c.start_paused = sched->start_paused;
   c.stepped = sched->exec_mode == BLINK_EXEC_STEPPED;
+  x->manual = sched->exec_mode == BLINK_EXEC_MANUAL;
   c.gemm_tc = 0;
   if (!c.control_only && model->dtype == BLINK_DTYPE_BF16 && sched->gemm_impl != BLINK_GEMM_SIMT) c.gemm_tc = tc_available();
   if (sched->gemm_impl == BLINK_GEMM_TC && !c.gemm_tc) { delete x; return BLINK_EINVAL; }
@@ -576,7 +582,7 @@ int blink_create(const blink_model_cfg* model, const blink_sched_cfg* sched, con
   if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, loop_fn, FWD_THREADS, x->smem_bytes) != cudaSuccess || occ < 1)
     return fail(BLINK_ECUDA);
   if (cudaDeviceSynchronize() != cudaSuccess) return fail(BLINK_ECUDA);
-  if (!c.stepped) {
+  if (!c.stepped && !x->manual) {
     rc = launch_loop(x);
     if (rc != BLINK_OK) return fail(rc);
   } else {
@@ -696,6 +702,25 @@ int blink_step(blink_ctx* x, int n_iterations) {
   x->launches += 1;
   if (cudaStreamSynchronize(x->stream) != cudaSuccess) return BLINK_ECUDA;
   return x->mbox->device_status > 0 && x->mbox->device_status != DEV_ERR_TRACE_OVERFLOW ? BLINK_EDEVICE : BLINK_OK;
+}
+
+int blink_run(blink_ctx* x, int64_t n_iterations, float* elapsed_ms) {
+  if (!x || n_iterations < 1) return BLINK_EINVAL;
+  if (!x->manual) return BLINK_EINVAL;
+  std::lock_guard<std::mutex> g(x->mu);
+  if (x->final_stop) return BLINK_ESTOPPED;
+  if (x->mbox->device_status > 0 && x->mbox->device_status != DEV_ERR_TRACE_OVERFLOW) return BLINK_EDEVICE;
+  if (!x->ev0 && (cudaEventCreate(&x->ev0) != cudaSuccess || cudaEventCreate(&x->ev1) != cudaSuccess)) return BLINK_ECUDA;
+  x->dc.iteration_budget = n_iterations;
+  if (cudaEventRecord(x->ev0, x->stream) != cudaSuccess) return BLINK_ECUDA;
+  const int rc = launch_loop(x);
+  if (rc != BLINK_OK) return rc;
+  if (cudaEventRecord(x->ev1, x->stream) != cudaSuccess) return BLINK_ECUDA;
+  if (cudaEventSynchronize(x->ev1) != cudaSuccess) return BLINK_ECUDA;
+  float ms = 0.f;
+  if (cudaEventElapsedTime(&ms, x->ev0, x->ev1) != cudaSuccess) return BLINK_ECUDA;
+  if (elapsed_ms) *elapsed_ms = ms;
+  return x->mbox->loop_state == BLINK_LOOP_EXIT_ERROR ? BLINK_EDEVICE : BLINK_OK;
 }
 
 int blink_stop(blink_ctx* x, int final, int timeout_ms) {

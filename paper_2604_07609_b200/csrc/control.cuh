@@ -213,6 +213,7 @@ __device__ void post_step(const DevCtx& c) {
       st.n_sample_rows = n_rows;
       st.n_items = n_items;
       st.ctx_tokens = ss->cur_ctx;
+      st.kv_tokens = ss->cur_kv;
     }
     ss->iter += 1;
     ss->cur_hdr = -1;
@@ -299,12 +300,12 @@ __device__ int schedule_step(const DevCtx& c, unsigned long long visible) {
   __shared__ int s_item_b[MAX_BATCH];
   __shared__ int s_n_admit;
   __shared__ int s_trace_ok;
-  __shared__ unsigned long long s_ctx;
+  __shared__ unsigned long long s_ctx, s_kv;
   __shared__ int s_ndec;
 
   const uint64_t t_begin = global_timer_ns();
   s_phase[tid] = tid < MB ? c.b_phase[tid] : -1;
-  if (tid == 0) { s_n_admit = 0; s_ctx = 0; s_ndec = 0; }
+  if (tid == 0) { s_n_admit = 0; s_ctx = 0; s_kv = 0; s_ndec = 0; }
   __syncthreads();
 
   // open a trace record (header is completed later)
@@ -465,6 +466,7 @@ __device__ int schedule_step(const DevCtx& c, unsigned long long visible) {
                                                      : (unsigned long long)take * start +
                                                            (unsigned long long)take * (take + 1) / 2;
     atomicAdd(&s_ctx, ctx);
+    atomicAdd(&s_kv, (unsigned long long)new_len);
     if (phase == PHASE_DECODE) atomicAdd(&s_ndec, 1);
   }
   if (tid == 0) s_qstart[n_items] = T;
@@ -497,6 +499,7 @@ __device__ int schedule_step(const DevCtx& c, unsigned long long visible) {
     ss->cur_rows = n_rows;
     ss->cur_decode = s_ndec;
     ss->cur_ctx = (long long)s_ctx;
+    ss->cur_kv = (long long)s_kv;
     ss->cur_t_begin = t_begin;
     ss->pending_post = 1;
     if (tr) {

@@ -92,6 +92,7 @@ struct SchedState {
   int reserved;                     // blocks promised to admitted requests
   int cur_T, cur_items, cur_rows, cur_decode;
   long long cur_ctx;
+  long long cur_kv;
   int cmd;
   int pending_post;                 // a forward ran and its post step is outstanding
   int trace_off;                    // tracing stopped (overflow)
@@ -107,6 +108,7 @@ struct IterStat {
   uint64_t t_begin_ns, t_forward_ns, t_end_ns;
   int32_t n_tokens, n_decode, n_sample_rows, n_items;
   int64_t ctx_tokens;
+  int64_t kv_tokens;
 };
 
 constexpr int TRACE_HDR_WORDS = 12;
