@@ -469,7 +469,8 @@ int blink_create(const blink_model_cfg* model, const blink_sched_cfg* sched, con
   c.stepped = sched->exec_mode == BLINK_EXEC_STEPPED;
   x->manual = sched->exec_mode == BLINK_EXEC_MANUAL;
   c.gemm_tc = 0;
-  if (!c.control_only && model->dtype == BLINK_DTYPE_BF16 && sched->gemm_impl != BLINK_GEMM_SIMT) c.gemm_tc = tc_available();
+  if (!c.control_only && model->dtype == BLINK_DTYPE_BF16 && sched->gemm_impl != BLINK_GEMM_SIMT)
+    c.gemm_tc = tc_available() && tc_shape_ok(c);
   if (sched->gemm_impl == BLINK_GEMM_TC && !c.gemm_tc) { delete x; return BLINK_EINVAL; }
   c.iteration_budget = c.stepped ? 0 : sched->iteration_budget;
   const double cyc_per_us = 2000.0;  // upper bound on the SM clock: time-outs only get longer at lower clocks

@@ -169,6 +169,7 @@ struct DevCtx {
   float* logits;  // [MB][V]
   float *rope_cos, *rope_sin;  // [max_pos][hd/2]
   void* kv_base;               // [L][2][n_blocks][Hkv][bs][hd] operand type
+  const void* tc_maps;         // TMA descriptors of the tensor-core path (device memory)
   // diagnostics
   int32_t* trace;
   long long trace_cap;

@@ -54,6 +54,14 @@ __device__ __forceinline__ const float* wptr_f(const DevCtx& c, int id) {
   return reinterpret_cast<const float*>(c.w_base + c.w_off[id]);
 }
 
+// zero n_floats (a multiple of 4) floats starting at p, grid-strided
+__device__ __forceinline__ void zero_floats(float* p, long long n_floats) {
+  float4* q = reinterpret_cast<float4*>(p);
+  const long long n4 = n_floats >> 2;
+  for (long long i = (long long)blockIdx.x * FWD_THREADS + threadIdx.x; i < n4; i += (long long)gridDim.x * FWD_THREADS)
+    q[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+}
+
 // ---- RMSNorm of the residual rows into the operand buffer; layer 0 gathers the
 // embedding first.  n = x / sqrt(mean(x^2) + eps) * g
 template <typename WT>
@@ -62,6 +70,8 @@ __device__ void phase_norm(const DevCtx& c, int layer, int which /*0: norm1, 1: 
   const int T = c.ss->cur_T;
   const float* g = wptr_f(c, which == 0 ? 6 : 7) + (size_t)layer * c.d;
   WT* out = reinterpret_cast<WT*>(c.xn);
+  // the split-K tensor-core GEMM that follows adds partial sums into its output
+  if (c.gemm_tc) zero_floats(which == 0 ? c.qkv : c.gu, (long long)T * (which == 0 ? c.qkv_dim : 2 * c.F));
   for (int t = blockIdx.x; t < T; t += gridDim.x) {
     float* hrow = c.h + (size_t)t * c.d;
     if (which == 0 && layer == 0) {
@@ -86,6 +96,7 @@ __device__ void phase_final_norm(const DevCtx& c) {
   const int R = c.ss->cur_rows;
   const float* g = wptr_f(c, 8);
   WT* out = reinterpret_cast<WT*>(c.xs);
+  if (c.gemm_tc) zero_floats(c.logits, (long long)R * c.V);
   for (int r = blockIdx.x; r < R; r += gridDim.x) {
     const float* hrow = c.h + (size_t)c.row_tok[r] * c.d;
     float ss = 0.f;

@@ -1,27 +1,388 @@
-// Tensor-core path of the dense contractions (tcgen05 + TMEM accumulators fed by
-// TMA), bf16 operands, fp32 accumulate.
+// Tensor-core path of the dense contractions: tcgen05.mma with TMEM accumulators, operands
+// staged in shared memory by TMA (128-byte swizzle), bf16 x bf16 -> fp32.
+//
+//   out[t][n] (+)= sum_k x[t][k] * w[n][k]
+//
+// Operand roles are swapped relative to the usual GEMM: the 128 rows of an MMA tile are
+// rows of W (output features), the MMA's N is the token tile (16..256 rows of x).  Decode
+// steps have few tokens and stream every weight once, so the weight tile fills the fixed
+// 128-row dimension and the token count only sets the cheap N.
+//
+// Work split ("stream-K"): the (pass, n-tile, k-block) units of one GEMM are flattened and
+// cut into gridDim.x equal contiguous ranges, so every SM streams the same number of weight
+// bytes whatever the shape.  A CTA's range is a handful of segments (one n-tile each); a
+// segment that covers the whole K of its tile stores its result, a partial one adds it
+// with red.global.add.f32 (the output is zeroed or already holds the residual).
+//
+// Warp roles in the 256-thread CTA: warp 0 = TMA producer (one lane), warp 1 = MMA issuer
+// (one lane), warps 4..7 = epilogue (TMEM -> registers -> global), two accumulator buffers
+// of 256 TMEM columns so the epilogue of one segment overlaps the MMAs of the next.
+// Every wait is bounded: on a time-out the CTA records DEV_ERR_PIPE_TIMEOUT, raises the
+// loop's abort flag and skips all further waits.
 #pragma once
+#include <cuda.h>
+
+#include "control.cuh"
 #include "dev_ctx.cuh"
 #include "forward.cuh"
 
 namespace blink {
 
-enum GemmWhich : int { GEMM_QKV = 0, GEMM_O, GEMM_GU, GEMM_DOWN, GEMM_LMHEAD };
+enum GemmWhich : int { GEMM_QKV = 0, GEMM_O, GEMM_GU, GEMM_DOWN, GEMM_LMHEAD, GEMM_KINDS };
+enum ActBuf : int { ACT_XN = 0, ACT_ATTN, ACT_ACT, ACT_XS, ACT_BUFS };
+constexpr int TC_BOXES = 5;  // token-tile boxes of 16, 32, 64, 128, 256 rows
+constexpr int TC_MAX_STAGES = 8;
+constexpr int TC_A_BYTES = 128 * 128;  // 128 weight rows x 64 bf16
+constexpr int TC_TILE_BUDGET = 196608;
 
+// Per-thread pipeline bookkeeping that survives from one GEMM phase to the next (the
+// mbarriers are initialised once per kernel).  Bit s of a mask is the parity of the next
+// phase to wait for on barrier s; only the thread that owns a role uses its masks.
 struct TcState {
   uint32_t tmem_base;
+  uint32_t fill_bits;   // producer: stages filled so far, parity per stage
+  uint32_t use_bits;    // MMA issuer: stages consumed so far, parity per stage
+  uint32_t acc_mma;     // MMA issuer: accumulator buffers claimed, parity per buffer
+  uint32_t acc_epi;     // epilogue: accumulator buffers drained, parity per buffer
 };
+
+struct TcShared {
+  uint64_t full[TC_MAX_STAGES], empty[TC_MAX_STAGES], acc_full[2], acc_empty[2];
+  uint32_t tmem;
+  int dead;
+};
+__shared__ __align__(8) TcShared g_tc;
+
 struct TcHost {
-  int unused;
+  void* d_maps = nullptr;
 };
 
-inline int tc_available() { return 0; }
-inline size_t tc_smem_bytes() { return 0; }
-inline int tc_host_setup(TcHost&, DevCtx&) { return 0; }
-inline void tc_host_free(TcHost&) {}
+// ---- PTX wrappers -------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
-__device__ __forceinline__ void tc_init(const DevCtx&, float*, TcState& s) { s.tmem_base = 0; }
-__device__ __forceinline__ void tc_fini(const DevCtx&, TcState&) {}
-__device__ __forceinline__ void phase_gemm_tc(const DevCtx&, const GemmArgs&, int, int, float*, TcState&) {}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  `dead` (shared) is set by whoever times out first; once set every wait returns at once.
+__device__ __forceinline__ bool mbar_wait(const DevCtx& c, uint64_t* bar, uint32_t parity, volatile int* dead) {
+  if (*dead) return false;
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  unsigned int spins = 0;
+  while (!mbar_try_wait(bar, parity)) {
+    if ((++spins & 255u) == 0) {
+      if (*dead) return false;
+      if ((unsigned long long)(clock64() - t0) > c.barrier_timeout_cycles) {
+        *dead = 1;
+        dev_fail(c, DEV_ERR_PIPE_TIMEOUT);
+        return false;
+      }
+    }
+  }
+  return true;
+}
+
+__device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
+          smem_u32(smem_dst)),
+      "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar))
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// D[tmem] (+)= A[smem] * B[smem]^T, M = 128, K = 16 per instruction
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
+      "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// arrive on `bar` once all MMAs issued so far by this thread have completed
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+// 32 lanes x 16 consecutive 32-bit columns -> 16 registers per thread
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, "
+      "[%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Shared-memory matrix descriptor: K-major tile of rows x 64 bf16 (128-byte rows), 128-byte
+// swizzle, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);  // start address, 16-byte units
+  d |= (uint64_t)1 << 16;                    // leading byte offset (unused for swizzled K-major)
+  d |= (uint64_t)(1024 >> 4) << 32;          // stride byte offset between 8-row groups
+  d |= (uint64_t)1 << 46;                    // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;                    // 128-byte swizzle
+  return d;
+}
+// Instruction descriptor: bf16 A and B (both K-major), fp32 accumulator, M = 128, N = n.
+__device__ __forceinline__ uint32_t idesc_bf16(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+}
+
+// ---- TMEM allocation for the life of the kernel ---------------------------------------------
+__device__ __forceinline__ void tc_init(const DevCtx& c, float*, TcState& s) {
+  s.tmem_base = 0;
+  s.fill_bits = s.use_bits = s.acc_mma = s.acc_epi = 0;
+  if (!c.gemm_tc) return;
+  if (threadIdx.x == 32) {
+    for (int i = 0; i < TC_MAX_STAGES; ++i) { mbar_init(&g_tc.full[i], 1); mbar_init(&g_tc.empty[i], 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&g_tc.acc_full[b], 1); mbar_init(&g_tc.acc_empty[b], 4); }
+    g_tc.dead = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (threadIdx.x < 32) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&g_tc.tmem))
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  s.tmem_base = *(volatile uint32_t*)&g_tc.tmem;
+}
+__device__ __forceinline__ void tc_fini(const DevCtx& c, TcState& s) {
+  if (!c.gemm_tc) return;
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(s.tmem_base) : "memory");
+  }
+}
+
+struct TcMaps {
+  CUtensorMap w[GEMM_KINDS];
+  CUtensorMap act[ACT_BUFS][TC_BOXES];
+};
+
+// ---- the GEMM phase -----------------------------------------------------------------------------
+__device__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int which, int layer, float* smem_f, TcState& tc) {
+  const int T = a.M, N = a.N, K = a.K;
+  if (T <= 0) return;  // uniform over the grid
+  const TcMaps* maps = reinterpret_cast<const TcMaps*>(c.tc_maps);
+  const int kblocks = K / 64;
+  const int ntiles = (N + 127) / 128;
+  const int passes = (T + 255) / 256;
+  int box_id = TC_BOXES - 1;
+  if (passes == 1) {
+    box_id = 0;
+    while ((16 << box_id) < T) ++box_id;
+  }
+  const int box_rows = 16 << box_id;
+  const int act_id = which == GEMM_O ? ACT_ATTN : which == GEMM_DOWN ? ACT_ACT : which == GEMM_LMHEAD ? ACT_XS : ACT_XN;
+  const CUtensorMap* map_a = &maps->w[which];
+  const CUtensorMap* map_b = &maps->act[act_id][box_id];
+  const int row_a0 = which == GEMM_LMHEAD ? 0 : layer * N;
+  const uint32_t stage_bytes = TC_A_BYTES + (uint32_t)box_rows * 128u;
+  int S = TC_TILE_BUDGET / (int)stage_bytes;
+  if (S > TC_MAX_STAGES) S = TC_MAX_STAGES;
+  // tiles need 1024-byte alignment for the 128-byte swizzle
+  const uint32_t raw = smem_u32(smem_f);
+  char* tiles = reinterpret_cast<char*>(smem_f) + (((raw + 1023u) & ~1023u) - raw);
+
+  const long long total = (long long)passes * ntiles * kblocks;
+  const long long u0 = total * blockIdx.x / gridDim.x, u1 = total * (blockIdx.x + 1) / gridDim.x;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  volatile int* dead = &g_tc.dead;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      int stage = 0;
+      for (long long u = u0; u < u1; ++u) {
+        const int kb = (int)(u % kblocks);
+        const int nt = (int)((u / kblocks) % ntiles);
+        const int pass = (int)(u / ((long long)kblocks * ntiles));
+        // the n-th fill of a stage waits for its (n-1)-th release
+        if (!mbar_wait(c, &g_tc.empty[stage], ((tc.fill_bits >> stage) & 1u) ^ 1u, dead)) break;
+        tc.fill_bits ^= 1u << stage;
+        mbar_expect_tx(&g_tc.full[stage], stage_bytes);
+        char* sa = tiles + (size_t)stage * stage_bytes;
+        tma_load_2d(sa, map_a, kb * 64, row_a0 + nt * 128, &g_tc.full[stage]);
+        tma_load_2d(sa + TC_A_BYTES, map_b, kb * 64, pass * 256, &g_tc.full[stage]);
+        if (++stage == S) stage = 0;
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      int stage = 0;
+      int abuf = 0;
+      long long u = u0;
+      while (u < u1) {
+        const long long seg_end = min(u1, (u / kblocks + 1) * (long long)kblocks);
+        const int pass = (int)(u / ((long long)kblocks * ntiles));
+        const int rows = min(256, T - pass * 256);
+        const int n_mma = (rows + 15) & ~15;
+        const uint32_t idesc = idesc_bf16(n_mma);
+        const uint32_t d_tmem = tc.tmem_base + (uint32_t)abuf * 256u;
+        if (!mbar_wait(c, &g_tc.acc_empty[abuf], ((tc.acc_mma >> abuf) & 1u) ^ 1u, dead)) break;
+        tc.acc_mma ^= 1u << abuf;
+        tc_fence_after();
+        bool first = true;
+        bool ok = true;
+        for (; u < seg_end; ++u) {
+          if (!mbar_wait(c, &g_tc.full[stage], (tc.use_bits >> stage) & 1u, dead)) { ok = false; break; }
+          tc.use_bits ^= 1u << stage;
+          tc_fence_after();
+          const uint32_t sa = smem_u32(tiles + (size_t)stage * stage_bytes);
+          const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sa + TC_A_BYTES);
+#pragma unroll
+          for (int k16 = 0; k16 < 4; ++k16) {
+            // 16 bf16 = 32 bytes further along K inside the swizzle atom: +2 in 16-byte units
+            umma_bf16(d_tmem, da + (uint64_t)(2 * k16), db + (uint64_t)(2 * k16), idesc, (first && k16 == 0) ? 0u : 1u);
+          }
+          first = false;
+          umma_commit(&g_tc.empty[stage]);
+          if (++stage == S) stage = 0;
+        }
+        if (!ok) break;
+        umma_commit(&g_tc.acc_full[abuf]);
+        abuf ^= 1;
+      }
+    }
+  } else if (warp >= 4) {
+    const int q = warp & 3;  // TMEM lane quarter this warp may read
+    int abuf = 0;
+    long long u = u0;
+    while (u < u1) {
+      const long long seg_end = min(u1, (u / kblocks + 1) * (long long)kblocks);
+      const int kb0 = (int)(u % kblocks);
+      const int kb1 = kb0 + (int)(seg_end - u);
+      const int nt = (int)((u / kblocks) % ntiles);
+      const int pass = (int)(u / ((long long)kblocks * ntiles));
+      const int rows = min(256, T - pass * 256);
+      const int n_mma = (rows + 15) & ~15;
+      const bool whole = (kb0 == 0 && kb1 == kblocks);
+      if (!mbar_wait(c, &g_tc.acc_full[abuf], (tc.acc_epi >> abuf) & 1u, dead)) break;
+      tc.acc_epi ^= 1u << abuf;
+      tc_fence_after();
+      const int n = nt * 128 + q * 32 + lane;
+      const uint32_t taddr = tc.tmem_base + (uint32_t)abuf * 256u + ((uint32_t)(q * 32) << 16);
+      for (int c0 = 0; c0 < n_mma; c0 += 16) {
+        float v[16];
+        tmem_ld16(taddr + (uint32_t)c0, v);
+        if (n < N) {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const int t = pass * 256 + c0 + j;
+            if (t < T) {
+              float* o = a.out + (size_t)t * a.ldo + n;
+              if (whole && !a.accumulate) *o = v[j];
+              else atomicAdd(o, v[j]);
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&g_tc.acc_empty[abuf]);
+      abuf ^= 1;
+      u = seg_end;
+    }
+  }
+  __syncthreads();
+}
+
+// ---- host side: tensor maps ----------------------------------------------------------------
+inline size_t tc_smem_bytes() { return (size_t)TC_TILE_BUDGET + 1024; }
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+inline EncodeTiledFn tc_encode_fn() {
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess) return nullptr;
+  if (qres != cudaDriverEntryPointSuccess) return nullptr;
+  return reinterpret_cast<EncodeTiledFn>(fn);
+}
+
+// bf16 row-major [rows][cols] matrix, box = box_rows x 64 columns, 128-byte swizzle
+inline bool tc_make_map(EncodeTiledFn enc, CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols,
+                        uint32_t box_rows, bool streaming) {
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {cols * 2};
+  cuuint32_t box[2] = {64, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  const CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                         streaming ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+// The tensor-core path needs every contraction length to be a multiple of 64 (one swizzled
+// smem row) and 16-byte aligned rows.
+inline int tc_shape_ok(const DevCtx& c) {
+  return c.dtype == 0 && c.d % 64 == 0 && c.q_dim % 64 == 0 && c.F % 64 == 0 && c.V % 4 == 0 && c.E == 0;
+}
+inline int tc_available() { return tc_encode_fn() != nullptr; }
+
+inline int tc_host_setup(TcHost& h, DevCtx& c) {
+  EncodeTiledFn enc = tc_encode_fn();
+  if (!enc) return -7;
+  TcMaps* hm = new TcMaps();
+  const char* w = c.w_base;
+  const uint64_t L = c.L;
+  bool ok = true;
+  ok &= tc_make_map(enc, &hm->w[GEMM_QKV], w + c.w_off[1], L * c.qkv_dim, c.d, 128, true);
+  ok &= tc_make_map(enc, &hm->w[GEMM_O], w + c.w_off[2], L * c.d, c.q_dim, 128, true);
+  ok &= tc_make_map(enc, &hm->w[GEMM_GU], w + c.w_off[3], L * 2 * c.F, c.d, 128, true);
+  ok &= tc_make_map(enc, &hm->w[GEMM_DOWN], w + c.w_off[4], L * c.d, c.F, 128, true);
+  ok &= tc_make_map(enc, &hm->w[GEMM_LMHEAD], w + c.w_off[9], c.V, c.d, 128, true);
+  const void* bufs[ACT_BUFS] = {c.xn, c.attn, c.act, c.xs};
+  const uint64_t rows[ACT_BUFS] = {(uint64_t)c.Tmax, (uint64_t)c.Tmax, (uint64_t)c.Tmax, (uint64_t)c.MB};
+  const uint64_t cols[ACT_BUFS] = {(uint64_t)c.d, (uint64_t)c.q_dim, (uint64_t)c.F, (uint64_t)c.d};
+  for (int b = 0; b < ACT_BUFS; ++b)
+    for (int i = 0; i < TC_BOXES; ++i) ok &= tc_make_map(enc, &hm->act[b][i], bufs[b], rows[b], cols[b], 16u << i, false);
+  int rc = 0;
+  if (!ok) rc = -7;
+  if (rc == 0 && cudaMalloc(&h.d_maps, sizeof(TcMaps)) != cudaSuccess) rc = -6;
+  if (rc == 0 && cudaMemcpy(h.d_maps, hm, sizeof(TcMaps), cudaMemcpyHostToDevice) != cudaSuccess) rc = -7;
+  delete hm;
+  if (rc == 0) c.tc_maps = h.d_maps;
+  return rc;
+}
+inline void tc_host_free(TcHost& h) {
+  if (h.d_maps) cudaFree(h.d_maps);
+  h.d_maps = nullptr;
+}
 
 }  // namespace blink

@@ -126,3 +126,41 @@ def test_sampler_alone_bit_exact_on_oracle_logits():
                         np.full(n, 7, np.uint64), np.arange(n, dtype=np.int32), np.full(n, 42, np.uint64))
     w2 = [S.sample(logits[5], 50, 0.8, 7, i, 42) for i in range(n)]
     assert list(g2) == w2
+
+
+# ---- tensor-core (tcgen05 / TMEM / TMA) path of the dense contractions ---------------------------
+def test_config1_bf16_tensor_core_path_matches_oracle():
+    model, sched = model_cfg(1, dtype="bf16"), sched_cfg(1)
+    reqs = make_requests(1)
+    w = make_weights(model, 1234, "cpu")
+    err, n_margin, trace, toks, ora = _compare(model, sched, reqs, w, O2.round_bf16, TOL_BF16, gemm_impl=B.GEMM_TC)
+    print(f"C1 bf16 tensor cores: max-abs logit error {err:.3e}, {n_margin} in-margin decisions")
+    assert err <= TOL_BF16
+
+
+def test_tensor_core_path_multi_pass_ragged_shapes():
+    """More than 256 rows in a step (two token passes), 24 k-blocks, 35 n-tiles, GQA 4:1 with
+    head_dim 128, non-unit gains: every stream-K segment kind (whole tile, head, tail) occurs."""
+    model = model_cfg(1, d_model=512, n_q_heads=4, n_kv_heads=1, head_dim=128, d_ff=1536, vocab=4480, dtype="bf16")
+    sched = sched_cfg(1, prefill_chunk_tokens=300, max_batch=8, n_blocks=256, max_prompt=320, max_new=8)
+    rng = np.random.default_rng(21)
+    from synth.workload import Request
+    reqs = [Request(t, 0.0, rng.integers(0, model.vocab, size=int(p)).astype(np.int32), 6)
+            for t, p in enumerate([310, 17, 301, 64, 129, 256, 5, 300, 33])]
+    w = make_weights(model, 77, "cpu", random_gains=True)
+    err, n_margin, trace, toks, ora = _compare(model, sched, reqs, w, O2.round_bf16, TOL_BF16, gemm_impl=B.GEMM_TC)
+    print(f"multi-pass tensor cores: max-abs logit error {err:.3e}; max rows/step "
+          f"{max(sum(s[4] for s in r['scheduled']) for r in trace)}")
+    assert err <= TOL_BF16
+    assert max(sum(s[4] for s in r["scheduled"]) for r in trace) > 256
+
+
+def test_tensor_core_and_cuda_core_paths_agree():
+    model, sched = model_cfg(1, dtype="bf16"), sched_cfg(1)
+    reqs = make_requests(1, n_requests=4)
+    w = make_weights(model, 3, "cpu", random_gains=True)
+    forced = {r.ticket: [int(x) for x in np.random.default_rng(r.ticket).integers(0, 4096, size=r.max_new)] for r in reqs}
+    a = gpu_run_forced(model, sched, reqs, w, forced, gemm_impl=B.GEMM_SIMT)
+    b = gpu_run_forced(model, sched, reqs, w, forced, gemm_impl=B.GEMM_TC, exec_mode=B.EXEC_STEPPED)
+    assert np.abs(a[2] - b[2]).max() < TOL_BF16  # same bf16 products, other summation order, so roundings flip
+    assert_traces_equal([{**r, "sampled": []} for r in a[0]], [{**r, "sampled": []} for r in b[0]])
