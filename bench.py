@@ -283,6 +283,11 @@ def main():
     ap.add_argument("--skip-latency", action="store_true")
     ap.add_argument("--closed-batch", default="", help="N,I,O: use an N x I -> O closed batch instead of the stream")
     ap.add_argument("--kv-fraction", type=float, default=0.8)
+    ap.add_argument("--kv-blocks", type=int, default=0, help="cap the KV pool at this many blocks")
+    ap.add_argument("--layers", type=int, default=0,
+                    help="profiling aid: keep only this many layers of the configuration's shape")
+    ap.add_argument("--exec", default="manual", choices=["manual", "stepped"],
+                    help="stepped = one host launch per phase (profiling aid for ncu; prints no bench value)")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -293,8 +298,12 @@ def main():
     from synth.workload import closed_batch
     cfg_i = args.config
     m = model_cfg(cfg_i)
+    if args.layers > 0:
+        m = m.with_(n_layers=args.layers)
     sched = sched_cfg(cfg_i)
     workload = f"C{cfg_i} {('8B' if cfg_i in (3, 4) else '')} stream".replace("  ", " ")
+    if args.layers > 0:
+        workload += f" ({args.layers} layers only)"
 
     if args.impl == "reference":
         if rank != 0:
@@ -354,6 +363,8 @@ def main():
     n_blocks = int((free - lib_reserve) * args.kv_fraction) // blk
     if sched.n_blocks > 0:
         n_blocks = min(n_blocks, sched.n_blocks)
+    if args.kv_blocks > 0:
+        n_blocks = min(n_blocks, args.kv_blocks)
     kv = torch.empty(n_blocks * blk, dtype=torch.uint8, device=dev)
     sched = sched.with_(n_blocks=n_blocks)
     log(f"[bench] KV pool {n_blocks} blocks = {n_blocks * blk / 1e9:.1f} GB ({n_blocks * 16} tokens)")
@@ -367,8 +378,30 @@ def main():
         reqs = make_requests(cfg_i, rate=args.rate)
         ramp = args.ramp if args.ramp >= 0 else 600
 
-    # ---- closed-loop saturation run: ramp, W warm-up steps, then exactly K timed steps --------
     W, K = max(3, args.warmup), args.steps
+    if args.exec == "stepped":
+        # profiling aid: the same device code, one host launch per phase, so that a profiler sees
+        # the phases as separate kernels (1 control launch + 9 per layer + 3 per iteration)
+        eng = B.Blink(m, sched, wbuf, kv, exec_mode=B.EXEC_STEPPED, gemm_impl=gemm_impl, stats_iters=ramp + W + K + 64)
+        try:
+            for r in reqs:
+                eng.submit_request(r)
+            eng.blink_step(ramp + W)
+            eng.blink_poll(4096, 0)
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            eng.blink_step(K)
+            dt = time.perf_counter() - t0
+            its = eng.blink_get_iter_stats()[-K:]
+            print(json.dumps(dict(mode="stepped (profiling aid, not a bench value)", workload=workload, steps=K,
+                                  wall_ms_per_step=dt * 1e3 / K, rows_per_step=float(its["n_tokens"].mean()),
+                                  decode_rows_per_step=float(its["n_decode"].mean()),
+                                  launches_per_step=1 + 9 * m.n_layers + 3)), flush=True)
+        finally:
+            eng.blink_destroy()
+        return
+
+    # ---- closed-loop saturation run: ramp, W warm-up steps, then exactly K timed steps --------
     eng = B.Blink(m, sched, wbuf, kv, exec_mode=B.EXEC_MANUAL, gemm_impl=gemm_impl, stats_iters=ramp + W + K + 64,
                   idle_exit_us=200_000)
     try:
@@ -445,6 +478,7 @@ def main():
                             parallelism="replicas" if world > 1 else "1 GPU", gemm=args.gemm),
                 gpu_launches=1, clocks=clk, roofline=roof,
                 step_ms_device=dict(p50=float(np.median(step_dev_ms)), max=float(step_dev_ms.max())),
+                phase_ms_per_step={n: float(its["phase_ns"][:, i].mean() / 1e6) for i, n in enumerate(B.PHASE_NAMES)},
                 control_plane_us=dict(p50=float(np.median(ctrl_us)), max=float(ctrl_us.max())))
     if cpu_baseline is not None:
         line["cpu_baseline"] = cpu_baseline

@@ -173,6 +173,11 @@ typedef struct blink_iter_stat {
   int64_t ctx_tokens;     /* sum over rows of keys attended (attention flops)  */
   int64_t kv_tokens;      /* sum over requests in the step of their context length after the
                              step: KV tokens an ideal kernel reads once per step              */
+  uint64_t phase_ns[16];  /* persistent / manual mode: device time per phase kind, summed over the
+                             layers, each including the grid barrier that closes it.  Index:
+                             0 norm1(+embedding) 1 QKV 2 RoPE+KV write 3 attention 4 O 5 norm2
+                             6 gate/up 7 SwiGLU 8 down 9 final norm 10 LM head 11 sampling;
+                             12..15 unused (zero)                                             */
 } blink_iter_stat;
 
 /* Bytes of the flat weight buffer for a model shape (dtype taken from cfg). */

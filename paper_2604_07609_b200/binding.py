@@ -69,12 +69,16 @@ class blink_stats(C.Structure):
 class blink_iter_stat(C.Structure):
     _fields_ = [("t_begin_ns", C.c_uint64), ("t_forward_ns", C.c_uint64), ("t_end_ns", C.c_uint64),
                 ("n_tokens", C.c_int32), ("n_decode", C.c_int32), ("n_sample_rows", C.c_int32),
-                ("n_items", C.c_int32), ("ctx_tokens", C.c_int64), ("kv_tokens", C.c_int64)]
+                ("n_items", C.c_int32), ("ctx_tokens", C.c_int64), ("kv_tokens", C.c_int64),
+                ("phase_ns", C.c_uint64 * 16)]
 
 
 ITER_STAT_DTYPE = np.dtype([("t_begin_ns", "<u8"), ("t_forward_ns", "<u8"), ("t_end_ns", "<u8"),
                             ("n_tokens", "<i4"), ("n_decode", "<i4"), ("n_sample_rows", "<i4"),
-                            ("n_items", "<i4"), ("ctx_tokens", "<i8"), ("kv_tokens", "<i8")])
+                            ("n_items", "<i4"), ("ctx_tokens", "<i8"), ("kv_tokens", "<i8"),
+                            ("phase_ns", "<u8", (16,))])
+PHASE_NAMES = ["norm1", "qkv", "rope_kv", "attention", "o", "norm2", "gate_up", "swiglu", "down", "final_norm",
+               "lm_head", "sample"]
 EVENT_DTYPE = np.dtype([("ticket", "<u8"), ("user_tag", "<u8"), ("index", "<i4"), ("token", "<i4"),
                         ("is_first", "<i4"), ("is_last", "<i4"), ("t_device_ns", "<u8"), ("t_host_ns", "<u8"),
                         ("t_submit_ns", "<u8")])

@@ -103,19 +103,24 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) blink_loop_kernel(const __grid
     if (*(volatile int*)&c.ss->cmd != CMD_RUN) break;
     if (!c.control_only) {
       bool ok = true;
+      // CTA 0 keeps a per-phase-kind device time of the open iteration (a phase's time includes
+      // the barrier that closes it); recorded only when per-iteration statistics are kept
+      const bool timed = c.stats_cap > 0 && blockIdx.x == 0 && threadIdx.x == 0;
+      uint64_t t_prev = timed ? global_timer_ns() : 0;
       for (int layer = 0; layer < c.L && ok; ++layer) {
         for (int ph = PH_NORM1; ph <= PH_DOWN && ok; ++ph) {
           run_phase<WT>(c, ph, layer, smem, tc);
           ok = grid_barrier(c, gen);
+          if (timed) { const uint64_t t = global_timer_ns(); c.ss->cur_phase_ns[ph] += t - t_prev; t_prev = t; }
         }
       }
       for (int ph = PH_FNORM; ph <= PH_SAMPLE && ok; ++ph) {
         run_phase<WT>(c, ph, 0, smem, tc);
-        if (ph != PH_SAMPLE) ok = grid_barrier(c, gen);
+        ok = grid_barrier(c, gen);
+        if (timed) { const uint64_t t = global_timer_ns(); c.ss->cur_phase_ns[ph] += t - t_prev; t_prev = t; }
       }
       if (!ok) break;
-    }
-    if (!grid_barrier(c, gen)) break;
+    } else if (!grid_barrier(c, gen)) break;
   }
   tc_fini(c, tc);
   if (blockIdx.x == 0 && threadIdx.x == 0) {

@@ -214,7 +214,9 @@ __device__ void post_step(const DevCtx& c) {
       st.n_items = n_items;
       st.ctx_tokens = ss->cur_ctx;
       st.kv_tokens = ss->cur_kv;
+      for (int i = 0; i < N_PHASE_TIMERS; ++i) st.phase_ns[i] = ss->cur_phase_ns[i];
     }
+    for (int i = 0; i < N_PHASE_TIMERS; ++i) ss->cur_phase_ns[i] = 0;
     ss->iter += 1;
     ss->cur_hdr = -1;
     ss->pending_post = 0;

@@ -77,6 +77,8 @@ enum DevError : int32_t {
 enum StepCmd : int32_t { CMD_NONE = 0, CMD_RUN = 1, CMD_EXIT = 2 };
 enum { PHASE_FREE = 0, PHASE_PREFILL = 1, PHASE_DECODE = 2 };
 
+constexpr int N_PHASE_TIMERS = 16;
+
 // Scalars of the scheduler that live in HBM and survive kernel re-instantiation.
 struct SchedState {
   unsigned long long seen;          // submit entries moved into the ring
@@ -102,6 +104,7 @@ struct SchedState {
   unsigned long long cur_t_begin, cur_t_forward;
   int exit_reason;
   int pad;
+  unsigned long long cur_phase_ns[N_PHASE_TIMERS];  // device time per phase kind of the open iteration
 };
 
 struct IterStat {
@@ -109,6 +112,7 @@ struct IterStat {
   int32_t n_tokens, n_decode, n_sample_rows, n_items;
   int64_t ctx_tokens;
   int64_t kv_tokens;
+  uint64_t phase_ns[N_PHASE_TIMERS];
 };
 
 constexpr int TRACE_HDR_WORDS = 12;
