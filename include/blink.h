@@ -46,7 +46,8 @@ enum {
   BLINK_EDEVICE = -4,   /* the device loop reported an error (see blink_stats)  */
   BLINK_ETIMEDOUT = -5, /* a bounded wait ran out                               */
   BLINK_ENOMEM = -6,    /* allocation failed / pool too small                   */
-  BLINK_ECUDA = -7      /* a CUDA runtime or driver call failed                 */
+  BLINK_ECUDA = -7,     /* a CUDA runtime or driver call failed                 */
+  BLINK_ETOOBIG = -8    /* size beyond a fixed capacity (see blink_sample_noalloc) */
 };
 
 enum { BLINK_DTYPE_BF16 = 0, BLINK_DTYPE_FP32 = 1 };
@@ -261,6 +262,32 @@ int blink_get_iter_stats(blink_ctx* ctx, blink_iter_stat* out, int64_t capacity,
  * and frees a small device scratch. */
 int blink_sample(const float* logits, int rows, int vocab, const int32_t* top_k, const float* temperature,
                  const uint64_t* ticket, const int32_t* gen_index, const uint64_t* seed, int32_t* out);
+
+/* blink_sample for callers that cannot allocate.  The paper has no counterpart: this is a
+ * convenience of this library.  Some callers must not call cudaMalloc / cudaFree once they
+ * are running: a server that handed all free device memory to the KV pool at start-up (a
+ * later allocation can simply fail), or code on a path where the implicit device-wide
+ * synchronisation of cudaFree is not acceptable.  This variant computes exactly what
+ * blink_sample computes, row for row, but keeps its per-row parameters and results in a
+ * fixed scratch array that is part of the library image (32 KiB of device memory on every
+ * GPU that loads the library, held until the process exits) instead of a temporary
+ * allocation.  It calls no cudaMalloc, cudaFree or other allocating routine.
+ *
+ * Arguments as for blink_sample (`logits` DEVICE [rows][vocab] fp32; the parameter arrays and
+ * `out` HOST, length rows).  rows must not exceed BLINK_SAMPLE_NOALLOC_MAX_ROWS: a larger
+ * value is refused with BLINK_ETOOBIG before anything is touched; split the rows over
+ * several calls instead.
+ *
+ * The first call on each device looks up the device address of the scratch array (one
+ * runtime query, with that device current); make that first call before any stream capture
+ * begins.  All calls on a device share the one scratch array and it keeps the previous call's
+ * contents: every call overwrites the part it uses before the kernel reads it, nothing has
+ * to start at zero.  Calls that overlap on the same GPU (from several threads or processes
+ * sharing a context) would race on the array: the library serialises its own callers with a
+ * mutex, and the call is synchronous, so a single process is safe. */
+#define BLINK_SAMPLE_NOALLOC_MAX_ROWS 1024
+int blink_sample_noalloc(const float* logits, int rows, int vocab, const int32_t* top_k, const float* temperature,
+                         const uint64_t* ticket, const int32_t* gen_index, const uint64_t* seed, int32_t* out);
 
 const char* blink_strerror(int code);
 

@@ -16,7 +16,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libblink.so")
 
 BLINK_OK, BLINK_EAGAIN, BLINK_EINVAL, BLINK_ESTOPPED, BLINK_EDEVICE = 0, -1, -2, -3, -4
-BLINK_ETIMEDOUT, BLINK_ENOMEM, BLINK_ECUDA = -5, -6, -7
+BLINK_ETIMEDOUT, BLINK_ENOMEM, BLINK_ECUDA, BLINK_ETOOBIG = -5, -6, -7, -8
+SAMPLE_NOALLOC_MAX_ROWS = 1024
 DTYPE_BF16, DTYPE_FP32 = 0, 1
 EXEC_PERSISTENT, EXEC_STEPPED, EXEC_MANUAL = 0, 1, 2
 GEMM_AUTO, GEMM_SIMT, GEMM_TC = 0, 1, 2
@@ -85,7 +86,8 @@ EVENT_DTYPE = np.dtype([("ticket", "<u8"), ("user_tag", "<u8"), ("index", "<i4")
 
 EXPORTS = ["blink_weights_bytes", "blink_weight_offset", "blink_kv_blocks_for_bytes", "blink_create",
            "blink_start", "blink_submit", "blink_poll", "blink_step", "blink_run", "blink_stop", "blink_destroy",
-           "blink_get_stats", "blink_get_trace", "blink_get_iter_stats", "blink_sample", "blink_strerror"]
+           "blink_get_stats", "blink_get_trace", "blink_get_iter_stats", "blink_sample", "blink_sample_noalloc",
+           "blink_strerror"]
 
 _lib = None
 
@@ -130,6 +132,8 @@ def lib():
     L.blink_get_iter_stats.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, P(C.c_int64)]
     L.blink_sample.restype = C.c_int
     L.blink_sample.argtypes = [C.c_void_p, C.c_int, C.c_int] + [C.c_void_p] * 6
+    L.blink_sample_noalloc.restype = C.c_int
+    L.blink_sample_noalloc.argtypes = [C.c_void_p, C.c_int, C.c_int] + [C.c_void_p] * 6
     L.blink_strerror.restype = C.c_char_p
     L.blink_strerror.argtypes = [C.c_int]
     _lib = L
@@ -176,6 +180,27 @@ def blink_sample(logits, top_k, temperature, ticket, gen_index, seed) -> np.ndar
                             gi.ctypes.data, sd.ctypes.data, out.ctypes.data)
     if rc != BLINK_OK:
         raise BlinkError(rc, "blink_sample")
+    return out
+
+
+def blink_sample_noalloc(logits, top_k, temperature, ticket, gen_index, seed, raise_on_error=True):
+    """Same sampling as blink_sample, for callers that cannot allocate device memory (a server
+    whose memory budget is fixed at start-up, or code that must avoid the device-wide
+    synchronisation of cudaFree): the per-row parameters go through a fixed scratch array inside
+    the library, so at most SAMPLE_NOALLOC_MAX_ROWS rows per call.  Returns the tokens, or the
+    negative error code when raise_on_error is false."""
+    rows, vocab = logits.shape
+    assert logits.is_cuda and logits.is_contiguous() and logits.dtype.is_floating_point and logits.element_size() == 4
+    a = lambda v, dt: np.ascontiguousarray(v, dtype=dt)
+    tk, tp, ti, gi, sd = a(top_k, np.int32), a(temperature, np.float32), a(ticket, np.uint64), \
+        a(gen_index, np.int32), a(seed, np.uint64)
+    out = np.zeros(rows, dtype=np.int32)
+    rc = lib().blink_sample_noalloc(logits.data_ptr(), rows, vocab, tk.ctypes.data, tp.ctypes.data, ti.ctypes.data,
+                                    gi.ctypes.data, sd.ctypes.data, out.ctypes.data)
+    if rc != BLINK_OK:
+        if raise_on_error:
+            raise BlinkError(rc, "blink_sample_noalloc")
+        return rc
     return out
 
 

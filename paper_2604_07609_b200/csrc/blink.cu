@@ -368,6 +368,7 @@ const char* blink_strerror(int code) {
     case BLINK_ETIMEDOUT: return "timed out";
     case BLINK_ENOMEM: return "out of memory or pool too small";
     case BLINK_ECUDA: return "CUDA call failed";
+    case BLINK_ETOOBIG: return "size exceeds a fixed capacity";
     default: return "unknown error";
   }
 }
@@ -421,6 +422,67 @@ int blink_sample(const float* logits, int rows, int vocab, const int32_t* top_k,
   }
   cudaFree(d);
   return rc;
+}
+
+// ---- sampler for callers that cannot allocate --------------------------------------------------
+// Per-row parameters and results live in a fixed array inside the library image.  In host code
+// the symbol below is only a handle: the device address comes from cudaGetSymbolAddress, once
+// per device, with that device current.
+namespace {
+constexpr size_t NOALLOC_ROW_BYTES = 8 + 8 + 4 + 4 + 4 + 4;  // ticket, seed, top_k, temperature, gen_index, out
+constexpr int NOALLOC_MAX_DEVICES = 64;
+}  // namespace
+static __device__ __align__(256) unsigned char g_sample_scratch[BLINK_SAMPLE_NOALLOC_MAX_ROWS * NOALLOC_ROW_BYTES];
+namespace {
+std::mutex g_noalloc_mu;
+void* g_noalloc_ptr[NOALLOC_MAX_DEVICES] = {nullptr};
+}  // namespace
+
+int blink_sample_noalloc(const float* logits, int rows, int vocab, const int32_t* top_k, const float* temperature,
+                         const uint64_t* ticket, const int32_t* gen_index, const uint64_t* seed, int32_t* out) {
+  if (!logits || rows < 1 || vocab < 2 || !top_k || !temperature || !ticket || !gen_index || !seed || !out)
+    return BLINK_EINVAL;
+  if (rows > BLINK_SAMPLE_NOALLOC_MAX_ROWS) {
+    fprintf(stderr, "blink_sample_noalloc: %d rows exceed the fixed scratch capacity of %d rows; split the call\n", rows,
+            BLINK_SAMPLE_NOALLOC_MAX_ROWS);
+    return BLINK_ETOOBIG;
+  }
+  for (int r = 0; r < rows; ++r)
+    if (top_k[r] < 0 || top_k[r] > MAX_TOPK || (top_k[r] > 0 && !(temperature[r] > 0.f))) return BLINK_EINVAL;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= NOALLOC_MAX_DEVICES) return BLINK_ECUDA;
+  std::lock_guard<std::mutex> g(g_noalloc_mu);  // one user of the shared scratch at a time
+  if (!g_noalloc_ptr[dev]) {
+    void* p = nullptr;
+    const cudaError_t e = cudaGetSymbolAddress(&p, g_sample_scratch);
+    if (e != cudaSuccess || !p) {
+      fprintf(stderr, "blink_sample_noalloc: cudaGetSymbolAddress failed: %s\n", cudaGetErrorString(e));
+      return BLINK_ECUDA;
+    }
+    g_noalloc_ptr[dev] = p;
+  }
+  // carve the scratch with the capacity as stride, so every sub-array stays naturally aligned
+  char* d = static_cast<char*>(g_noalloc_ptr[dev]);
+  const size_t cap = BLINK_SAMPLE_NOALLOC_MAX_ROWS, n = (size_t)rows;
+  unsigned long long* d_ticket = reinterpret_cast<unsigned long long*>(d);
+  unsigned long long* d_seed = d_ticket + cap;
+  int* d_topk = reinterpret_cast<int*>(d_seed + cap);
+  float* d_temp = reinterpret_cast<float*>(d_topk + cap);
+  int* d_gen = reinterpret_cast<int*>(d_temp + cap);
+  int* d_out = d_gen + cap;
+  if (cudaMemcpy(d_ticket, ticket, n * 8, cudaMemcpyHostToDevice) != cudaSuccess ||
+      cudaMemcpy(d_seed, seed, n * 8, cudaMemcpyHostToDevice) != cudaSuccess ||
+      cudaMemcpy(d_topk, top_k, n * 4, cudaMemcpyHostToDevice) != cudaSuccess ||
+      cudaMemcpy(d_temp, temperature, n * 4, cudaMemcpyHostToDevice) != cudaSuccess ||
+      cudaMemcpy(d_gen, gen_index, n * 4, cudaMemcpyHostToDevice) != cudaSuccess ||
+      cudaMemset(d_out, 0xff, n * 4) != cudaSuccess)  // results of an earlier call must not show through
+    return BLINK_ECUDA;
+  const int grid = rows < 1184 ? rows : 1184;
+  blink_sample_kernel<<<grid, FWD_THREADS, SAMPLE_SMEM_FLOATS * sizeof(float)>>>(logits, rows, vocab, d_topk, d_temp,
+                                                                                 d_ticket, d_gen, d_seed, d_out);
+  if (cudaGetLastError() != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) return BLINK_ECUDA;
+  if (cudaMemcpy(out, d_out, n * 4, cudaMemcpyDeviceToHost) != cudaSuccess) return BLINK_ECUDA;
+  return BLINK_OK;
 }
 
 int blink_create(const blink_model_cfg* model, const blink_sched_cfg* sched, const blink_kv_pool* kv,
