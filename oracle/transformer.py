@@ -19,7 +19,8 @@ KV pool, driven by the scheduler oracle's block tables).
 
 `act_round` models the reduced-precision storage points of the bf16 mode: values
 are rounded to bf16 exactly where the bf16 data path stores 16-bit values (GEMM
-operand inputs and the KV pool); everything else stays in `dtype` (float64 by
+operand inputs, the rotated queries handed to attention, and the KV pool; the
+paper's engine runs its attention in 16-bit precision, Section 6.1); everything else stays in `dtype` (float64 by
 default).  With act_round=None this is the pure high-precision reference.
 """
 from __future__ import annotations
@@ -143,7 +144,7 @@ def forward_dense(cfg, W: Weights, tokens, act_round=None, return_hidden=False):
         q = qkv[:, : cfg.q_dim].reshape(T, cfg.n_q_heads, cfg.head_dim)
         k = qkv[:, cfg.q_dim: cfg.q_dim + cfg.kv_dim].reshape(T, cfg.n_kv_heads, cfg.head_dim)
         v = qkv[:, cfg.q_dim + cfg.kv_dim:].reshape(T, cfg.n_kv_heads, cfg.head_dim)
-        q = rope(q, pos, cfg.rope_theta)
+        q = rb(rope(q, pos, cfg.rope_theta))       # q is a 16-bit operand of the attention contraction
         k = rb(rope(k, pos, cfg.rope_theta))       # K/V are stored in the cache dtype
         v = rb(v)
         a = attention_rows(q, k, v, pos, n_rep).reshape(T, cfg.q_dim)
@@ -196,7 +197,7 @@ class PagedModel:
             q = qkv[:, : cfg.q_dim].reshape(T, cfg.n_q_heads, cfg.head_dim)
             k = qkv[:, cfg.q_dim: cfg.q_dim + cfg.kv_dim].reshape(T, cfg.n_kv_heads, cfg.head_dim)
             v = qkv[:, cfg.q_dim + cfg.kv_dim:].reshape(T, cfg.n_kv_heads, cfg.head_dim)
-            q = rope(q, pos, cfg.rope_theta)
+            q = rb(rope(q, pos, cfg.rope_theta))
             k = rb(rope(k, pos, cfg.rope_theta))
             v = rb(v)
             # write this step's K/V into the pool at block_table[pos // block], pos % block

@@ -4,10 +4,12 @@ from __future__ import annotations
 import os
 import subprocess
 import sys
+from concurrent.futures import ThreadPoolExecutor
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libblink.so")
+OBJ = os.path.join(HERE, "_build")
 
 
 def _newest(paths):
@@ -25,18 +27,32 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= _newest(srcs):
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-           "-Xcompiler", "-fPIC", "-shared",
-           "-o", LIB, os.path.join(CSRC, "blink.cu")]
+    flags = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC"]
     if verbose:
-        cmd.insert(1, "-Xptxas")
-        cmd.insert(2, "-v")
-    r = subprocess.run(cmd, capture_output=True, text=True)
+        flags += ["-Xptxas", "-v"]
+    os.makedirs(OBJ, exist_ok=True)
+    units = [f for f in sorted(os.listdir(CSRC)) if f.endswith(".cu")]
+
+    def compile_one(f):
+        obj = os.path.join(OBJ, f[:-3] + ".o")
+        r = subprocess.run([nvcc] + flags + ["-c", os.path.join(CSRC, f), "-o", obj], capture_output=True, text=True)
+        return f, obj, r
+
+    # one translation unit per kernel variant family, compiled side by side
+    with ThreadPoolExecutor(max_workers=min(len(units), os.cpu_count() or 1)) as ex:
+        results = list(ex.map(compile_one, units))
+    log = ""
+    for f, obj, r in results:
+        log += f"==== {f}\n{r.stdout}{r.stderr}"
+        if r.returncode != 0:
+            sys.stderr.write(log)
+            raise RuntimeError(f"nvcc failed compiling {f}")
+    r = subprocess.run([nvcc, "-shared", "-o", LIB] + [obj for _, obj, _ in results], capture_output=True, text=True)
     if r.returncode != 0:
         sys.stderr.write(r.stdout + r.stderr)
-        raise RuntimeError("nvcc failed building libblink.so")
+        raise RuntimeError("nvcc failed linking libblink.so")
     if verbose:
-        print(r.stdout + r.stderr)
+        print(log)
     return LIB
 
 

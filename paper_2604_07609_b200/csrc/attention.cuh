@@ -244,7 +244,7 @@ __device__ __forceinline__ void attn_decode_stream(const DevCtx& c, int layer, c
       }
     }
     const int s = n_consumed % ATT_NS;
-    if (!mbar_wait(c, &bars[s], (as.par >> s) & 1u, dead)) break;
+    if (!__all_sync(FULL, mbar_wait(c, &bars[s], (as.par >> s) & 1u, dead))) break;  // uniform exit
     as.par ^= 1u << s;
     const char* kt = ring + s * STAGE;
     const char* vt = kt + TILE;

@@ -23,113 +23,10 @@
 #include "dev_ctx.cuh"
 #include "forward.cuh"
 #include "gemm_tc.cuh"
+#include "attention.cuh"
+#include "kernel_set.h"
 
 namespace blink {
-
-enum Phase : int {
-  PH_NORM1 = 0, PH_QKV, PH_ROPE, PH_ATTN, PH_O, PH_NORM2, PH_GU, PH_SILU, PH_DOWN,
-  PH_FNORM, PH_LMHEAD, PH_SAMPLE, PH_COUNT
-};
-
-template <typename WT>
-__device__ __forceinline__ void gemm_dispatch(const DevCtx& c, const GemmArgs& a, int which, int layer, float* smem,
-                                              TcState& tc) {
-  if (c.gemm_tc) phase_gemm_tc(c, a, which, layer, smem, tc);
-  else phase_gemm_simt<WT>(a);
-}
-
-template <typename WT, int HD>
-__device__ __forceinline__ void attention_dispatch(const DevCtx& c, int layer, float* smem) {
-  switch (c.n_rep) {
-    case 1: phase_attention<WT, HD, 1>(c, layer, smem); break;
-    case 2: phase_attention<WT, HD, 2>(c, layer, smem); break;
-    case 4: phase_attention<WT, HD, 4>(c, layer, smem); break;
-    default: phase_attention<WT, HD, 8>(c, layer, smem); break;
-  }
-}
-
-template <typename WT>
-__device__ void run_phase(const DevCtx& c, int phase, int layer, float* smem, TcState& tc) {
-  const int T = c.ss->cur_T;
-  const size_t esz = sizeof(WT);
-  switch (phase) {
-    case PH_NORM1: phase_norm<WT>(c, layer, 0); break;
-    case PH_QKV: {
-      GemmArgs a{c.xn, c.w_base + c.w_off[1] + (size_t)layer * c.qkv_dim * c.d * esz, c.qkv, T, c.qkv_dim, c.d,
-                 c.qkv_dim, 0};
-      gemm_dispatch<WT>(c, a, GEMM_QKV, layer, smem, tc);
-    } break;
-    case PH_ROPE: phase_rope_kv<WT>(c, layer); break;
-    case PH_ATTN:
-      if (c.hd == 64) attention_dispatch<WT, 64>(c, layer, smem);
-      else attention_dispatch<WT, 128>(c, layer, smem);
-      break;
-    case PH_O: {
-      GemmArgs a{c.attn, c.w_base + c.w_off[2] + (size_t)layer * c.d * c.q_dim * esz, c.h, T, c.d, c.q_dim, c.d, 1};
-      gemm_dispatch<WT>(c, a, GEMM_O, layer, smem, tc);
-    } break;
-    case PH_NORM2: phase_norm<WT>(c, layer, 1); break;
-    case PH_GU: {
-      GemmArgs a{c.xn, c.w_base + c.w_off[3] + (size_t)layer * 2 * c.F * c.d * esz, c.gu, T, 2 * c.F, c.d, 2 * c.F, 0};
-      gemm_dispatch<WT>(c, a, GEMM_GU, layer, smem, tc);
-    } break;
-    case PH_SILU: phase_silu_mul<WT>(c); break;
-    case PH_DOWN: {
-      GemmArgs a{c.act, c.w_base + c.w_off[4] + (size_t)layer * c.d * c.F * esz, c.h, T, c.d, c.F, c.d, 1};
-      gemm_dispatch<WT>(c, a, GEMM_DOWN, layer, smem, tc);
-    } break;
-    case PH_FNORM: phase_final_norm<WT>(c); break;
-    case PH_LMHEAD: {
-      GemmArgs a{c.xs, c.w_base + c.w_off[9], c.logits, c.ss->cur_rows, c.V, c.d, c.V, 0};
-      gemm_dispatch<WT>(c, a, GEMM_LMHEAD, 0, smem, tc);
-    } break;
-    case PH_SAMPLE: phase_sample(c, smem); break;
-    default: break;
-  }
-}
-
-// ---- persistent loop -----------------------------------------------------------------
-template <typename WT>
-__global__ void __launch_bounds__(FWD_THREADS, 1) blink_loop_kernel(const __grid_constant__ DevCtx c) {
-  extern __shared__ __align__(1024) float smem[];
-  unsigned int gen = 0;
-  if (threadIdx.x == 0) gen = ld_acquire_gpu_u32(&c.ss->bar_gen);
-  long long launch_iters = 0;
-  TcState tc;
-  tc_init(c, smem, tc);
-  while (true) {
-    if (blockIdx.x == 0) control_phase(c, launch_iters);
-    if (!grid_barrier(c, gen)) break;
-    if (*(volatile int*)&c.ss->cmd != CMD_RUN) break;
-    if (!c.control_only) {
-      bool ok = true;
-      // CTA 0 keeps a per-phase-kind device time of the open iteration (a phase's time includes
-      // the barrier that closes it); recorded only when per-iteration statistics are kept
-      const bool timed = c.stats_cap > 0 && blockIdx.x == 0 && threadIdx.x == 0;
-      uint64_t t_prev = timed ? global_timer_ns() : 0;
-      for (int layer = 0; layer < c.L && ok; ++layer) {
-        for (int ph = PH_NORM1; ph <= PH_DOWN && ok; ++ph) {
-          run_phase<WT>(c, ph, layer, smem, tc);
-          ok = grid_barrier(c, gen);
-          if (timed) { const uint64_t t = global_timer_ns(); c.ss->cur_phase_ns[ph] += t - t_prev; t_prev = t; }
-        }
-      }
-      for (int ph = PH_FNORM; ph <= PH_SAMPLE && ok; ++ph) {
-        run_phase<WT>(c, ph, 0, smem, tc);
-        ok = grid_barrier(c, gen);
-        if (timed) { const uint64_t t = global_timer_ns(); c.ss->cur_phase_ns[ph] += t - t_prev; t_prev = t; }
-      }
-      if (!ok) break;
-    } else if (!grid_barrier(c, gen)) break;
-  }
-  tc_fini(c, tc);
-  if (blockIdx.x == 0 && threadIdx.x == 0) {
-    const int aborted = *(volatile int*)&c.ss->abort_flag;
-    __threadfence_system();
-    c.mbox->loop_state = aborted ? (uint32_t)BLINK_LOOP_EXIT_ERROR : (uint32_t)c.ss->exit_reason;
-    __threadfence_system();
-  }
-}
 
 // ---- stepped mode ----------------------------------------------------------------------
 __global__ void __launch_bounds__(CTRL_THREADS, 1) blink_control_kernel(const __grid_constant__ DevCtx c, int post_only) {
@@ -140,16 +37,6 @@ __global__ void __launch_bounds__(CTRL_THREADS, 1) blink_control_kernel(const __
   }
   long long li = 0;
   control_phase(c, li);
-}
-
-template <typename WT>
-__global__ void __launch_bounds__(FWD_THREADS, 1) blink_phase_kernel(const __grid_constant__ DevCtx c, int phase, int layer) {
-  extern __shared__ __align__(1024) float smem[];
-  if (c.ss->cmd != CMD_RUN) return;
-  TcState tc;
-  tc_init(c, smem, tc);
-  run_phase<WT>(c, phase, layer, smem, tc);
-  tc_fini(c, tc);
 }
 
 // Sampler alone over caller-provided logits (one CTA per row).
@@ -254,6 +141,7 @@ struct blink_ctx {
   size_t smem_bytes = 0;
   int grid = 1;
   TcHost tc_host;
+  KernelSet ks{nullptr, nullptr};
   bool manual = false;
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
 };
@@ -303,6 +191,10 @@ size_t phase_smem_bytes(const blink_ctx* x) {
   size_t s = sizeof(float) * (size_t)SAMPLE_SMEM_FLOATS;
   size_t m = a > s ? a : s;
   if (x->dc.gemm_tc && tc_smem_bytes() > m) m = tc_smem_bytes();
+  if (x->dc.dtype == BLINK_DTYPE_BF16) {
+    const size_t ab = x->dc.hd == 64 ? (size_t)att_smem_bytes<64>() : (size_t)att_smem_bytes<128>();
+    if (ab > m) m = ab;
+  }
   return m;
 }
 
@@ -311,8 +203,7 @@ int launch_loop(blink_ctx* x) {
   x->mbox->loop_state = BLINK_LOOP_RUNNING;
   std::atomic_thread_fence(std::memory_order_seq_cst);
   void* args[] = {(void*)&x->dc};
-  const void* fn = x->dc.dtype == BLINK_DTYPE_BF16 ? (const void*)blink_loop_kernel<__nv_bfloat16>
-                                                    : (const void*)blink_loop_kernel<float>;
+  const void* fn = x->ks.loop;
   cudaError_t e = cudaLaunchCooperativeKernel(fn, dim3(x->grid), dim3(FWD_THREADS), args, x->smem_bytes, x->stream);
   if (e != cudaSuccess) {
     x->mbox->loop_state = BLINK_LOOP_EXIT_ERROR;
@@ -336,20 +227,19 @@ int pump(blink_ctx* x) {
   return launch_loop(x);
 }
 
-template <typename WT>
 void launch_phase(blink_ctx* x, int phase, int layer) {
-  blink_phase_kernel<WT><<<x->grid, FWD_THREADS, x->smem_bytes, x->stream>>>(x->dc, phase, layer);
+  void* args[] = {(void*)&x->dc, (void*)&phase, (void*)&layer};
+  cudaLaunchKernel(x->ks.phase, dim3(x->grid), dim3(FWD_THREADS), args, x->smem_bytes, x->stream);
   x->launches += 1;
 }
 
-template <typename WT>
 int step_once(blink_ctx* x) {
   blink_control_kernel<<<1, CTRL_THREADS, 0, x->stream>>>(x->dc, 0);
   x->launches += 1;
   if (!x->dc.control_only) {
     for (int l = 0; l < x->dc.L; ++l)
-      for (int ph = PH_NORM1; ph <= PH_DOWN; ++ph) launch_phase<WT>(x, ph, l);
-    for (int ph = PH_FNORM; ph <= PH_SAMPLE; ++ph) launch_phase<WT>(x, ph, 0);
+      for (int ph = PH_NORM1; ph <= PH_DOWN; ++ph) launch_phase(x, ph, l);
+    for (int ph = PH_FNORM; ph <= PH_SAMPLE; ++ph) launch_phase(x, ph, 0);
   }
   return cudaGetLastError() == cudaSuccess ? BLINK_OK : BLINK_ECUDA;
 }
@@ -582,6 +472,16 @@ int blink_create(const blink_model_cfg* model, const blink_sched_cfg* sched, con
     TRY(dev_alloc(x, &c.h, TM * c.d));
     TRY(dev_alloc(x, &p, TM * c.d * esz)); c.xn = p;
     TRY(dev_alloc(x, &c.qkv, TM * c.qkv_dim));
+    if (c.dtype == BLINK_DTYPE_BF16) {
+      TRY(dev_alloc(x, &p, TM * c.q_dim * esz)); c.qb = p;
+      c.n_warps_grid = x->n_sms * (FWD_THREADS / 32);
+      c.att_sub_max = 4ll * c.n_warps_grid + (long long)MB * c.Hkv * c.max_blocks_seq / 64 + 8;
+      TRY(dev_alloc(x, &c.dec_row, MB)); TRY(dev_alloc(x, &c.dec_bslot, MB)); TRY(dev_alloc(x, &c.dec_nctx, MB));
+      TRY(dev_alloc(x, &c.dec_kbpre, MB + 1));
+      TRY(dev_alloc(x, &c.pf_item, TM / 16 + MB + 1)); TRY(dev_alloc(x, &c.pf_qb, TM / 16 + MB + 1));
+      TRY(dev_alloc(x, &c.att_ctr, (size_t)c.L)); TRY(dev_alloc(x, &c.att_cnt, MB * c.Hkv));
+      TRY(dev_alloc(x, &c.att_part, (size_t)(2 * c.att_sub_max) * c.n_rep * (c.hd + 2), false));
+    }
     TRY(dev_alloc(x, &p, TM * c.q_dim * esz)); c.attn = p;
     TRY(dev_alloc(x, &c.gu, TM * 2 * c.F));
     TRY(dev_alloc(x, &p, TM * c.F * esz)); c.act = p;
@@ -639,10 +539,11 @@ int blink_create(const blink_model_cfg* model, const blink_sched_cfg* sched, con
 
   x->smem_bytes = phase_smem_bytes(x);
   x->grid = c.control_only ? 1 : x->n_sms;
-  const void* loop_fn = c.dtype == BLINK_DTYPE_BF16 ? (const void*)blink_loop_kernel<__nv_bfloat16>
-                                                     : (const void*)blink_loop_kernel<float>;
-  const void* ph_fn = c.dtype == BLINK_DTYPE_BF16 ? (const void*)blink_phase_kernel<__nv_bfloat16>
-                                                   : (const void*)blink_phase_kernel<float>;
+  x->ks = c.dtype == BLINK_DTYPE_BF16 ? (c.hd == 64 ? kernels_bf16_hd64(c.n_rep) : kernels_bf16_hd128(c.n_rep))
+                                      : (c.hd == 64 ? kernels_fp32_hd64(c.n_rep) : kernels_fp32_hd128(c.n_rep));
+  const void* loop_fn = x->ks.loop;
+  const void* ph_fn = x->ks.phase;
+  if (!loop_fn || !ph_fn) return fail(BLINK_EINVAL);
   if (cudaFuncSetAttribute(loop_fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)x->smem_bytes) != cudaSuccess ||
       cudaFuncSetAttribute(ph_fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)x->smem_bytes) != cudaSuccess)
     return fail(BLINK_ECUDA);
@@ -763,7 +664,7 @@ int blink_step(blink_ctx* x, int n_iterations) {
   if (!x->dc.stepped) return BLINK_EINVAL;
   std::lock_guard<std::mutex> g(x->mu);
   for (int i = 0; i < n_iterations; ++i) {
-    const int rc = x->dc.dtype == BLINK_DTYPE_BF16 ? step_once<__nv_bfloat16>(x) : step_once<float>(x);
+    const int rc = step_once(x);
     if (rc != BLINK_OK) return rc;
   }
   blink_control_kernel<<<1, CTRL_THREADS, 0, x->stream>>>(x->dc, 1);

@@ -122,7 +122,7 @@ __device__ __forceinline__ int32_t fake_token(unsigned long long ticket, int gen
 __device__ __forceinline__ bool trace_on(const DevCtx& c) { return c.trace_cap > 0 && !c.ss->trace_off; }
 
 // ---- step 5 of the iteration: publish, retire, free -------------------------------------
-__device__ void post_step(const DevCtx& c) {
+static __device__ void post_step(const DevCtx& c) {
   SchedState* ss = c.ss;
   const int tid = threadIdx.x;
   const int n_items = ss->cur_items;
@@ -226,7 +226,7 @@ __device__ void post_step(const DevCtx& c) {
 }
 
 // ---- stand-in for the frontend's RDMA write: pinned submit area -> HBM ring --------------
-__device__ void ingress(const DevCtx& c, unsigned long long tail) {
+static __device__ void ingress(const DevCtx& c, unsigned long long tail) {
   SchedState* ss = c.ss;
   const int tid = threadIdx.x;
   for (unsigned long long e = ss->seen; e < tail; ++e) {
@@ -273,7 +273,7 @@ __device__ void ingress(const DevCtx& c, unsigned long long tail) {
 }
 
 // ---- parallel slot scan + CAS claim (Section 4.2 "Parallel slot scanning") ----------------
-__device__ void scan_and_claim(const DevCtx& c) {
+static __device__ void scan_and_claim(const DevCtx& c) {
   const int per = (c.n_slots + CTRL_THREADS - 1) / CTRL_THREADS;
   const int lo = threadIdx.x * per;
   const int hi = min(c.n_slots, lo + per);
@@ -291,7 +291,7 @@ __device__ void scan_and_claim(const DevCtx& c) {
 
 // ---- steps 1-3: admit, compose, allocate, build metadata ----------------------------------
 // Returns the number of rows T of the composed step (0 = nothing to run).
-__device__ int schedule_step(const DevCtx& c, unsigned long long visible) {
+static __device__ int schedule_step(const DevCtx& c, unsigned long long visible) {
   SchedState* ss = c.ss;
   const int tid = threadIdx.x;
   const int MB = c.MB;
@@ -410,6 +410,16 @@ __device__ int schedule_step(const DevCtx& c, unsigned long long visible) {
   // blocks that post_step may free at most (for the trace space check)
   int tot_may_free;
   block_exscan(sample ? have + want : 0, &tot_may_free);
+  // attention work lists: single-row requests stream their KV blocks, multi-row requests are
+  // cut into blocks of 128 / n_rep query rows
+  const int q_rows = 128 / c.n_rep;
+  const int is_dec = f && take == 1;
+  const int nkb_att = is_dec ? (new_len + c.bs - 1) / c.bs : 0;
+  const int n_qb = (f && take > 1) ? (take + q_rows - 1) / q_rows : 0;
+  int n_dec_att, tot_kb, n_pf;
+  const int dec_idx = block_exscan(is_dec, &n_dec_att);
+  const int kb_pre = block_exscan(nkb_att, &tot_kb);
+  const int pf_off = block_exscan(n_qb, &n_pf);
 
   if (T == 0) return 0;  // uniform: every thread sees the same T
 
@@ -457,6 +467,18 @@ __device__ int schedule_step(const DevCtx& c, unsigned long long visible) {
       c.row_tok[row] = qstart + take - 1;
       c.row_item[row] = item;
     }
+    if (c.dec_row != nullptr) {
+      if (is_dec) {
+        c.dec_row[dec_idx] = qstart;
+        c.dec_bslot[dec_idx] = tid;
+        c.dec_nctx[dec_idx] = new_len;
+        c.dec_kbpre[dec_idx] = kb_pre;
+      }
+      for (int q = 0; q < n_qb; ++q) {   // heaviest (last) row block first
+        c.pf_item[pf_off + q] = item;
+        c.pf_qb[pf_off + q] = n_qb - 1 - q;
+      }
+    }
     if (tr) {
       rec_sched[5 * item] = tid;
       rec_sched[5 * item + 1] = (int32_t)ticket;
@@ -476,6 +498,8 @@ __device__ int schedule_step(const DevCtx& c, unsigned long long visible) {
   __syncthreads();
 
   // per-row metadata: token id, position, owning item, KV slot
+  if (c.att_ctr != nullptr)
+    for (int i = tid; i < c.L; i += CTRL_THREADS) c.att_ctr[i] = 0;
   for (int r = tid; r < T; r += CTRL_THREADS) {
     int lo = 0, hi = n_items;  // last item with qstart <= r
     while (hi - lo > 1) {
@@ -504,6 +528,18 @@ __device__ int schedule_step(const DevCtx& c, unsigned long long visible) {
     ss->cur_kv = (long long)s_kv;
     ss->cur_t_begin = t_begin;
     ss->pending_post = 1;
+    if (c.dec_row != nullptr) {
+      const long long TT = (long long)tot_kb * c.Hkv;
+      long long S = (TT + 4ll * c.n_warps_grid - 1) / (4ll * c.n_warps_grid);
+      if (S < 1) S = 1;
+      if (S > 64) S = 64;
+      while ((TT + S - 1) / S > c.att_sub_max) S *= 2;   // cannot happen with the sizes set at create
+      c.dec_kbpre[n_dec_att] = tot_kb;
+      ss->cur_ndec = n_dec_att;
+      ss->cur_TT = (int)TT;
+      ss->cur_S = (int)S;
+      ss->cur_npf = n_pf;
+    }
     if (tr) {
       rec[0] = TRACE_MAGIC;
       rec[1] = (int32_t)ss->iter;
@@ -526,7 +562,7 @@ __device__ int schedule_step(const DevCtx& c, unsigned long long visible) {
 // One pass of the control plane.  `launch_iters` counts the iterations this kernel
 // launch has started.  Sets ss->cmd to CMD_RUN (a step was composed), CMD_EXIT
 // (leave the GPU; reason in ss->exit_reason) or CMD_NONE (stepped mode, idle).
-__device__ void control_phase(const DevCtx& c, long long& launch_iters) {
+static __device__ void control_phase(const DevCtx& c, long long& launch_iters) {
   SchedState* ss = c.ss;
   const int tid = threadIdx.x;
   __shared__ int s_cmd;

@@ -93,6 +93,10 @@ struct SchedState {
   int free_top;                     // entries in the free stack
   int reserved;                     // blocks promised to admitted requests
   int cur_T, cur_items, cur_rows, cur_decode;
+  int cur_ndec;   // attention: requests with one query row in this step
+  int cur_TT;     // attention: (row, kv head, KV block) tiles of those rows
+  int cur_S;      // attention: tiles per sub-range of the flat tile sequence
+  int cur_npf;    // attention: (request, query-row block) units of the multi-row requests
   long long cur_ctx;
   long long cur_kv;
   int cmd;
@@ -131,6 +135,7 @@ struct DevCtx {
   // scheduler shape
   int MB, chunk, n_slots, max_prompt, max_new, Tmax, bs, n_blocks, max_blocks_seq, max_pos;
   int control_only, start_paused, stepped, gemm_tc;
+  int n_warps_grid;  // warps of the whole grid (attention work split)
   long long iteration_budget;
   unsigned long long idle_exit_cycles, barrier_timeout_cycles;
   // ring in HBM
@@ -162,10 +167,18 @@ struct DevCtx {
   int32_t *it_bslot, *it_start, *it_ntok, *it_qstart, *it_row;  // [MB] per item
   int32_t *tok_id, *tok_pos, *tok_item, *tok_slotmap;           // [Tmax] per row
   int32_t *row_tok, *row_item, *row_sampled;                    // [MB] per sample row
+  // attention work lists of the step (bf16 path)
+  int32_t *dec_row, *dec_bslot, *dec_nctx, *dec_kbpre;          // [MB] (+1 for the prefix) single-row requests
+  int32_t *pf_item, *pf_qb;                                     // [Tmax/16 + MB + 1] multi-row tile units
+  int32_t* att_ctr;      // [L] sub-range counters, zeroed every iteration
+  int32_t* att_cnt;      // [MB * Hkv] parts delivered per (row, kv head) unit; self-resetting
+  float* att_part;       // partial (acc, m, l) records, two per sub-range
+  long long att_sub_max; // sub-ranges the record buffer can hold
   // activations
   float* h;       // [Tmax][d]
   void* xn;       // [Tmax][d]      operand type
   float* qkv;     // [Tmax][qkv_dim]
+  void* qb;       // [Tmax][q_dim]  bf16 path: q after RoPE, as the attention operand
   void* attn;     // [Tmax][q_dim]  operand type
   float* gu;      // [Tmax][2F]
   void* act;      // [Tmax][F]      operand type

@@ -65,7 +65,7 @@ __device__ __forceinline__ void zero_floats(float* p, long long n_floats) {
 // ---- RMSNorm of the residual rows into the operand buffer; layer 0 gathers the
 // embedding first.  n = x / sqrt(mean(x^2) + eps) * g
 template <typename WT>
-__device__ void phase_norm(const DevCtx& c, int layer, int which /*0: norm1, 1: norm2*/) {
+static __device__ void phase_norm(const DevCtx& c, int layer, int which /*0: norm1, 1: norm2*/) {
   __shared__ float s_red[FWD_THREADS / 32];
   const int T = c.ss->cur_T;
   const float* g = wptr_f(c, which == 0 ? 6 : 7) + (size_t)layer * c.d;
@@ -91,7 +91,7 @@ __device__ void phase_norm(const DevCtx& c, int layer, int which /*0: norm1, 1: 
 
 // Final norm of the sampled rows only (the LM head runs on those rows).
 template <typename WT>
-__device__ void phase_final_norm(const DevCtx& c) {
+static __device__ void phase_final_norm(const DevCtx& c) {
   __shared__ float s_red[FWD_THREADS / 32];
   const int R = c.ss->cur_rows;
   const float* g = wptr_f(c, 8);
@@ -120,7 +120,7 @@ struct GemmArgs {
 };
 
 template <typename WT>
-__device__ void phase_gemm_simt(const GemmArgs& a) {
+static __device__ void phase_gemm_simt(const GemmArgs& a) {
   constexpr int BM = 64, BN = 64, BK = 16;
   __shared__ float xs[BK][BM + 4];
   __shared__ float ws[BK][BN + 4];
@@ -187,7 +187,7 @@ __device__ __forceinline__ WT* kv_tile(const DevCtx& c, int layer, int kv, int b
 }
 
 template <typename WT>
-__device__ void phase_rope_kv(const DevCtx& c, int layer) {
+static __device__ void phase_rope_kv(const DevCtx& c, int layer) {
   const int T = c.ss->cur_T;
   const int half = c.hd / 2;
   const int heads = c.Hq + 2 * c.Hkv;
@@ -204,8 +204,14 @@ __device__ void phase_rope_kv(const DevCtx& c, int layer) {
       const float cs = c.rope_cos[(size_t)pos * half + i], sn = c.rope_sin[(size_t)pos * half + i];
       const float y1 = x1 * cs - x2 * sn, y2 = x2 * cs + x1 * sn;
       if (hh < c.Hq) {
-        row[i] = y1;
-        row[i + half] = y2;
+        if constexpr (sizeof(WT) == 2) {   // 16-bit path: q is an operand of the attention contraction
+          WT* qd = reinterpret_cast<WT*>(c.qb) + (size_t)t * c.q_dim + (size_t)hh * c.hd;
+          qd[i] = OpType<WT>::from_f(y1);
+          qd[i + half] = OpType<WT>::from_f(y2);
+        } else {
+          row[i] = y1;
+          row[i + half] = y2;
+        }
       } else {
         const int sm = c.tok_slotmap[t];
         WT* dst = kv_tile<WT>(c, layer, 0, sm / c.bs, hh - c.Hq) + (size_t)(sm % c.bs) * c.hd;
@@ -227,7 +233,7 @@ __device__ void phase_rope_kv(const DevCtx& c, int layer) {
 // vector load per lane covers whole (block, head) tiles with coalesced 512-byte rows.
 // Online softmax per warp, merged across warps in shared memory at the end.
 template <typename WT, int HD, int NREP>
-__device__ void phase_attention(const DevCtx& c, int layer, float* smem) {
+static __device__ void phase_attention(const DevCtx& c, int layer, float* smem) {
   constexpr int CE = 16 / (int)sizeof(WT);  // elements per 16-byte chunk
   constexpr int LPK = HD / CE;              // lanes per key
   constexpr int KPP = 32 / LPK;             // keys per pass
@@ -359,7 +365,7 @@ constexpr int ATTN_SMEM_FLOATS(int HD, int NREP) { return NREP * HD + 2 * 8 * NR
 
 // ---- SwiGLU gate: act = silu(gate) * up ------------------------------------------------
 template <typename WT>
-__device__ void phase_silu_mul(const DevCtx& c) {
+static __device__ void phase_silu_mul(const DevCtx& c) {
   const int T = c.ss->cur_T;
   WT* out = reinterpret_cast<WT*>(c.act);
   const long long total = (long long)T * c.F;
@@ -397,7 +403,7 @@ __device__ __forceinline__ uint32_t float_key(float f) {
 // (IEEE fp32 divide); the k largest by (z desc, index asc) are found with a radix select
 // on the float keys; weights exp(z - z0) and the inverse-CDF walk run in fp64.
 // The result is returned by thread 0 (other threads return -1).
-__device__ int sample_row(const float* lg, int V, int top_k, float temp, unsigned long long ticket, int gen_index,
+static __device__ int sample_row(const float* lg, int V, int top_k, float temp, unsigned long long ticket, int gen_index,
                           unsigned long long seed, float* smem) {
   constexpr int CAND_MAX = 1024;
   const int tid = threadIdx.x;
@@ -514,7 +520,7 @@ __device__ int sample_row(const float* lg, int V, int top_k, float temp, unsigne
   return result;
 }
 
-__device__ void phase_sample(const DevCtx& c, float* smem) {
+static __device__ void phase_sample(const DevCtx& c, float* smem) {
   const int R = c.ss->cur_rows;
   const int V = c.V;
   const int tid = threadIdx.x;

@@ -193,7 +193,7 @@ struct TcMaps {
 };
 
 // ---- the GEMM phase -----------------------------------------------------------------------------
-__device__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int which, int layer, float* smem_f, TcState& tc) {
+static __device__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int which, int layer, float* smem_f, TcState& tc) {
   const int T = a.M, N = a.N, K = a.K;
   if (T <= 0) return;  // uniform over the grid
   const TcMaps* maps = reinterpret_cast<const TcMaps*>(c.tc_maps);

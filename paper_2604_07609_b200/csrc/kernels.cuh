@@ -1,0 +1,132 @@
+// The kernels of the serving loop, instantiated per (operand type, head_dim, query heads per
+// kv head) so that each instance carries exactly one attention variant: the persistent
+// cooperative loop and the one-phase kernel of stepped mode.
+#pragma once
+#include <cuda_runtime.h>
+
+#include "../../include/blink.h"
+#include "attention.cuh"
+#include "control.cuh"
+#include "dev_ctx.cuh"
+#include "forward.cuh"
+#include "gemm_tc.cuh"
+#include "kernel_set.h"
+
+namespace blink {
+
+template <typename WT>
+__device__ __forceinline__ void gemm_dispatch(const DevCtx& c, const GemmArgs& a, int which, int layer, float* smem,
+                                              TcState& tc) {
+  if (c.gemm_tc) phase_gemm_tc(c, a, which, layer, smem, tc);
+  else phase_gemm_simt<WT>(a);
+}
+
+template <typename WT, int HD, int NREP>
+__device__ __forceinline__ void run_phase(const DevCtx& c, int phase, int layer, float* smem, TcState& tc, AttState& as) {
+  const int T = c.ss->cur_T;
+  const size_t esz = sizeof(WT);
+  switch (phase) {
+    case PH_NORM1: phase_norm<WT>(c, layer, 0); break;
+    case PH_QKV: {
+      GemmArgs a{c.xn, c.w_base + c.w_off[1] + (size_t)layer * c.qkv_dim * c.d * esz, c.qkv, T, c.qkv_dim, c.d,
+                 c.qkv_dim, 0};
+      gemm_dispatch<WT>(c, a, GEMM_QKV, layer, smem, tc);
+    } break;
+    case PH_ROPE: phase_rope_kv<WT>(c, layer); break;
+    case PH_ATTN:
+      if constexpr (sizeof(WT) == 2) phase_attention_bf16<HD, NREP>(c, layer, smem, as);
+      else phase_attention<WT, HD, NREP>(c, layer, smem);
+      break;
+    case PH_O: {
+      GemmArgs a{c.attn, c.w_base + c.w_off[2] + (size_t)layer * c.d * c.q_dim * esz, c.h, T, c.d, c.q_dim, c.d, 1};
+      gemm_dispatch<WT>(c, a, GEMM_O, layer, smem, tc);
+    } break;
+    case PH_NORM2: phase_norm<WT>(c, layer, 1); break;
+    case PH_GU: {
+      GemmArgs a{c.xn, c.w_base + c.w_off[3] + (size_t)layer * 2 * c.F * c.d * esz, c.gu, T, 2 * c.F, c.d, 2 * c.F, 0};
+      gemm_dispatch<WT>(c, a, GEMM_GU, layer, smem, tc);
+    } break;
+    case PH_SILU: phase_silu_mul<WT>(c); break;
+    case PH_DOWN: {
+      GemmArgs a{c.act, c.w_base + c.w_off[4] + (size_t)layer * c.d * c.F * esz, c.h, T, c.d, c.F, c.d, 1};
+      gemm_dispatch<WT>(c, a, GEMM_DOWN, layer, smem, tc);
+    } break;
+    case PH_FNORM: phase_final_norm<WT>(c); break;
+    case PH_LMHEAD: {
+      GemmArgs a{c.xs, c.w_base + c.w_off[9], c.logits, c.ss->cur_rows, c.V, c.d, c.V, 0};
+      gemm_dispatch<WT>(c, a, GEMM_LMHEAD, 0, smem, tc);
+    } break;
+    case PH_SAMPLE: phase_sample(c, smem); break;
+    default: break;
+  }
+}
+
+// ---- persistent loop -----------------------------------------------------------------
+template <typename WT, int HD, int NREP>
+__global__ void __launch_bounds__(FWD_THREADS, 1) blink_loop_kernel(const __grid_constant__ DevCtx c) {
+  extern __shared__ __align__(1024) float smem[];
+  unsigned int gen = 0;
+  if (threadIdx.x == 0) gen = ld_acquire_gpu_u32(&c.ss->bar_gen);
+  long long launch_iters = 0;
+  TcState tc;
+  tc_init(c, smem, tc);
+  AttState as;
+  att_init(c, as);
+  while (true) {
+    if (blockIdx.x == 0) control_phase(c, launch_iters);
+    if (!grid_barrier(c, gen)) break;
+    if (*(volatile int*)&c.ss->cmd != CMD_RUN) break;
+    if (!c.control_only) {
+      bool ok = true;
+      // CTA 0 keeps a per-phase-kind device time of the open iteration (a phase's time includes
+      // the barrier that closes it); recorded only when per-iteration statistics are kept
+      const bool timed = c.stats_cap > 0 && blockIdx.x == 0 && threadIdx.x == 0;
+      uint64_t t_prev = timed ? global_timer_ns() : 0;
+      for (int layer = 0; layer < c.L && ok; ++layer) {
+        for (int ph = PH_NORM1; ph <= PH_DOWN && ok; ++ph) {
+          run_phase<WT, HD, NREP>(c, ph, layer, smem, tc, as);
+          ok = grid_barrier(c, gen);
+          if (timed) { const uint64_t t = global_timer_ns(); c.ss->cur_phase_ns[ph] += t - t_prev; t_prev = t; }
+        }
+      }
+      for (int ph = PH_FNORM; ph <= PH_SAMPLE && ok; ++ph) {
+        run_phase<WT, HD, NREP>(c, ph, 0, smem, tc, as);
+        ok = grid_barrier(c, gen);
+        if (timed) { const uint64_t t = global_timer_ns(); c.ss->cur_phase_ns[ph] += t - t_prev; t_prev = t; }
+      }
+      if (!ok) break;
+    } else if (!grid_barrier(c, gen)) break;
+  }
+  tc_fini(c, tc);
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    const int aborted = *(volatile int*)&c.ss->abort_flag;
+    __threadfence_system();
+    c.mbox->loop_state = aborted ? (uint32_t)BLINK_LOOP_EXIT_ERROR : (uint32_t)c.ss->exit_reason;
+    __threadfence_system();
+  }
+}
+
+template <typename WT, int HD, int NREP>
+__global__ void __launch_bounds__(FWD_THREADS, 1) blink_phase_kernel(const __grid_constant__ DevCtx c, int phase, int layer) {
+  extern __shared__ __align__(1024) float smem[];
+  if (c.ss->cmd != CMD_RUN) return;
+  TcState tc;
+  tc_init(c, smem, tc);
+  AttState as;
+  att_init(c, as);
+  run_phase<WT, HD, NREP>(c, phase, layer, smem, tc, as);
+  tc_fini(c, tc);
+}
+
+template <typename WT, int HD>
+inline KernelSet kernel_set_for(int n_rep) {
+  switch (n_rep) {
+    case 1: return {(const void*)blink_loop_kernel<WT, HD, 1>, (const void*)blink_phase_kernel<WT, HD, 1>};
+    case 2: return {(const void*)blink_loop_kernel<WT, HD, 2>, (const void*)blink_phase_kernel<WT, HD, 2>};
+    case 4: return {(const void*)blink_loop_kernel<WT, HD, 4>, (const void*)blink_phase_kernel<WT, HD, 4>};
+    case 8: return {(const void*)blink_loop_kernel<WT, HD, 8>, (const void*)blink_phase_kernel<WT, HD, 8>};
+    default: return {nullptr, nullptr};
+  }
+}
+
+}  // namespace blink
