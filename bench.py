@@ -209,10 +209,11 @@ def percentiles(x):
     return dict(p50=float(np.percentile(x, 50)), p99=float(np.percentile(x, 99)), mean=float(np.mean(x)))
 
 
-def realtime_run(B, m, sched, wbuf, kv, reqs, time_limit_s, use_arrivals=True):
+def realtime_run(B, m, sched, wbuf, kv, reqs, time_limit_s, use_arrivals=True, weights_layout=0):
     """Persistent loop, requests submitted at their arrival times from host buffers, tokens
     read back with blink_poll.  Returns throughput and latency figures."""
-    eng = B.Blink(m, sched, wbuf, kv, exec_mode=B.EXEC_PERSISTENT, stats_iters=1 << 17, idle_exit_us=2_000_000)
+    eng = B.Blink(m, sched, wbuf, kv, exec_mode=B.EXEC_PERSISTENT, stats_iters=1 << 17, idle_exit_us=2_000_000,
+                  weights_layout=weights_layout)
     try:
         off = eng.blink_get_stats().device_clock_offset_ns
         n_expected = 0
@@ -274,6 +275,8 @@ def main():
     ap.add_argument("--config", type=int, default=3, help="BASELINE configuration (1..4)")
     ap.add_argument("--ramp", type=int, default=-1, help="untimed iterations that bring the batch to steady state")
     ap.add_argument("--gemm", default="auto", choices=["auto", "simt", "tc"])
+    ap.add_argument("--weights", default="streaming", choices=["streaming", "row-major"],
+                    help="storage of the GEMM matrices: tile-contiguous streaming layout or plain row-major")
     ap.add_argument("--rate", type=float, default=16.0, help="offered load of the real-time run (req/s)")
     ap.add_argument("--e2e-seconds", type=float, default=15.0)
     ap.add_argument("--latency-seconds", type=float, default=20.0)
@@ -356,6 +359,10 @@ def main():
             cpu_baseline = dict(value=None, unit="output tok/s", cores=os.cpu_count(), kind="oracle",
                                 sample=f"failed: {e!r}")
 
+    wl = B.WEIGHTS_ROW_MAJOR
+    if args.weights == "streaming" and m.dtype == "bf16" and args.gemm != "simt":
+        B.blink_convert_weights(m, wbuf, B.WEIGHTS_ROW_MAJOR, B.WEIGHTS_STREAMING)   # set-up, once, in place
+        wl = B.WEIGHTS_STREAMING
     # ---- KV pool: a fraction of what is free after the weights ---------------------------
     free, total = torch.cuda.mem_get_info(dev)
     lib_reserve = 6 << 30      # ring, arenas, activations and logits the library allocates itself
@@ -382,7 +389,8 @@ def main():
     if args.exec == "stepped":
         # profiling aid: the same device code, one host launch per phase, so that a profiler sees
         # the phases as separate kernels (1 control launch + 9 per layer + 3 per iteration)
-        eng = B.Blink(m, sched, wbuf, kv, exec_mode=B.EXEC_STEPPED, gemm_impl=gemm_impl, stats_iters=ramp + W + K + 64)
+        eng = B.Blink(m, sched, wbuf, kv, exec_mode=B.EXEC_STEPPED, gemm_impl=gemm_impl, stats_iters=ramp + W + K + 64,
+                      weights_layout=wl)
         try:
             for r in reqs:
                 eng.submit_request(r)
@@ -403,7 +411,7 @@ def main():
 
     # ---- closed-loop saturation run: ramp, W warm-up steps, then exactly K timed steps --------
     eng = B.Blink(m, sched, wbuf, kv, exec_mode=B.EXEC_MANUAL, gemm_impl=gemm_impl, stats_iters=ramp + W + K + 64,
-                  idle_exit_us=200_000)
+                  idle_exit_us=200_000, weights_layout=wl)
     try:
         for r in reqs:
             eng.submit_request(r)
@@ -475,7 +483,8 @@ def main():
                             l2="per-step inputs (weights + KV) exceed L2 many times over; no flush needed",
                             rows_per_step=float(its["n_tokens"].mean()),
                             decode_rows_per_step=float(its["n_decode"].mean()),
-                            parallelism="replicas" if world > 1 else "1 GPU", gemm=args.gemm),
+                            parallelism="replicas" if world > 1 else "1 GPU", gemm=args.gemm,
+                            weights_layout="streaming" if wl else "row-major"),
                 gpu_launches=1, clocks=clk, roofline=roof,
                 step_ms_device=dict(p50=float(np.median(step_dev_ms)), max=float(step_dev_ms.max())),
                 phase_ms_per_step={n: float(its["phase_ns"][:, i].mean() / 1e6) for i, n in enumerate(B.PHASE_NAMES)},
@@ -485,7 +494,7 @@ def main():
 
     # ---- end to end through the public API with host buffers ------------------------------
     if not args.skip_e2e:
-        r = realtime_run(B, m, sched, wbuf, kv, reqs, args.e2e_seconds, use_arrivals=False)
+        r = realtime_run(B, m, sched, wbuf, kv, reqs, args.e2e_seconds, use_arrivals=False, weights_layout=wl)
         e_val = torch.tensor([r["tok_s"]], dtype=torch.float64, device=dev)
         if world > 1:
             dist.all_reduce(e_val, op=dist.ReduceOp.SUM)
@@ -502,7 +511,7 @@ def main():
             stress.start()
         try:
             lreqs = [q for q in reqs if q.arrival_s <= args.latency_seconds]
-            r = realtime_run(B, m, sched, wbuf, kv, lreqs, args.latency_seconds * 3, use_arrivals=True)
+            r = realtime_run(B, m, sched, wbuf, kv, lreqs, args.latency_seconds * 3, use_arrivals=True, weights_layout=wl)
         finally:
             if stress:
                 stress.stop()

@@ -52,6 +52,20 @@ enum {
 
 enum { BLINK_DTYPE_BF16 = 0, BLINK_DTYPE_FP32 = 1 };
 
+/* Storage of the GEMM matrices (tensor ids 1, 2, 3, 4, 9) inside the flat weight buffer.  Tensor
+ * offsets and sizes are the same in both layouts; embedding, router and norm tensors are always
+ * row-major.
+ *   ROW_MAJOR : [out][in], the documented exchange layout.
+ *   STREAMING : bf16 only.  Each matrix is cut into panels of 128 output rows; a panel keeps its
+ *     byte range but is stored as K/64 consecutive tiles of 128 rows x 64 columns (16 KiB), tile
+ *     kb holding columns [64 kb, 64 kb + 64).  Inside a tile row r is at byte r * 128 and its
+ *     16-byte chunk c (columns 8 c .. 8 c + 7) sits at chunk position c ^ (r % 8): the operand
+ *     image the tensor cores read from shared memory, so a weight tile reaches the SM as one
+ *     contiguous 16 KiB copy and every SM streams long sequential runs of HBM.  Requires every
+ *     matrix to have a multiple of 128 rows per layer and a multiple of 64 columns.
+ * blink_convert_weights switches a buffer between the two, in place. */
+enum { BLINK_WEIGHTS_ROW_MAJOR = 0, BLINK_WEIGHTS_STREAMING = 1 };
+
 /* how the iteration is executed */
 enum {
   BLINK_EXEC_PERSISTENT = 0, /* one cooperative kernel loops on the device (product mode)           */
@@ -88,6 +102,7 @@ typedef struct blink_model_cfg {
   float rope_theta;
   float rms_eps;
   int32_t dtype;         /* BLINK_DTYPE_*: storage type of matrices, KV pool and GEMM operands */
+  int32_t weights_layout;/* BLINK_WEIGHTS_*: how the five GEMM matrices are stored inside `weights` */
   const void* weights;   /* DEVICE, caller-owned, layout: see blink_weight_offset; may be NULL when control_only */
   uint64_t weights_bytes;
 } blink_model_cfg;
@@ -191,6 +206,14 @@ uint64_t blink_weights_bytes(const blink_model_cfg* cfg);
  * 8 normf[d] fp32, 9 lm_head[V,d].  All matrices row-major [out, in]; every tensor
  * starts on a 256-byte boundary. */
 uint64_t blink_weight_offset(const blink_model_cfg* cfg, int tensor_id);
+
+/* Convert the GEMM matrices of `weights` (DEVICE, caller-owned, blink_weights_bytes(cfg) bytes)
+ * in place from cfg->weights_layout to `to_layout`.  Part of set-up (the provisioning plane of
+ * Section 4.1: the host prepares the engine once, then leaves the inference path).  Synchronous;
+ * uses a temporary device scratch of one 128-row panel per SM.  BLINK_EINVAL when the shape does
+ * not admit the streaming layout or the dtype is not bf16; a no-op when the layouts are equal.
+ * No context may be using the buffer meanwhile. */
+int blink_convert_weights(const blink_model_cfg* cfg, void* weights, int to_layout);
 
 /* KV blocks a pool of `bytes` yields for this model shape and block size. */
 int64_t blink_kv_blocks_for_bytes(const blink_model_cfg* cfg, int block_size, uint64_t bytes);

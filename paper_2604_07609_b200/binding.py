@@ -21,6 +21,7 @@ SAMPLE_NOALLOC_MAX_ROWS = 1024
 DTYPE_BF16, DTYPE_FP32 = 0, 1
 EXEC_PERSISTENT, EXEC_STEPPED, EXEC_MANUAL = 0, 1, 2
 GEMM_AUTO, GEMM_SIMT, GEMM_TC = 0, 1, 2
+WEIGHTS_ROW_MAJOR, WEIGHTS_STREAMING = 0, 1
 LOOP_NOT_STARTED, LOOP_RUNNING, LOOP_EXIT_STOP, LOOP_EXIT_BUDGET, LOOP_EXIT_IDLE, LOOP_EXIT_ERROR = range(6)
 TRACE_MAGIC = 0x424C4B31
 TRACE_HDR_WORDS = 12
@@ -30,7 +31,8 @@ class blink_model_cfg(C.Structure):
     _fields_ = [("size", C.c_uint32), ("n_layers", C.c_int32), ("d_model", C.c_int32), ("n_q_heads", C.c_int32),
                 ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32), ("d_ff", C.c_int32), ("vocab", C.c_int32),
                 ("n_experts", C.c_int32), ("top_k_experts", C.c_int32), ("rope_theta", C.c_float),
-                ("rms_eps", C.c_float), ("dtype", C.c_int32), ("weights", C.c_void_p), ("weights_bytes", C.c_uint64)]
+                ("rms_eps", C.c_float), ("dtype", C.c_int32), ("weights_layout", C.c_int32), ("weights", C.c_void_p),
+                ("weights_bytes", C.c_uint64)]
 
 
 class blink_sched_cfg(C.Structure):
@@ -84,7 +86,7 @@ EVENT_DTYPE = np.dtype([("ticket", "<u8"), ("user_tag", "<u8"), ("index", "<i4")
                         ("is_first", "<i4"), ("is_last", "<i4"), ("t_device_ns", "<u8"), ("t_host_ns", "<u8"),
                         ("t_submit_ns", "<u8")])
 
-EXPORTS = ["blink_weights_bytes", "blink_weight_offset", "blink_kv_blocks_for_bytes", "blink_create",
+EXPORTS = ["blink_weights_bytes", "blink_weight_offset", "blink_convert_weights", "blink_kv_blocks_for_bytes", "blink_create",
            "blink_start", "blink_submit", "blink_poll", "blink_step", "blink_run", "blink_stop", "blink_destroy",
            "blink_get_stats", "blink_get_trace", "blink_get_iter_stats", "blink_sample", "blink_sample_noalloc",
            "blink_strerror"]
@@ -106,6 +108,8 @@ def lib():
     L.blink_weights_bytes.argtypes = [P(blink_model_cfg)]
     L.blink_weight_offset.restype = C.c_uint64
     L.blink_weight_offset.argtypes = [P(blink_model_cfg), C.c_int]
+    L.blink_convert_weights.restype = C.c_int
+    L.blink_convert_weights.argtypes = [P(blink_model_cfg), C.c_void_p, C.c_int]
     L.blink_kv_blocks_for_bytes.restype = C.c_int64
     L.blink_kv_blocks_for_bytes.argtypes = [P(blink_model_cfg), C.c_int, C.c_uint64]
     L.blink_create.restype = C.c_int
@@ -146,11 +150,11 @@ class BlinkError(RuntimeError):
         super().__init__(f"{where}: {lib().blink_strerror(code).decode()} ({code})")
 
 
-def make_model_cfg(m, weights_ptr=0, weights_bytes=0) -> blink_model_cfg:
+def make_model_cfg(m, weights_ptr=0, weights_bytes=0, weights_layout=0) -> blink_model_cfg:
     """m: synth.ModelCfg-like object (n_layers, d_model, ..., dtype 'bf16'|'fp32')."""
     return blink_model_cfg(C.sizeof(blink_model_cfg), m.n_layers, m.d_model, m.n_q_heads, m.n_kv_heads, m.head_dim,
                            m.d_ff, m.vocab, m.n_experts, m.top_k_experts, m.rope_theta, m.rms_eps,
-                           DTYPE_BF16 if m.dtype == "bf16" else DTYPE_FP32, weights_ptr, weights_bytes)
+                           DTYPE_BF16 if m.dtype == "bf16" else DTYPE_FP32, weights_layout, weights_ptr, weights_bytes)
 
 
 def blink_weights_bytes(m) -> int:
@@ -161,6 +165,15 @@ def blink_weights_bytes(m) -> int:
 def blink_weight_offset(m, tensor_id: int) -> int:
     cfg = make_model_cfg(m)
     return int(lib().blink_weight_offset(C.byref(cfg), tensor_id))
+
+
+def blink_convert_weights(m, weights, from_layout: int, to_layout: int, raise_on_error=True) -> int:
+    """weights: torch CUDA tensor holding the flat weight buffer; converted in place."""
+    cfg = make_model_cfg(m, weights.data_ptr(), weights.numel() * weights.element_size(), from_layout)
+    rc = lib().blink_convert_weights(C.byref(cfg), weights.data_ptr(), to_layout)
+    if rc != BLINK_OK and raise_on_error:
+        raise BlinkError(rc, "blink_convert_weights")
+    return rc
 
 
 def blink_kv_blocks_for_bytes(m, block_size: int, nbytes: int) -> int:
@@ -261,13 +274,13 @@ class Blink:
 
     def __init__(self, model, sched, weights=None, kv_pool=None, *, exec_mode=EXEC_PERSISTENT, gemm_impl=GEMM_AUTO,
                  control_only=False, start_paused=False, iteration_budget=0, idle_exit_us=0, trace_words=0,
-                 stats_iters=0, logits_capture=None, kv_bytes=None):
+                 stats_iters=0, logits_capture=None, kv_bytes=None, weights_layout=WEIGHTS_ROW_MAJOR):
         L = lib()
         self.model, self.sched = model, sched
         self._keep = (weights, kv_pool, logits_capture)
         wptr = weights.data_ptr() if weights is not None else 0
         wbytes = weights.numel() * weights.element_size() if weights is not None else 0
-        mc = make_model_cfg(model, wptr, wbytes)
+        mc = make_model_cfg(model, wptr, wbytes, weights_layout)
         cap_ptr = logits_capture.data_ptr() if logits_capture is not None else 0
         cap_rows = logits_capture.shape[0] if logits_capture is not None else 0
         sc = blink_sched_cfg(C.sizeof(blink_sched_cfg), sched.max_batch, sched.prefill_chunk_tokens, sched.n_slots,

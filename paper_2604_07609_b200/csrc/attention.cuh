@@ -81,6 +81,10 @@ __device__ __forceinline__ float fast_ex2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+__device__ __forceinline__ uint32_t pack_bf2(float lo, float hi) {
+  const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&v);
+}
 __device__ __forceinline__ float ldcg_f(const float* p) {
   float v;
   asm volatile("ld.global.cg.f32 %0, [%1];" : "=f"(v) : "l"(p) : "memory");
@@ -154,7 +158,7 @@ __device__ __forceinline__ void attn_decode_stream(const DevCtx& c, int layer, c
   constexpr int OC = NV >= LPK ? NV / LPK : 1;
   constexpr int NA = NREP * 8;       // accumulator values per lane
   constexpr int OWN = NA / KG;       // ... and after the sum over the key groups
-  constexpr int REC = NREP * (HD + 2);
+  constexpr int REC = NREP * HD + ((2 * NREP + 3) & ~3);  // floats per partial record, 16-byte multiple
   constexpr unsigned FULL = 0xffffffffu;
   const SchedState* ss = c.ss;
   const int n_dec = ss->cur_ndec, TT = ss->cur_TT, S = ss->cur_S;
@@ -188,9 +192,11 @@ __device__ __forceinline__ void attn_decode_stream(const DevCtx& c, int layer, c
     // ---- producer: keep up to ATT_NS tiles in flight ----
     while (!p_done && n_issued - n_consumed < ATT_NS) {
       if (pc.f == pc.f_end) {
-        int id = 0;
-        if (lane == 0) id = atomicAdd(ctr, 1);
-        id = __shfl_sync(FULL, id, 0);
+        int id = blockIdx.x * ATT_WARPS + w;   // first sub-range: the warp's own index
+        if (p_k > 0) {
+          if (lane == 0) id = atomicAdd(ctr, 1);
+          id = __shfl_sync(FULL, id, 0);
+        }
         if (lane == 0) g_att.ids[w][p_k & 7] = id;
         __syncwarp();
         p_k += 1;
@@ -403,21 +409,30 @@ __device__ __forceinline__ void attn_decode_stream(const DevCtx& c, int layer, c
         old = __shfl_sync(FULL, old, 0);
         if (old == j_last - j_first) {  // this warp delivered the last part: merge in sub-range order
           __threadfence();
-          for (int idx = lane; idx < NREP * HD; idx += 32) {
-            const int h = idx / HD;
+          // each lane merges four consecutive dims at a time; loads of the parts are independent
+          for (int i4 = lane; i4 < NREP * HD / 4; i4 += 32) {
+            const int h = (i4 * 4) / HD;
             float M = -INFINITY;
+#pragma unroll 4
             for (int j = j_first; j <= j_last; ++j) {
               const float* r = c.att_part + (size_t)(2 * j + (us <= j * S ? 0 : 1)) * REC;
-              M = fmaxf(M, ldcg_f(r + NREP * HD + h));
+              M = fmaxf(M, __ldcg(r + NREP * HD + h));
             }
-            float num = 0.f, den = 0.f;
+            float4 num = make_float4(0.f, 0.f, 0.f, 0.f);
+            float den = 0.f;
+#pragma unroll 4
             for (int j = j_first; j <= j_last; ++j) {
               const float* r = c.att_part + (size_t)(2 * j + (us <= j * S ? 0 : 1)) * REC;
-              const float f = fast_ex2(ldcg_f(r + NREP * HD + h) - M);
-              num += f * ldcg_f(r + idx);
-              den += f * ldcg_f(r + NREP * HD + NREP + h);
+              const float f = fast_ex2(__ldcg(r + NREP * HD + h) - M);
+              const float4 a4 = __ldcg(reinterpret_cast<const float4*>(r) + i4);
+              num.x += f * a4.x; num.y += f * a4.y; num.z += f * a4.z; num.w += f * a4.w;
+              den += f * __ldcg(r + NREP * HD + NREP + h);
             }
-            out[(size_t)t_row * c.q_dim + (size_t)(cc.g * NREP) * HD + idx] = __float2bfloat16_rn(num / den);
+            const float inv = 1.0f / den;
+            uint2 o2;
+            o2.x = pack_bf2(num.x * inv, num.y * inv);
+            o2.y = pack_bf2(num.z * inv, num.w * inv);
+            *reinterpret_cast<uint2*>(out + (size_t)t_row * c.q_dim + (size_t)(cc.g * NREP) * HD + i4 * 4) = o2;
           }
           if (lane == 0) c.att_cnt[unit] = 0;
         }
@@ -444,10 +459,6 @@ __device__ __forceinline__ void mma_bf16_16816(float* d, const uint32_t* a, uint
 }
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
-}
-__device__ __forceinline__ uint32_t pack_bf2(float lo, float hi) {
-  const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<const uint32_t*>(&v);
 }
 
 // One CTA: query rows [qblk*QROWS, +QROWS) of one request's chunk, one kv head; the NREP query

@@ -51,6 +51,30 @@ blink_sample_kernel(const float* logits, int rows, int V, const int* top_k, cons
   }
 }
 
+// In-place conversion of one GEMM matrix between row-major and the streaming tile layout.
+// A 128-row panel keeps its byte range; one CTA copies the panel to its scratch slot, then
+// writes it back in the other layout.
+__global__ void __launch_bounds__(256) blink_retile_kernel(char* base, long long n_panels, int K, char* scratch,
+                                                           int to_streaming) {
+  const size_t panel_bytes = (size_t)128 * K * 2;
+  const int cpr = K / 8;  // 16-byte chunks per row
+  uint4* tmp = reinterpret_cast<uint4*>(scratch + (size_t)blockIdx.x * panel_bytes);
+  for (long long p = blockIdx.x; p < n_panels; p += gridDim.x) {
+    uint4* panel = reinterpret_cast<uint4*>(base + (size_t)p * panel_bytes);
+    const int n16 = 128 * cpr;
+    for (int i = threadIdx.x; i < n16; i += blockDim.x) tmp[i] = panel[i];
+    __syncthreads();
+    for (int i = threadIdx.x; i < n16; i += blockDim.x) {
+      const int r = i / cpr, cc = i % cpr;
+      const int kb = cc >> 3, c8 = cc & 7;
+      const int tiled = kb * 1024 + r * 8 + (c8 ^ (r & 7));  // in 16-byte units
+      if (to_streaming) panel[tiled] = tmp[i];
+      else panel[i] = tmp[tiled];
+    }
+    __syncthreads();
+  }
+}
+
 __global__ void blink_clock_probe_kernel(Mailbox* mb) {
   mb->clock_probe = global_timer_ns();
   __threadfence_system();
@@ -88,7 +112,7 @@ bool model_ok(const blink_model_cfg* m) {
   if (rep != 1 && rep != 2 && rep != 4 && rep != 8) return false;
   if (m->dtype != BLINK_DTYPE_BF16 && m->dtype != BLINK_DTYPE_FP32) return false;
   if (m->n_experts < 0 || (m->n_experts > 0 && (m->top_k_experts < 1 || m->top_k_experts > m->n_experts))) return false;
-  if (m->d_model % 8 || m->d_ff % 8) return false;
+  if (m->d_model % 8 || m->d_model > 8192 || m->d_ff % 8) return false;   // rows move as 16-byte vectors
   return true;
 }
 
@@ -204,6 +228,8 @@ int launch_loop(blink_ctx* x) {
   std::atomic_thread_fence(std::memory_order_seq_cst);
   void* args[] = {(void*)&x->dc};
   const void* fn = x->ks.loop;
+  // the grid barrier counts arrivals from zero in every launch
+  if (cudaMemsetAsync(&x->dc.ss->bar_ctr, 0, sizeof(unsigned long long), x->stream) != cudaSuccess) return BLINK_ECUDA;
   cudaError_t e = cudaLaunchCooperativeKernel(fn, dim3(x->grid), dim3(FWD_THREADS), args, x->smem_bytes, x->stream);
   if (e != cudaSuccess) {
     x->mbox->loop_state = BLINK_LOOP_EXIT_ERROR;
@@ -271,6 +297,42 @@ uint64_t blink_weights_bytes(const blink_model_cfg* cfg) {
 uint64_t blink_weight_offset(const blink_model_cfg* cfg, int tensor_id) {
   if (!model_ok(cfg) || tensor_id < 0 || tensor_id > 9) return UINT64_MAX;
   return weight_layout(cfg).off[tensor_id];
+}
+
+int blink_convert_weights(const blink_model_cfg* cfg, void* weights, int to_layout) {
+  if (!model_ok(cfg) || !weights || ((uintptr_t)weights & 255)) return BLINK_EINVAL;
+  if (to_layout != BLINK_WEIGHTS_ROW_MAJOR && to_layout != BLINK_WEIGHTS_STREAMING) return BLINK_EINVAL;
+  if (cfg->weights_layout != BLINK_WEIGHTS_ROW_MAJOR && cfg->weights_layout != BLINK_WEIGHTS_STREAMING) return BLINK_EINVAL;
+  if (cfg->weights_layout == to_layout) return BLINK_OK;
+  if (cfg->dtype != BLINK_DTYPE_BF16) return BLINK_EINVAL;
+  const long long L = cfg->n_layers, d = cfg->d_model, F = cfg->d_ff, V = cfg->vocab;
+  const long long qd = (long long)cfg->n_q_heads * cfg->head_dim, kvd = (long long)cfg->n_kv_heads * cfg->head_dim;
+  const long long E1 = cfg->n_experts > 0 ? cfg->n_experts : 1;
+  // (tensor id, rows per layer slice, total rows, columns)
+  const long long rows_per[5] = {qd + 2 * kvd, d, 2 * F, d, V};
+  const long long rows_tot[5] = {L * (qd + 2 * kvd), L * d, L * E1 * 2 * F, L * E1 * d, V};
+  const long long cols[5] = {d, qd, d, F, d};
+  const int ids[5] = {1, 2, 3, 4, 9};
+  long long max_k = 0;
+  for (int i = 0; i < 5; ++i) {
+    if (rows_per[i] % 128 || cols[i] % 64) return BLINK_EINVAL;
+    if (cols[i] > max_k) max_k = cols[i];
+  }
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return BLINK_ECUDA;
+  char* scratch = nullptr;
+  if (cudaMalloc(&scratch, (size_t)sms * 128 * max_k * 2) != cudaSuccess) return BLINK_ENOMEM;
+  const Layout lo = weight_layout(cfg);
+  int rc = BLINK_OK;
+  for (int i = 0; i < 5 && rc == BLINK_OK; ++i) {
+    blink_retile_kernel<<<sms, 256>>>(static_cast<char*>(weights) + lo.off[ids[i]], rows_tot[i] / 128, (int)cols[i], scratch,
+                                      to_layout == BLINK_WEIGHTS_STREAMING);
+    if (cudaGetLastError() != cudaSuccess) rc = BLINK_ECUDA;
+  }
+  if (cudaDeviceSynchronize() != cudaSuccess) rc = BLINK_ECUDA;
+  cudaFree(scratch);
+  return rc;
 }
 
 int64_t blink_kv_blocks_for_bytes(const blink_model_cfg* cfg, int block_size, uint64_t bytes) {
@@ -429,6 +491,10 @@ int blink_create(const blink_model_cfg* model, const blink_sched_cfg* sched, con
   if (!c.control_only && model->dtype == BLINK_DTYPE_BF16 && sched->gemm_impl != BLINK_GEMM_SIMT)
     c.gemm_tc = tc_available() && tc_shape_ok(c);
   if (sched->gemm_impl == BLINK_GEMM_TC && !c.gemm_tc) { delete x; return BLINK_EINVAL; }
+  c.w_streaming = model->weights_layout == BLINK_WEIGHTS_STREAMING;
+  if (model->weights_layout != BLINK_WEIGHTS_ROW_MAJOR && model->weights_layout != BLINK_WEIGHTS_STREAMING) { delete x; return BLINK_EINVAL; }
+  // the streaming layout is read by the tensor-core path only
+  if (c.w_streaming && !c.control_only && (!c.gemm_tc || !tc_streaming_ok(c))) { delete x; return BLINK_EINVAL; }
   c.iteration_budget = c.stepped ? 0 : sched->iteration_budget;
   const double cyc_per_us = 2000.0;  // upper bound on the SM clock: time-outs only get longer at lower clocks
   const int64_t idle_us = sched->idle_exit_us > 0 ? sched->idle_exit_us : 2000000;
@@ -475,12 +541,12 @@ int blink_create(const blink_model_cfg* model, const blink_sched_cfg* sched, con
     if (c.dtype == BLINK_DTYPE_BF16) {
       TRY(dev_alloc(x, &p, TM * c.q_dim * esz)); c.qb = p;
       c.n_warps_grid = x->n_sms * (FWD_THREADS / 32);
-      c.att_sub_max = 4ll * c.n_warps_grid + (long long)MB * c.Hkv * c.max_blocks_seq / 64 + 8;
+      c.att_sub_max = 2ll * c.n_warps_grid + (long long)MB * c.Hkv * c.max_blocks_seq / 24 + 8;
       TRY(dev_alloc(x, &c.dec_row, MB)); TRY(dev_alloc(x, &c.dec_bslot, MB)); TRY(dev_alloc(x, &c.dec_nctx, MB));
       TRY(dev_alloc(x, &c.dec_kbpre, MB + 1));
       TRY(dev_alloc(x, &c.pf_item, TM / 16 + MB + 1)); TRY(dev_alloc(x, &c.pf_qb, TM / 16 + MB + 1));
       TRY(dev_alloc(x, &c.att_ctr, (size_t)c.L)); TRY(dev_alloc(x, &c.att_cnt, MB * c.Hkv));
-      TRY(dev_alloc(x, &c.att_part, (size_t)(2 * c.att_sub_max) * c.n_rep * (c.hd + 2), false));
+      TRY(dev_alloc(x, &c.att_part, (size_t)(2 * c.att_sub_max) * (c.n_rep * c.hd + ((2 * c.n_rep + 3) & ~3)), false));
     }
     TRY(dev_alloc(x, &p, TM * c.q_dim * esz)); c.attn = p;
     TRY(dev_alloc(x, &c.gu, TM * 2 * c.F));

@@ -45,38 +45,40 @@ __device__ __forceinline__ void dev_fail(const DevCtx& c, int code) {
   atomicExch(&c.ss->abort_flag, 1);
 }
 
-// Grid-wide barrier with a bounded wait.  Returns false when the loop must unwind
-// (time-out here or abort raised elsewhere).  `gen` is the caller's private copy of
-// the barrier generation (thread 0 of each CTA keeps it).
-__device__ __forceinline__ bool grid_barrier(const DevCtx& c, unsigned int& gen) {
+__device__ __forceinline__ unsigned long long ld_acquire_gpu_u64(const unsigned long long* p) {
+  unsigned long long v;
+  asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+  return v;
+}
+
+// Grid-wide barrier with a bounded wait: every CTA adds one to a monotone counter (reset by the
+// host before each launch) and waits until it reaches the next multiple of the grid size.
+// Returns false when the loop must unwind (time-out here or abort raised elsewhere).  `target`
+// is the caller's private running total (thread 0 of each CTA keeps it).
+__device__ __forceinline__ bool grid_barrier(const DevCtx& c, unsigned long long& target) {
   __shared__ int s_ok;
   __syncthreads();
   if (threadIdx.x == 0) {
     int ok = 1;
     SchedState* ss = c.ss;
+    target += gridDim.x;
     __threadfence();
-    unsigned int prev = atomicAdd(&ss->bar_count, 1u);
-    if (prev == gridDim.x - 1) {
-      ss->bar_count = 0;
-      __threadfence();
-      st_release_gpu_u32(&ss->bar_gen, gen + 1);
-    } else {
-      long long t0 = clock64();
-      unsigned int polls = 0;
-      while (ld_acquire_gpu_u32(&ss->bar_gen) == gen) {
-        if ((++polls & 63u) == 0) {
-          if (*(volatile int*)&ss->abort_flag) { ok = 0; break; }
-          if ((unsigned long long)(clock64() - t0) > c.barrier_timeout_cycles) {
-            dev_fail(c, DEV_ERR_BARRIER_TIMEOUT);
-            ok = 0;
-            break;
-          }
-          if (polls > 4096u) __nanosleep(200);
+    asm volatile("red.release.gpu.global.add.u64 [%0], 1;" ::"l"(&ss->bar_ctr) : "memory");
+    long long t0 = 0;
+    unsigned int polls = 0;
+    while (ld_acquire_gpu_u64(&ss->bar_ctr) < target) {
+      if ((++polls & 63u) == 0) {
+        if (*(volatile int*)&ss->abort_flag) { ok = 0; break; }
+        if (t0 == 0) t0 = clock64();
+        if ((unsigned long long)(clock64() - t0) > c.barrier_timeout_cycles) {
+          dev_fail(c, DEV_ERR_BARRIER_TIMEOUT);
+          ok = 0;
+          break;
         }
+        if (polls > 4096u) __nanosleep(200);
       }
     }
     if (*(volatile int*)&ss->abort_flag) ok = 0;
-    gen += 1;
     s_ok = ok;
   }
   __syncthreads();
@@ -498,8 +500,9 @@ static __device__ int schedule_step(const DevCtx& c, unsigned long long visible)
   __syncthreads();
 
   // per-row metadata: token id, position, owning item, KV slot
+  // every warp of the grid starts on the sub-range of its own index; the counter hands out the rest
   if (c.att_ctr != nullptr)
-    for (int i = tid; i < c.L; i += CTRL_THREADS) c.att_ctr[i] = 0;
+    for (int i = tid; i < c.L; i += CTRL_THREADS) c.att_ctr[i] = c.n_warps_grid;
   for (int r = tid; r < T; r += CTRL_THREADS) {
     int lo = 0, hi = n_items;  // last item with qstart <= r
     while (hi - lo > 1) {
@@ -530,9 +533,11 @@ static __device__ int schedule_step(const DevCtx& c, unsigned long long visible)
     ss->pending_post = 1;
     if (c.dec_row != nullptr) {
       const long long TT = (long long)tot_kb * c.Hkv;
-      long long S = (TT + 4ll * c.n_warps_grid - 1) / (4ll * c.n_warps_grid);
+      // sub-ranges: k per warp of the grid, about 32 to 64 tiles each once there is that much work
+      const long long NW = c.n_warps_grid;
+      const long long k = (TT + 48 * NW - 1) / (48 * NW) > 1 ? (TT + 48 * NW - 1) / (48 * NW) : 1;
+      long long S = (TT + k * NW - 1) / (k * NW);
       if (S < 1) S = 1;
-      if (S > 64) S = 64;
       while ((TT + S - 1) / S > c.att_sub_max) S *= 2;   // cannot happen with the sizes set at create
       c.dec_kbpre[n_dec_att] = tot_kb;
       ss->cur_ndec = n_dec_att;

@@ -103,8 +103,7 @@ struct SchedState {
   int pending_post;                 // a forward ran and its post step is outstanding
   int trace_off;                    // tracing stopped (overflow)
   int abort_flag;
-  unsigned int bar_count;
-  unsigned int bar_gen;
+  unsigned long long bar_ctr;       // grid barrier: arrivals since the launch (the host zeroes it before a launch)
   unsigned long long cur_t_begin, cur_t_forward;
   int exit_reason;
   int pad;
@@ -136,6 +135,7 @@ struct DevCtx {
   int MB, chunk, n_slots, max_prompt, max_new, Tmax, bs, n_blocks, max_blocks_seq, max_pos;
   int control_only, start_paused, stepped, gemm_tc;
   int n_warps_grid;  // warps of the whole grid (attention work split)
+  int w_streaming;   // GEMM matrices are stored as contiguous pre-swizzled 128 x 64 tiles
   long long iteration_budget;
   unsigned long long idle_exit_cycles, barrier_timeout_cycles;
   // ring in HBM

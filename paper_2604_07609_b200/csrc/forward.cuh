@@ -62,8 +62,77 @@ __device__ __forceinline__ void zero_floats(float* p, long long n_floats) {
     q[i] = make_float4(0.f, 0.f, 0.f, 0.f);
 }
 
+// store four consecutive values in the operand type
+template <typename WT>
+__device__ __forceinline__ void store4(WT* p, float a, float b, float c, float d);
+template <>
+__device__ __forceinline__ void store4<float>(float* p, float a, float b, float c, float d) {
+  *reinterpret_cast<float4*>(p) = make_float4(a, b, c, d);
+}
+template <>
+__device__ __forceinline__ void store4<__nv_bfloat16>(__nv_bfloat16* p, float a, float b, float c, float d) {
+  const __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
+  uint2 v;
+  v.x = *reinterpret_cast<const uint32_t*>(&lo);
+  v.y = *reinterpret_cast<const uint32_t*>(&hi);
+  *reinterpret_cast<uint2*>(p) = v;
+}
+template <typename WT>
+__device__ __forceinline__ float4 load4(const WT* p);
+template <>
+__device__ __forceinline__ float4 load4<float>(const float* p) { return *reinterpret_cast<const float4*>(p); }
+template <>
+__device__ __forceinline__ float4 load4<__nv_bfloat16>(const __nv_bfloat16* p) {
+  const uint2 v = *reinterpret_cast<const uint2*>(p);
+  const __nv_bfloat162 lo = *reinterpret_cast<const __nv_bfloat162*>(&v.x), hi = *reinterpret_cast<const __nv_bfloat162*>(&v.y);
+  const float2 a = __bfloat1622float2(lo), b = __bfloat1622float2(hi);
+  return make_float4(a.x, a.y, b.x, b.y);
+}
+
+// One CTA normalises one row: n = x / sqrt(mean(x^2) + eps) * g.  Every thread keeps its part of
+// the row (16-byte vectors, up to NORM_MAXV of them: d <= 8192) in registers between the sum and
+// the scaling, so the row is read once.  `src_embed` non-null: the row is first gathered from
+// the embedding table into the residual stream.
+constexpr int NORM_MAXV = 8;
+template <typename WT>
+__device__ __forceinline__ void norm_row_cta(const DevCtx& c, float* hrow, const WT* src_embed, const float* g, WT* orow,
+                                             float* s_red) {
+  const int d = c.d;
+  float4 v[NORM_MAXV];
+  float ss = 0.f;
+#pragma unroll
+  for (int k = 0; k < NORM_MAXV; ++k) {
+    const int i = (k * FWD_THREADS + threadIdx.x) * 4;
+    if (i < d) {
+      if (src_embed != nullptr) {
+        v[k] = load4<WT>(src_embed + i);
+        *reinterpret_cast<float4*>(hrow + i) = v[k];
+      } else {
+        v[k] = *reinterpret_cast<const float4*>(hrow + i);
+      }
+    }
+  }
+#pragma unroll
+  for (int k = 0; k < NORM_MAXV; ++k) {
+    const int i = (k * FWD_THREADS + threadIdx.x) * 4;
+    if (i < d) {  // fixed order
+      ss = fmaf(v[k].x, v[k].x, ss); ss = fmaf(v[k].y, v[k].y, ss); ss = fmaf(v[k].z, v[k].z, ss); ss = fmaf(v[k].w, v[k].w, ss);
+    }
+  }
+  ss = block_sum(ss, s_red);
+  const float inv = 1.0f / sqrtf(ss / (float)d + c.rms_eps);
+#pragma unroll
+  for (int k = 0; k < NORM_MAXV; ++k) {
+    const int i = (k * FWD_THREADS + threadIdx.x) * 4;
+    if (i < d) {
+      const float4 gg = *reinterpret_cast<const float4*>(g + i);
+      store4<WT>(orow + i, v[k].x * inv * gg.x, v[k].y * inv * gg.y, v[k].z * inv * gg.z, v[k].w * inv * gg.w);
+    }
+  }
+}
+
 // ---- RMSNorm of the residual rows into the operand buffer; layer 0 gathers the
-// embedding first.  n = x / sqrt(mean(x^2) + eps) * g
+// embedding first.
 template <typename WT>
 static __device__ void phase_norm(const DevCtx& c, int layer, int which /*0: norm1, 1: norm2*/) {
   __shared__ float s_red[FWD_THREADS / 32];
@@ -73,19 +142,8 @@ static __device__ void phase_norm(const DevCtx& c, int layer, int which /*0: nor
   // the split-K tensor-core GEMM that follows adds partial sums into its output
   if (c.gemm_tc) zero_floats(which == 0 ? c.qkv : c.gu, (long long)T * (which == 0 ? c.qkv_dim : 2 * c.F));
   for (int t = blockIdx.x; t < T; t += gridDim.x) {
-    float* hrow = c.h + (size_t)t * c.d;
-    if (which == 0 && layer == 0) {
-      const WT* e = wptr<WT>(c, 0) + (size_t)c.tok_id[t] * c.d;
-      for (int i = threadIdx.x; i < c.d; i += FWD_THREADS) hrow[i] = OpType<WT>::to_f(e[i]);
-      __syncthreads();
-    }
-    float ss = 0.f;
-    for (int i = threadIdx.x; i < c.d; i += FWD_THREADS) { const float v = hrow[i]; ss += v * v; }
-    ss = block_sum(ss, s_red);
-    const float inv = 1.0f / sqrtf(ss / (float)c.d + c.rms_eps);
-    for (int i = threadIdx.x; i < c.d; i += FWD_THREADS)
-      out[(size_t)t * c.d + i] = OpType<WT>::from_f(hrow[i] * inv * g[i]);
-    __syncthreads();
+    const WT* e = (which == 0 && layer == 0) ? wptr<WT>(c, 0) + (size_t)c.tok_id[t] * c.d : nullptr;
+    norm_row_cta<WT>(c, c.h + (size_t)t * c.d, e, g, out + (size_t)t * c.d, s_red);
   }
 }
 
@@ -97,16 +155,8 @@ static __device__ void phase_final_norm(const DevCtx& c) {
   const float* g = wptr_f(c, 8);
   WT* out = reinterpret_cast<WT*>(c.xs);
   if (c.gemm_tc) zero_floats(c.logits, (long long)R * c.V);
-  for (int r = blockIdx.x; r < R; r += gridDim.x) {
-    const float* hrow = c.h + (size_t)c.row_tok[r] * c.d;
-    float ss = 0.f;
-    for (int i = threadIdx.x; i < c.d; i += FWD_THREADS) { const float v = hrow[i]; ss += v * v; }
-    ss = block_sum(ss, s_red);
-    const float inv = 1.0f / sqrtf(ss / (float)c.d + c.rms_eps);
-    for (int i = threadIdx.x; i < c.d; i += FWD_THREADS)
-      out[(size_t)r * c.d + i] = OpType<WT>::from_f(hrow[i] * inv * g[i]);
-    __syncthreads();
-  }
+  for (int r = blockIdx.x; r < R; r += gridDim.x)
+    norm_row_cta<WT>(c, c.h + (size_t)c.row_tok[r] * c.d, nullptr, g, out + (size_t)r * c.d, s_red);
 }
 
 // ---- CUDA-core reference GEMM: out[t][n] (+)= sum_k x[t][k] * w[n][k], fp32 accumulate.
@@ -188,41 +238,51 @@ __device__ __forceinline__ WT* kv_tile(const DevCtx& c, int layer, int kv, int b
 
 template <typename WT>
 static __device__ void phase_rope_kv(const DevCtx& c, int layer) {
+  // one thread: four consecutive rotation pairs (i .. i+3, i+half .. i+half+3) of one head of one row
   const int T = c.ss->cur_T;
-  const int half = c.hd / 2;
+  const int half = c.hd / 2, quads = half / 4;
   const int heads = c.Hq + 2 * c.Hkv;
-  const long long total = (long long)T * heads * half;
+  const long long total = (long long)T * heads * quads;
   for (long long idx = (long long)blockIdx.x * FWD_THREADS + threadIdx.x; idx < total;
        idx += (long long)gridDim.x * FWD_THREADS) {
-    const int i = (int)(idx % half);
-    const int hh = (int)((idx / half) % heads);
-    const int t = (int)(idx / ((long long)half * heads));
+    const int i = (int)(idx % quads) * 4;
+    const int hh = (int)((idx / quads) % heads);
+    const int t = (int)(idx / ((long long)quads * heads));
     float* row = c.qkv + (size_t)t * c.qkv_dim + (size_t)hh * c.hd;
-    const int pos = c.tok_pos[t];
-    const float x1 = row[i], x2 = row[i + half];
+    const float4 x1 = *reinterpret_cast<const float4*>(row + i), x2 = *reinterpret_cast<const float4*>(row + i + half);
     if (hh < c.Hq + c.Hkv) {
-      const float cs = c.rope_cos[(size_t)pos * half + i], sn = c.rope_sin[(size_t)pos * half + i];
-      const float y1 = x1 * cs - x2 * sn, y2 = x2 * cs + x1 * sn;
+      const int pos = c.tok_pos[t];
+      const float4 cs = *reinterpret_cast<const float4*>(c.rope_cos + (size_t)pos * half + i);
+      const float4 sn = *reinterpret_cast<const float4*>(c.rope_sin + (size_t)pos * half + i);
+      // explicit fused forms: every instance of this code rounds the same way
+#define BLINK_ROT1(a, b, cc, ss_) fmaf((a), (cc), -__fmul_rn((b), (ss_)))
+#define BLINK_ROT2(a, b, cc, ss_) fmaf((b), (cc), __fmul_rn((a), (ss_)))
+      const float4 y1 = make_float4(BLINK_ROT1(x1.x, x2.x, cs.x, sn.x), BLINK_ROT1(x1.y, x2.y, cs.y, sn.y),
+                                    BLINK_ROT1(x1.z, x2.z, cs.z, sn.z), BLINK_ROT1(x1.w, x2.w, cs.w, sn.w));
+      const float4 y2 = make_float4(BLINK_ROT2(x1.x, x2.x, cs.x, sn.x), BLINK_ROT2(x1.y, x2.y, cs.y, sn.y),
+                                    BLINK_ROT2(x1.z, x2.z, cs.z, sn.z), BLINK_ROT2(x1.w, x2.w, cs.w, sn.w));
+#undef BLINK_ROT1
+#undef BLINK_ROT2
       if (hh < c.Hq) {
         if constexpr (sizeof(WT) == 2) {   // 16-bit path: q is an operand of the attention contraction
           WT* qd = reinterpret_cast<WT*>(c.qb) + (size_t)t * c.q_dim + (size_t)hh * c.hd;
-          qd[i] = OpType<WT>::from_f(y1);
-          qd[i + half] = OpType<WT>::from_f(y2);
+          store4<WT>(qd + i, y1.x, y1.y, y1.z, y1.w);
+          store4<WT>(qd + i + half, y2.x, y2.y, y2.z, y2.w);
         } else {
-          row[i] = y1;
-          row[i + half] = y2;
+          *reinterpret_cast<float4*>(row + i) = y1;
+          *reinterpret_cast<float4*>(row + i + half) = y2;
         }
       } else {
         const int sm = c.tok_slotmap[t];
         WT* dst = kv_tile<WT>(c, layer, 0, sm / c.bs, hh - c.Hq) + (size_t)(sm % c.bs) * c.hd;
-        dst[i] = OpType<WT>::from_f(y1);
-        dst[i + half] = OpType<WT>::from_f(y2);
+        store4<WT>(dst + i, y1.x, y1.y, y1.z, y1.w);
+        store4<WT>(dst + i + half, y2.x, y2.y, y2.z, y2.w);
       }
     } else {
       const int sm = c.tok_slotmap[t];
       WT* dst = kv_tile<WT>(c, layer, 1, sm / c.bs, hh - c.Hq - c.Hkv) + (size_t)(sm % c.bs) * c.hd;
-      dst[i] = OpType<WT>::from_f(x1);
-      dst[i + half] = OpType<WT>::from_f(x2);
+      store4<WT>(dst + i, x1.x, x1.y, x1.z, x1.w);
+      store4<WT>(dst + i + half, x2.x, x2.y, x2.z, x2.w);
     }
   }
 }
@@ -368,12 +428,15 @@ template <typename WT>
 static __device__ void phase_silu_mul(const DevCtx& c) {
   const int T = c.ss->cur_T;
   WT* out = reinterpret_cast<WT*>(c.act);
-  const long long total = (long long)T * c.F;
+  const int F4 = c.F / 4;
+  const long long total = (long long)T * F4;
   for (long long idx = (long long)blockIdx.x * FWD_THREADS + threadIdx.x; idx < total;
        idx += (long long)gridDim.x * FWD_THREADS) {
-    const int t = (int)(idx / c.F), j = (int)(idx % c.F);
-    const float gte = c.gu[(size_t)t * 2 * c.F + j], up = c.gu[(size_t)t * 2 * c.F + c.F + j];
-    out[idx] = OpType<WT>::from_f(gte / (1.0f + __expf(-gte)) * up);
+    const int t = (int)(idx / F4), j = (int)(idx % F4) * 4;
+    const float4 g = *reinterpret_cast<const float4*>(c.gu + (size_t)t * 2 * c.F + j);
+    const float4 u = *reinterpret_cast<const float4*>(c.gu + (size_t)t * 2 * c.F + c.F + j);
+    store4<WT>(out + (size_t)t * c.F + j, g.x / (1.0f + __expf(-g.x)) * u.x, g.y / (1.0f + __expf(-g.y)) * u.y,
+               g.z / (1.0f + __expf(-g.z)) * u.z, g.w / (1.0f + __expf(-g.w)) * u.w);
   }
 }
 

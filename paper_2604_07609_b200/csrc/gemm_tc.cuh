@@ -107,6 +107,13 @@ __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* m
       : "memory");
 }
 
+__device__ __forceinline__ void tma_bulk_load(void* smem_dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   smem_u32(smem_dst)),
+               "l"(src), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -162,7 +169,7 @@ __device__ __forceinline__ void tc_init(const DevCtx& c, float*, TcState& s) {
   s.fill_bits = s.use_bits = s.acc_mma = s.acc_epi = 0;
   if (!c.gemm_tc) return;
   if (threadIdx.x == 32) {
-    for (int i = 0; i < TC_MAX_STAGES; ++i) { mbar_init(&g_tc.full[i], 1); mbar_init(&g_tc.empty[i], 1); }
+    for (int i = 0; i < TC_MAX_STAGES; ++i) { mbar_init(&g_tc.full[i], 2); mbar_init(&g_tc.empty[i], 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(&g_tc.acc_full[b], 1); mbar_init(&g_tc.acc_empty[b], 4); }
     g_tc.dead = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -210,7 +217,11 @@ static __device__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int whi
   const CUtensorMap* map_a = &maps->w[which];
   const CUtensorMap* map_b = &maps->act[act_id][box_id];
   const int row_a0 = which == GEMM_LMHEAD ? 0 : layer * N;
-  const uint32_t stage_bytes = TC_A_BYTES + (uint32_t)box_rows * 128u;
+  // A stage holds one k-block, or two when the token tile is small and the weights are stored as
+  // contiguous tiles (then one bulk copy brings 32 KiB): fewer, larger copies per producer step.
+  const int KPS = (c.w_streaming && box_rows <= 128) ? 2 : 1;
+  const uint32_t b_bytes = (uint32_t)box_rows * 128u;
+  const uint32_t stage_bytes = (uint32_t)KPS * (TC_A_BYTES + b_bytes);
   int S = TC_TILE_BUDGET / (int)stage_bytes;
   if (S > TC_MAX_STAGES) S = TC_MAX_STAGES;
   // tiles need 1024-byte alignment for the 128-byte swizzle
@@ -222,20 +233,36 @@ static __device__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int whi
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile int* dead = &g_tc.dead;
 
-  if (warp == 0) {
+  if (warp == 0 || warp == 2) {
+    // two producer threads: warp 0 streams the weight tiles, warp 2 the token tiles; both walk the
+    // same sequence of stages (nk k-blocks of one segment each)
     if (lane == 0) {
       int stage = 0;
-      for (long long u = u0; u < u1; ++u) {
+      long long u = u0;
+      while (u < u1) {
+        const long long seg_end = min(u1, (u / kblocks + 1) * (long long)kblocks);
+        const int nk = (int)min((long long)KPS, seg_end - u);
         const int kb = (int)(u % kblocks);
         const int nt = (int)((u / kblocks) % ntiles);
         const int pass = (int)(u / ((long long)kblocks * ntiles));
         // the n-th fill of a stage waits for its (n-1)-th release
         if (!mbar_wait(c, &g_tc.empty[stage], ((tc.fill_bits >> stage) & 1u) ^ 1u, dead)) break;
         tc.fill_bits ^= 1u << stage;
-        mbar_expect_tx(&g_tc.full[stage], stage_bytes);
         char* sa = tiles + (size_t)stage * stage_bytes;
-        tma_load_2d(sa, map_a, kb * 64, row_a0 + nt * 128, &g_tc.full[stage]);
-        tma_load_2d(sa + TC_A_BYTES, map_b, kb * 64, pass * 256, &g_tc.full[stage]);
+        if (warp == 0) {
+          mbar_expect_tx(&g_tc.full[stage], (uint32_t)nk * TC_A_BYTES);
+          if (c.w_streaming) {  // contiguous tiles, already in the shared-memory operand image
+            tma_bulk_load(sa, reinterpret_cast<const char*>(a.w) + ((size_t)nt * kblocks + kb) * TC_A_BYTES,
+                          (uint32_t)nk * TC_A_BYTES, &g_tc.full[stage]);
+          } else {
+            tma_load_2d(sa, map_a, kb * 64, row_a0 + nt * 128, &g_tc.full[stage]);
+          }
+        } else {
+          mbar_expect_tx(&g_tc.full[stage], (uint32_t)nk * b_bytes);
+          for (int j = 0; j < nk; ++j)
+            tma_load_2d(sa + KPS * TC_A_BYTES + j * b_bytes, map_b, (kb + j) * 64, pass * 256, &g_tc.full[stage]);
+        }
+        u += nk;
         if (++stage == S) stage = 0;
       }
     }
@@ -256,19 +283,24 @@ static __device__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int whi
         tc_fence_after();
         bool first = true;
         bool ok = true;
-        for (; u < seg_end; ++u) {
+        while (u < seg_end) {
+          const int nk = (int)min((long long)KPS, seg_end - u);
           if (!mbar_wait(c, &g_tc.full[stage], (tc.use_bits >> stage) & 1u, dead)) { ok = false; break; }
           tc.use_bits ^= 1u << stage;
           tc_fence_after();
           const uint32_t sa = smem_u32(tiles + (size_t)stage * stage_bytes);
-          const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sa + TC_A_BYTES);
+          for (int j = 0; j < nk; ++j) {
+            const uint64_t da = smem_desc_sw128(sa + j * TC_A_BYTES);
+            const uint64_t db = smem_desc_sw128(sa + KPS * TC_A_BYTES + j * b_bytes);
 #pragma unroll
-          for (int k16 = 0; k16 < 4; ++k16) {
-            // 16 bf16 = 32 bytes further along K inside the swizzle atom: +2 in 16-byte units
-            umma_bf16(d_tmem, da + (uint64_t)(2 * k16), db + (uint64_t)(2 * k16), idesc, (first && k16 == 0) ? 0u : 1u);
+            for (int k16 = 0; k16 < 4; ++k16) {
+              // 16 bf16 = 32 bytes further along K inside the swizzle atom: +2 in 16-byte units
+              umma_bf16(d_tmem, da + (uint64_t)(2 * k16), db + (uint64_t)(2 * k16), idesc, (first && k16 == 0) ? 0u : 1u);
+            }
+            first = false;
           }
-          first = false;
           umma_commit(&g_tc.empty[stage]);
+          u += nk;
           if (++stage == S) stage = 0;
         }
         if (!ok) break;
@@ -354,6 +386,10 @@ inline int tc_shape_ok(const DevCtx& c) {
   return c.dtype == 0 && c.d % 64 == 0 && c.q_dim % 64 == 0 && c.F % 64 == 0 && c.V % 4 == 0 && c.E == 0;
 }
 inline int tc_available() { return tc_encode_fn() != nullptr; }
+// The streaming layout needs whole 128-row panels per layer in every GEMM matrix.
+inline int tc_streaming_ok(const DevCtx& c) {
+  return tc_shape_ok(c) && c.qkv_dim % 128 == 0 && c.d % 128 == 0 && (2 * c.F) % 128 == 0 && c.V % 128 == 0;
+}
 
 inline int tc_host_setup(TcHost& h, DevCtx& c) {
   EncodeTiledFn enc = tc_encode_fn();

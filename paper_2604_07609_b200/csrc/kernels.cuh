@@ -65,8 +65,7 @@ __device__ __forceinline__ void run_phase(const DevCtx& c, int phase, int layer,
 template <typename WT, int HD, int NREP>
 __global__ void __launch_bounds__(FWD_THREADS, 1) blink_loop_kernel(const __grid_constant__ DevCtx c) {
   extern __shared__ __align__(1024) float smem[];
-  unsigned int gen = 0;
-  if (threadIdx.x == 0) gen = ld_acquire_gpu_u32(&c.ss->bar_gen);
+  unsigned long long gen = 0;   // arrivals this CTA expects at its next grid barrier
   long long launch_iters = 0;
   TcState tc;
   tc_init(c, smem, tc);

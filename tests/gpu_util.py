@@ -62,18 +62,20 @@ def oracle_run(model, sched, reqs, weights_cpu, act_round, dtype=np.float64):
 
 
 def gpu_run_forced(model, sched, reqs, weights_cpu, forced, *, exec_mode=B.EXEC_PERSISTENT, gemm_impl=B.GEMM_AUTO,
-                   capture_rows=None, step_iters=4, iteration_budget=0):
+                   capture_rows=None, step_iters=4, iteration_budget=0, weights_layout=B.WEIGHTS_ROW_MAJOR):
     """Teacher-forced run: request t is fed forced[t] but reports its own samples.
     Returns (trace, sampled tokens by ticket, captured logits [rows, V] as numpy)."""
     dev = torch.device("cuda:0")
     wd = weights_cpu.to(dev)
+    if weights_layout != B.WEIGHTS_ROW_MAJOR:
+        B.blink_convert_weights(model, wd, B.WEIGHTS_ROW_MAJOR, weights_layout)
     kv = torch.zeros(sched.n_blocks * B.kv_bytes_per_block(model, sched.block_size), dtype=torch.uint8, device=dev)
     total = sum(r.max_new for r in reqs)
     cap = torch.zeros((capture_rows or total, model.vocab), dtype=torch.float32, device=dev)
     stepped = exec_mode == B.EXEC_STEPPED
     eng = B.Blink(model, sched, wd, kv, start_paused=True, exec_mode=exec_mode, gemm_impl=gemm_impl,
                   trace_words=1 << 22, stats_iters=1 << 14, logits_capture=cap, idle_exit_us=300_000,
-                  iteration_budget=iteration_budget)
+                  iteration_budget=iteration_budget, weights_layout=weights_layout)
     try:
         for r in reqs:
             eng.submit_request(r, forced_tokens=None if forced is None else forced[r.ticket])

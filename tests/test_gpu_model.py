@@ -164,3 +164,40 @@ def test_tensor_core_and_cuda_core_paths_agree():
     b = gpu_run_forced(model, sched, reqs, w, forced, gemm_impl=B.GEMM_TC, exec_mode=B.EXEC_STEPPED)
     assert np.abs(a[2] - b[2]).max() < TOL_BF16  # same bf16 products, other summation order, so roundings flip
     assert_traces_equal([{**r, "sampled": []} for r in a[0]], [{**r, "sampled": []} for r in b[0]])
+
+
+def test_streaming_weight_layout_round_trip_and_parity():
+    """The GEMM matrices converted in place to the tile-contiguous streaming layout: converting back
+    restores every byte, and the loop reading the streaming layout meets the same tolerance."""
+    model = model_cfg(1, d_model=512, n_q_heads=4, n_kv_heads=1, head_dim=128, d_ff=1536, vocab=4480, dtype="bf16")
+    sched = sched_cfg(1, prefill_chunk_tokens=300, max_batch=8, n_blocks=256, max_prompt=320, max_new=8)
+    rng = np.random.default_rng(22)
+    from synth.workload import Request
+    reqs = [Request(t, 0.0, rng.integers(0, model.vocab, size=int(p)).astype(np.int32), 6)
+            for t, p in enumerate([310, 17, 301, 64, 129, 5])]
+    w = make_weights(model, 78, "cpu", random_gains=True)
+    wd = w.cuda()
+    B.blink_convert_weights(model, wd, B.WEIGHTS_ROW_MAJOR, B.WEIGHTS_STREAMING)
+    assert not torch.equal(wd.cpu(), w)
+    back = wd.clone()
+    B.blink_convert_weights(model, back, B.WEIGHTS_STREAMING, B.WEIGHTS_ROW_MAJOR)
+    assert torch.equal(back.cpu(), w)
+    # a 128 x 64 tile of wqkv holds exactly the values of the row-major block it came from
+    off = B.blink_weight_offset(model, 1)
+    K = model.d_model
+    tile = wd[off:off + 16384].cpu().view(torch.bfloat16).view(128, 8, 8)          # [row][chunk position][8]
+    rm = w[off:off + 128 * K * 2].view(torch.bfloat16).view(128, K)[:, :64].reshape(128, 8, 8)
+    for r in (0, 1, 7, 8, 77, 127):
+        for c8 in range(8):
+            assert torch.equal(tile[r, c8 ^ (r & 7)], rm[r, c8])
+    ora = oracle_run(model, sched, reqs, w, O2.round_bf16)
+    trace, toks, logits, _ = gpu_run_forced(model, sched, reqs, w, ora["tokens"], gemm_impl=B.GEMM_TC,
+                                            weights_layout=B.WEIGHTS_STREAMING)
+    lo = np.stack([row for (_, _, _, _, row) in ora["logits"]])
+    err = np.abs(logits.astype(np.float64) - lo).max()
+    print(f"streaming layout: max-abs logit error {err:.3e}")
+    assert err <= TOL_BF16
+    assert_traces_equal([{**r, "sampled": []} for r in trace], [{**r, "sampled": []} for r in ora["trace"]])
+    # the SIMT path cannot read the streaming layout: refused, not misread
+    with pytest.raises(B.BlinkError):
+        gpu_run_forced(model, sched, reqs, w, ora["tokens"], gemm_impl=B.GEMM_SIMT, weights_layout=B.WEIGHTS_STREAMING)
