@@ -505,6 +505,70 @@ static __device__ int sample_row(const float* lg, int V, int top_k, float temp, 
     return result;
   }
   const int k = min(top_k, V);
+  // Fast path.  Every thread takes the maximum of its strided share of the row; the k-th largest
+  // of those 256 maxima, tau, is a lower bound of the k-th largest z of the row (k threads hold an
+  // element >= tau each), so {z >= tau} contains the top k and is usually a few dozen elements.
+  // z = logit / T is monotone in the logit, so the maxima can be taken on logits and divided once.
+  {
+    float* s_tm = smem;   // [FWD_THREADS] thread maxima of z (aliases the histogram, not live yet)
+    float lmax = -INFINITY;
+    const bool vec = (V & 3) == 0 && ((size_t)lg & 15) == 0;
+    if (vec) {
+      const float4* lg4 = reinterpret_cast<const float4*>(lg);
+#pragma unroll 8
+      for (int i = tid; i < V / 4; i += FWD_THREADS) {
+        const float4 v = lg4[i];
+        lmax = fmaxf(fmaxf(lmax, fmaxf(v.x, v.y)), fmaxf(v.z, v.w));
+      }
+    } else {
+      for (int i = tid; i < V; i += FWD_THREADS) lmax = fmaxf(lmax, lg[i]);
+    }
+    const float zmax = __fdiv_rn(lmax, temp);
+    s_tm[tid] = zmax;
+    if (tid == 0) s_ncand = 0;
+    __syncthreads();
+    int rank = 0;
+    for (int j = 0; j < FWD_THREADS; ++j) {
+      const float zj = s_tm[j];
+      rank += (zj > zmax) || (zj == zmax && j < tid);
+    }
+    __syncthreads();
+    if (rank == k - 1) s_tm[0] = zmax;
+    __syncthreads();
+    const float tau = s_tm[0];
+    __syncthreads();
+    if (tau > -INFINITY) {
+      // cheap conservative test on the logit first, the exact one on z for the survivors
+      const float x = tau * temp;
+      const float thr_l = x - fabsf(x) * 9.5367431640625e-7f - 1e-30f;
+      auto consider = [&](float v, int i) {
+        if (v >= thr_l) {
+          const float z = __fdiv_rn(v, temp);
+          if (z >= tau) {
+            const int p = atomicAdd(&s_ncand, 1);
+            if (p < CAND_MAX) { s_cz[p] = z; s_ci[p] = i; }
+          }
+        }
+      };
+      if (vec) {
+        const float4* lg4 = reinterpret_cast<const float4*>(lg);
+#pragma unroll 8
+        for (int i = tid; i < V / 4; i += FWD_THREADS) {
+          const float4 v = lg4[i];
+          if (fmaxf(fmaxf(v.x, v.y), fmaxf(v.z, v.w)) >= thr_l) {
+            consider(v.x, 4 * i); consider(v.y, 4 * i + 1); consider(v.z, 4 * i + 2); consider(v.w, 4 * i + 3);
+          }
+        }
+      } else {
+        for (int i = tid; i < V; i += FWD_THREADS) consider(lg[i], i);
+      }
+    }
+    __syncthreads();
+  }
+  const bool fast_ok = s_ncand >= k && s_ncand <= CAND_MAX;
+  __syncthreads();
+  if (!fast_ok) {
+  // Fallback (huge plateaus of equal values, or fewer than k finite thread maxima):
   // radix select over the composite key (z key, ~index): unique keys, so ties in z
   // break towards the lower index and the k-th key is exact.  Refine 8 bits at a time
   // until the set {key >= prefix} (>= k elements by construction) fits the sort buffer.
@@ -550,6 +614,7 @@ static __device__ int sample_row(const float* lg, int V, int top_k, float temp, 
     }
   }
   __syncthreads();
+  }  // fallback
   const int nc = min(s_ncand, CAND_MAX);
   // rank every candidate by (z desc, index asc); the k best land at their rank
   for (int a = tid; a < nc; a += FWD_THREADS) {

@@ -200,42 +200,91 @@ struct TcMaps {
 };
 
 // ---- the GEMM phase -----------------------------------------------------------------------------
+// Shape of one GEMM's pipeline for the current step; every role derives the same numbers.
+struct TcGeom {
+  int kblocks, ntiles, passes, box_id, box_rows, KPS, S;
+  uint32_t b_bytes, stage_bytes;
+  long long u0, u1;
+};
+__device__ __forceinline__ TcGeom tc_geom(const DevCtx& c, int T, int N, int K) {
+  TcGeom g;
+  g.kblocks = K / 64;
+  g.ntiles = (N + 127) / 128;
+  g.passes = (T + 255) / 256;
+  g.box_id = TC_BOXES - 1;
+  if (g.passes == 1) {
+    g.box_id = 0;
+    while ((16 << g.box_id) < T) ++g.box_id;
+  }
+  g.box_rows = 16 << g.box_id;
+  // A stage holds one k-block, or two when the token tile is small and the weights are stored as
+  // contiguous tiles (then one bulk copy brings 32 KiB): fewer, larger copies per producer step.
+  g.KPS = (c.w_streaming && g.box_rows <= 128) ? 2 : 1;
+  g.b_bytes = (uint32_t)g.box_rows * 128u;
+  g.stage_bytes = (uint32_t)g.KPS * (TC_A_BYTES + g.b_bytes);
+  g.S = TC_TILE_BUDGET / (int)g.stage_bytes;
+  if (g.S > TC_MAX_STAGES) g.S = TC_MAX_STAGES;
+  const long long total = (long long)g.passes * g.ntiles * g.kblocks;
+  g.u0 = total * blockIdx.x / gridDim.x;
+  g.u1 = total * (blockIdx.x + 1) / gridDim.x;
+  return g;
+}
+// tiles need 1024-byte alignment for the 128-byte swizzle
+__device__ __forceinline__ char* tc_tiles(float* smem_f) {
+  const uint32_t raw = smem_u32(smem_f);
+  return reinterpret_cast<char*>(smem_f) + (((raw + 1023u) & ~1023u) - raw);
+}
+
+// Weight producer (one thread): stream the weight tiles of this CTA's range through the ring.
+__device__ __forceinline__ void tc_produce_weights(const DevCtx& c, const void* w, int which, int layer, const TcGeom& g,
+                                                   char* tiles, TcState& tc) {
+  const TcMaps* maps = reinterpret_cast<const TcMaps*>(c.tc_maps);
+  const CUtensorMap* map_a = &maps->w[which];
+  const int row_a0 = which == GEMM_LMHEAD ? 0 : layer * (g.ntiles * 128);
+  volatile int* dead = &g_tc.dead;
+  long long u = g.u0;
+  int stage = 0;
+  while (u < g.u1) {
+    const long long seg_end = min(g.u1, (u / g.kblocks + 1) * (long long)g.kblocks);
+    const int nk = (int)min((long long)g.KPS, seg_end - u);
+    const int kb = (int)(u % g.kblocks);
+    const int nt = (int)((u / g.kblocks) % g.ntiles);
+    // the n-th fill of a stage waits for its (n-1)-th release
+    if (!mbar_wait(c, &g_tc.empty[stage], ((tc.fill_bits >> stage) & 1u) ^ 1u, dead)) break;
+    tc.fill_bits ^= 1u << stage;
+    char* sa = tiles + (size_t)stage * g.stage_bytes;
+    mbar_expect_tx(&g_tc.full[stage], (uint32_t)nk * TC_A_BYTES);
+    if (c.w_streaming) {  // contiguous tiles, already in the shared-memory operand image
+      tma_bulk_load(sa, reinterpret_cast<const char*>(w) + ((size_t)nt * g.kblocks + kb) * TC_A_BYTES,
+                    (uint32_t)nk * TC_A_BYTES, &g_tc.full[stage]);
+    } else {
+      tma_load_2d(sa, map_a, kb * 64, row_a0 + nt * 128, &g_tc.full[stage]);
+    }
+    u += nk;
+    if (++stage == g.S) stage = 0;
+  }
+}
+
 static __device__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int which, int layer, float* smem_f, TcState& tc) {
   const int T = a.M, N = a.N, K = a.K;
   if (T <= 0) return;  // uniform over the grid
   const TcMaps* maps = reinterpret_cast<const TcMaps*>(c.tc_maps);
-  const int kblocks = K / 64;
-  const int ntiles = (N + 127) / 128;
-  const int passes = (T + 255) / 256;
-  int box_id = TC_BOXES - 1;
-  if (passes == 1) {
-    box_id = 0;
-    while ((16 << box_id) < T) ++box_id;
-  }
-  const int box_rows = 16 << box_id;
+  const TcGeom g = tc_geom(c, T, N, K);
+  const int kblocks = g.kblocks, ntiles = g.ntiles, KPS = g.KPS, S = g.S;
+  const uint32_t b_bytes = g.b_bytes, stage_bytes = g.stage_bytes;
   const int act_id = which == GEMM_O ? ACT_ATTN : which == GEMM_DOWN ? ACT_ACT : which == GEMM_LMHEAD ? ACT_XS : ACT_XN;
-  const CUtensorMap* map_a = &maps->w[which];
-  const CUtensorMap* map_b = &maps->act[act_id][box_id];
-  const int row_a0 = which == GEMM_LMHEAD ? 0 : layer * N;
-  // A stage holds one k-block, or two when the token tile is small and the weights are stored as
-  // contiguous tiles (then one bulk copy brings 32 KiB): fewer, larger copies per producer step.
-  const int KPS = (c.w_streaming && box_rows <= 128) ? 2 : 1;
-  const uint32_t b_bytes = (uint32_t)box_rows * 128u;
-  const uint32_t stage_bytes = (uint32_t)KPS * (TC_A_BYTES + b_bytes);
-  int S = TC_TILE_BUDGET / (int)stage_bytes;
-  if (S > TC_MAX_STAGES) S = TC_MAX_STAGES;
-  // tiles need 1024-byte alignment for the 128-byte swizzle
-  const uint32_t raw = smem_u32(smem_f);
-  char* tiles = reinterpret_cast<char*>(smem_f) + (((raw + 1023u) & ~1023u) - raw);
-
-  const long long total = (long long)passes * ntiles * kblocks;
-  const long long u0 = total * blockIdx.x / gridDim.x, u1 = total * (blockIdx.x + 1) / gridDim.x;
+  const CUtensorMap* map_b = &maps->act[act_id][g.box_id];
+  char* tiles = tc_tiles(smem_f);
+  const long long u0 = g.u0, u1 = g.u1;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile int* dead = &g_tc.dead;
 
-  if (warp == 0 || warp == 2) {
-    // two producer threads: warp 0 streams the weight tiles, warp 2 the token tiles; both walk the
-    // same sequence of stages (nk k-blocks of one segment each)
+  if (warp == 0) {
+    if (lane == 0) {
+      tc_produce_weights(c, a.w, which, layer, g, tiles, tc);
+    }
+  } else if (warp == 2) {
+    // token-tile producer: walks the same sequence of stages (nk k-blocks of one segment each)
     if (lane == 0) {
       int stage = 0;
       long long u = u0;
@@ -243,25 +292,13 @@ static __device__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int whi
         const long long seg_end = min(u1, (u / kblocks + 1) * (long long)kblocks);
         const int nk = (int)min((long long)KPS, seg_end - u);
         const int kb = (int)(u % kblocks);
-        const int nt = (int)((u / kblocks) % ntiles);
         const int pass = (int)(u / ((long long)kblocks * ntiles));
-        // the n-th fill of a stage waits for its (n-1)-th release
         if (!mbar_wait(c, &g_tc.empty[stage], ((tc.fill_bits >> stage) & 1u) ^ 1u, dead)) break;
         tc.fill_bits ^= 1u << stage;
         char* sa = tiles + (size_t)stage * stage_bytes;
-        if (warp == 0) {
-          mbar_expect_tx(&g_tc.full[stage], (uint32_t)nk * TC_A_BYTES);
-          if (c.w_streaming) {  // contiguous tiles, already in the shared-memory operand image
-            tma_bulk_load(sa, reinterpret_cast<const char*>(a.w) + ((size_t)nt * kblocks + kb) * TC_A_BYTES,
-                          (uint32_t)nk * TC_A_BYTES, &g_tc.full[stage]);
-          } else {
-            tma_load_2d(sa, map_a, kb * 64, row_a0 + nt * 128, &g_tc.full[stage]);
-          }
-        } else {
-          mbar_expect_tx(&g_tc.full[stage], (uint32_t)nk * b_bytes);
-          for (int j = 0; j < nk; ++j)
-            tma_load_2d(sa + KPS * TC_A_BYTES + j * b_bytes, map_b, (kb + j) * 64, pass * 256, &g_tc.full[stage]);
-        }
+        mbar_expect_tx(&g_tc.full[stage], (uint32_t)nk * b_bytes);
+        for (int j = 0; j < nk; ++j)
+          tma_load_2d(sa + KPS * TC_A_BYTES + j * b_bytes, map_b, (kb + j) * 64, pass * 256, &g_tc.full[stage]);
         u += nk;
         if (++stage == S) stage = 0;
       }

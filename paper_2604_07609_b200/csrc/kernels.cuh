@@ -26,7 +26,9 @@ __device__ __forceinline__ void run_phase(const DevCtx& c, int phase, int layer,
   const int T = c.ss->cur_T;
   const size_t esz = sizeof(WT);
   switch (phase) {
-    case PH_NORM1: phase_norm<WT>(c, layer, 0); break;
+    case PH_NORM1:
+      phase_norm<WT>(c, layer, 0);
+      break;
     case PH_QKV: {
       GemmArgs a{c.xn, c.w_base + c.w_off[1] + (size_t)layer * c.qkv_dim * c.d * esz, c.qkv, T, c.qkv_dim, c.d,
                  c.qkv_dim, 0};
@@ -36,22 +38,29 @@ __device__ __forceinline__ void run_phase(const DevCtx& c, int phase, int layer,
     case PH_ATTN:
       if constexpr (sizeof(WT) == 2) phase_attention_bf16<HD, NREP>(c, layer, smem, as);
       else phase_attention<WT, HD, NREP>(c, layer, smem);
+
       break;
     case PH_O: {
       GemmArgs a{c.attn, c.w_base + c.w_off[2] + (size_t)layer * c.d * c.q_dim * esz, c.h, T, c.d, c.q_dim, c.d, 1};
       gemm_dispatch<WT>(c, a, GEMM_O, layer, smem, tc);
     } break;
-    case PH_NORM2: phase_norm<WT>(c, layer, 1); break;
+    case PH_NORM2:
+      phase_norm<WT>(c, layer, 1);
+      break;
     case PH_GU: {
       GemmArgs a{c.xn, c.w_base + c.w_off[3] + (size_t)layer * 2 * c.F * c.d * esz, c.gu, T, 2 * c.F, c.d, 2 * c.F, 0};
       gemm_dispatch<WT>(c, a, GEMM_GU, layer, smem, tc);
     } break;
-    case PH_SILU: phase_silu_mul<WT>(c); break;
+    case PH_SILU:
+      phase_silu_mul<WT>(c);
+      break;
     case PH_DOWN: {
       GemmArgs a{c.act, c.w_base + c.w_off[4] + (size_t)layer * c.d * c.F * esz, c.h, T, c.d, c.F, c.d, 1};
       gemm_dispatch<WT>(c, a, GEMM_DOWN, layer, smem, tc);
     } break;
-    case PH_FNORM: phase_final_norm<WT>(c); break;
+    case PH_FNORM:
+      phase_final_norm<WT>(c);
+      break;
     case PH_LMHEAD: {
       GemmArgs a{c.xs, c.w_base + c.w_off[9], c.logits, c.ss->cur_rows, c.V, c.d, c.V, 0};
       gemm_dispatch<WT>(c, a, GEMM_LMHEAD, 0, smem, tc);
