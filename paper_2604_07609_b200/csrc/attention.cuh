@@ -2,14 +2,13 @@
 // KV cache with decode attention and context attention inside the step).
 //
 // Two kinds of work share the phase:
-//   * decode rows (one query token per request): a bandwidth-bound CUDA-core kernel.  All
-//     (row, kv head, KV block) tiles of the step form one flat sequence that is cut into
-//     sub-ranges; warps fetch sub-ranges from a counter, stream the 16-key K and V tiles
-//     (contiguous in the pool) into a private shared-memory ring with bulk async copies
-//     (TMA engine, mbarrier completion), and keep an online softmax per (row, kv head)
-//     unit.  The query heads of a GQA group share every K/V load.  A unit cut by a
-//     sub-range boundary leaves partial (m, l, acc) records; whoever finishes the last part
-//     merges them in a fixed order.
+//   * decode rows (one query token per request): bandwidth-bound.  All (row, kv head, KV block)
+//     tiles of the step form one flat sequence that is cut into sub-ranges; warps fetch
+//     sub-ranges from a counter, stream the 16-key K and V tiles (contiguous in the pool) into
+//     a private shared-memory ring with TMA tile copies (mbarrier completion), and keep an
+//     online softmax per (row, kv head) unit.  The query heads of a GQA group share every K/V
+//     load.  A unit cut by a sub-range boundary leaves partial (m, l, acc) records; whoever
+//     finishes the last part merges them in a fixed order.
 //   * prefill-chunk rows (several query tokens of one request): a dense contraction, so it
 //     runs on tensor cores (mma.sync m16n8k16, flash-attention style tiling): one CTA per
 //     (request, block of query rows, kv head), 64-key K/V tiles through a double-buffered
@@ -21,6 +20,7 @@ namespace blink {
 
 constexpr int ATT_NS = 3;  // ring stages per warp (decode path)
 constexpr int ATT_WARPS = FWD_THREADS / 32;
+constexpr bool ATT_SNAP = false;  // keep units of at most 2 S tiles whole (see dec_bound)
 
 struct AttShared {
   uint64_t bar[ATT_WARPS][ATT_NS];
@@ -56,26 +56,6 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t by
                : "memory");
 }
 
-// packed fp32x2 arithmetic (two lanes of one 64-bit register)
-__device__ __forceinline__ unsigned long long ffma2(unsigned long long a, unsigned long long b, unsigned long long c) {
-  unsigned long long d;
-  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-  return d;
-}
-__device__ __forceinline__ unsigned long long fmul2(unsigned long long a, unsigned long long b) {
-  unsigned long long d;
-  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-  return d;
-}
-__device__ __forceinline__ unsigned long long pack2(float lo, float hi) {
-  return ((unsigned long long)__float_as_uint(hi) << 32) | (unsigned long long)__float_as_uint(lo);
-}
-__device__ __forceinline__ float lo2(unsigned long long v) { return __uint_as_float((uint32_t)v); }
-__device__ __forceinline__ float hi2(unsigned long long v) { return __uint_as_float((uint32_t)(v >> 32)); }
-// two bf16 in one word -> the same two values as fp32x2 (low half first)
-__device__ __forceinline__ unsigned long long bf2_to_f2(uint32_t w) {
-  return ((unsigned long long)(w & 0xffff0000u) << 32) | (unsigned long long)(w << 16);
-}
 __device__ __forceinline__ float fast_ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -85,30 +65,14 @@ __device__ __forceinline__ uint32_t pack_bf2(float lo, float hi) {
   const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<const uint32_t*>(&v);
 }
-__device__ __forceinline__ float ldcg_f(const float* p) {
-  float v;
-  asm volatile("ld.global.cg.f32 %0, [%1];" : "=f"(v) : "l"(p) : "memory");
-  return v;
-}
-
-// One halving step of a butterfly reduction: the lanes of a pair (xor MASK) hold N values
-// each; afterwards each holds N/2 sums (the lane with the MASK bit set keeps the upper half).
-template <int N, int MASK>
-__device__ __forceinline__ void halve_step(float* v, bool upper) {
-#pragma unroll
-  for (int i = 0; i < N / 2; ++i) {
-    const float send = upper ? v[i] : v[i + N / 2];
-    const float keep = upper ? v[i + N / 2] : v[i];
-    v[i] = keep + __shfl_xor_sync(0xffffffffu, send, MASK);
-  }
-}
-template <int N, int MASK>
-__device__ __forceinline__ void reduce_step(float* v, bool upper) {
-  if constexpr (N >= 2) {
-    halve_step<N, MASK>(v, upper);
-  } else {
-    v[0] += __shfl_xor_sync(0xffffffffu, v[0], MASK);
-  }
+// one TMA tile copy from a rank-5 tensor map
+__device__ __forceinline__ void tma_load_5d(void* smem_dst, const CUtensorMap* map, int c0, int c1, int c2, int c3, int c4,
+                                            uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];" ::"r"(
+          smem_u32(smem_dst)),
+      "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(smem_u32(bar))
+      : "memory");
 }
 
 // flat tile sequence of the decode rows: unit (d, g) owns tiles [Hkv*pre[d] + g*nkb, +nkb)
@@ -142,66 +106,103 @@ __device__ __forceinline__ void dec_advance(DecCursor& cur, int n_dec, int Hkv) 
   }
 }
 
+// Sub-range j of the flat tile sequence is [dec_bound(j S), dec_bound((j + 1) S)): a boundary that
+// would cut a unit of at most 2 S tiles moves to the end of that unit, so only long units are
+// ever split (and leave partial records); short ones stay with the sub-range they start in.
+__device__ __forceinline__ int dec_bound(int x, int S, int TT, int n_dec, int Hkv) {
+  if (x >= TT) return TT;
+  DecCursor t;
+  dec_seek(t, x, x, n_dec, Hkv);
+  return (ATT_SNAP && t.kb > 0 && t.nkb <= 2 * S) ? x + (t.nkb - t.kb) : x;
+}
+
+// ---- tensor-core and matrix-load wrappers ---------------------------------------------------------
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16_16816(float* d, const uint32_t* a, uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
 // ---- decode rows: warp-level streaming kernel -------------------------------------------------
-// Lane mapping inside a warp: every lane owns one 16-byte chunk (8 dims) of the head vector,
-// LPK = head_dim / 8 lanes cover a key, so the warp reads KG = 32 / LPK keys per pass as one
-// contiguous run of shared memory; pass p handles key KG * p + kg of the 16-key tile.
+// One warp owns a (row, kv head) unit at a time and walks its 16-key tiles.  A tile's K and V
+// ([16 keys][head_dim] each, contiguous in the pool) arrive through one TMA tile copy with the
+// 128-byte swizzle, so both can be read with ldmatrix (at most two-way bank conflicts).  The two small contractions
+// of a tile (scores = Q K^T for the query heads of the group, out += P V) run as m16n8k16 MMAs
+// with the group's heads in the first rows of the 16-row operand: written with CUDA-core FMAs
+// the same loop needs about 800 instructions per tile and the SM runs out of issue slots at
+// about half the HBM bandwidth; this form needs about 130.  Softmax statistics stay in fp32
+// registers and are combined with quad shuffles.
 template <int HD, int NREP>
-__device__ __forceinline__ void attn_decode_stream(const DevCtx& c, int layer, char* ring, float* sc, AttState& as) {
-  constexpr int LPK = HD / 8;        // lanes per key
-  constexpr int KG = 32 / LPK;       // keys per pass
-  constexpr int NP = 16 / KG;        // passes per tile
+__device__ __noinline__ void attn_decode_stream(const DevCtx& c, int layer, char* ring, AttState& as) {
   constexpr int RB = HD * 2;         // bytes per key row
+  constexpr int NBOX = HD / 64;      // 64-column boxes per tile row (128-byte swizzle span)
   constexpr int TILE = 16 * RB;      // bytes of one K (or V) tile of a (block, kv head)
   constexpr int STAGE = 2 * TILE;
-  constexpr int NV = NP * NREP;      // (pass, head) partial scores per lane per tile
-  constexpr int OC = NV >= LPK ? NV / LPK : 1;
-  constexpr int NA = NREP * 8;       // accumulator values per lane
-  constexpr int OWN = NA / KG;       // ... and after the sum over the key groups
+  constexpr int KS = HD / 16;        // k-steps of Q K^T
   constexpr int REC = NREP * HD + ((2 * NREP + 3) & ~3);  // floats per partial record, 16-byte multiple
   constexpr unsigned FULL = 0xffffffffu;
+  static_assert(NREP <= 8, "the group's heads must fit the first eight operand rows");
   const SchedState* ss = c.ss;
   const int n_dec = ss->cur_ndec, TT = ss->cur_TT, S = ss->cur_S;
   if (TT <= 0) return;
   const int n_sub = (TT + S - 1) / S;
   const int Hkv = c.Hkv;
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-  const int kg = lane / LPK, dc = lane % LPK;
+  const int gq = lane >> 2, tq = lane & 3;   // operand row (= head of the group) and column pair
+  const bool live = gq < NREP;
   uint64_t* bars = g_att.bar[w];
   volatile int* dead = &g_att.dead;
   int* ctr = c.att_ctr + layer;
+  const CUtensorMap* kv_map = reinterpret_cast<const CUtensorMap*>(c.kv_map);
   const __nv_bfloat16* qb = reinterpret_cast<const __nv_bfloat16*>(c.qb);
   __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(c.attn);
-  const char* kv_base = reinterpret_cast<const char*>(c.kv_base);
-  const size_t kv_stride = (size_t)c.n_blocks * Hkv * TILE;  // bytes between the K and V planes of a layer
-  const char* k_plane = kv_base + (size_t)layer * 2 * kv_stride;
   const float qscale = c.attn_scale * 1.4426950408889634f;
+  const uint32_t ring_s = smem_u32(ring);
 
   int n_issued = 0, n_consumed = 0, p_k = 0, c_k = 0;
-  bool p_done = false;
+  bool p_done = false, first_fetch = true;
   DecCursor pc{0, 0, 0, 0, 0, 1}, cc{0, 0, 0, 0, 0, 1};
   int p_blk = 0, p_blk_d = -1, p_blk_base = -1;
   int sub_start = 0, sub_id = 0;
   bool in_unit = false;
 
-  unsigned long long q2[NREP][4];
-  unsigned long long acc2[NREP][4];
-  float m[NREP], l[NREP];
+  uint32_t qf[KS][2];     // operand rows 8..15 are zero, so only a0 and a2 of each k-step are kept
+  float o[HD / 8][2];     // out rows 0..7 (c0, c1 of each n-tile)
+  float m = -INFINITY, l = 0.f;
 
   while (true) {
     // ---- producer: keep up to ATT_NS tiles in flight ----
     while (!p_done && n_issued - n_consumed < ATT_NS) {
       if (pc.f == pc.f_end) {
-        int id = blockIdx.x * ATT_WARPS + w;   // first sub-range: the warp's own index
-        if (p_k > 0) {
-          if (lane == 0) id = atomicAdd(ctr, 1);
-          id = __shfl_sync(FULL, id, 0);
+        // next non-empty sub-range: the warp's own index first, then whatever the counter hands out
+        int id = 0, b0 = 0, b1 = 0;
+        while (true) {
+          if (first_fetch) {
+            id = blockIdx.x * ATT_WARPS + w;
+            first_fetch = false;
+          } else {
+            if (lane == 0) id = atomicAdd(ctr, 1);
+            id = __shfl_sync(FULL, id, 0);
+          }
+          if (id >= n_sub) { p_done = true; break; }
+          b0 = dec_bound(id * S, S, TT, n_dec, Hkv);
+          b1 = dec_bound(id * S + S, S, TT, n_dec, Hkv);
+          if (b0 < b1) break;
         }
+        if (p_done) break;
         if (lane == 0) g_att.ids[w][p_k & 7] = id;
         __syncwarp();
         p_k += 1;
-        if (id >= n_sub) { p_done = true; break; }
-        dec_seek(pc, id * S, min(TT, id * S + S), n_dec, Hkv);
+        dec_seek(pc, b0, b1, n_dec, Hkv);
       }
       if (pc.d != p_blk_d || (pc.kb & ~31) != p_blk_base) {
         p_blk_d = pc.d;
@@ -212,10 +213,9 @@ __device__ __forceinline__ void attn_decode_stream(const DevCtx& c, int layer, c
       const int blk = __shfl_sync(FULL, p_blk, pc.kb & 31);
       if (lane == 0) {
         const int s = n_issued % ATT_NS;
-        const char* ksrc = k_plane + ((size_t)blk * Hkv + pc.g) * TILE;
+        // one copy brings the K tile and the V tile: box {64 dims, NBOX halves, 16 keys, K and V, this layer}
         mbar_expect_tx(&bars[s], STAGE);
-        bulk_g2s(ring + s * STAGE, ksrc, TILE, &bars[s]);
-        bulk_g2s(ring + s * STAGE + TILE, ksrc + kv_stride, TILE, &bars[s]);
+        tma_load_5d(ring + s * STAGE, kv_map, 0, 0, (blk * Hkv + pc.g) * 16, 0, layer, &bars[s]);
       }
       dec_advance(pc, n_dec, Hkv);
       n_issued += 1;
@@ -223,184 +223,133 @@ __device__ __forceinline__ void attn_decode_stream(const DevCtx& c, int layer, c
     if (n_consumed == n_issued) break;
 
     // ---- consumer: one tile ----
-    if (cc.f == cc.f_end) {
+    while (cc.f == cc.f_end) {   // next non-empty sub-range (the producer already issued a tile of it)
       sub_id = g_att.ids[w][c_k & 7];
       c_k += 1;
       sub_start = sub_id * S;
-      dec_seek(cc, sub_start, min(TT, sub_start + S), n_dec, Hkv);
+      dec_seek(cc, dec_bound(sub_start, S, TT, n_dec, Hkv), dec_bound(sub_start + S, S, TT, n_dec, Hkv), n_dec, Hkv);
       in_unit = false;
     }
     const int t_row = g_att_row[cc.d];
     const int n_ctx = g_att_nctx[cc.d];
     if (!in_unit) {  // a unit (or this sub-range's part of it) starts here
       in_unit = true;
+      m = -INFINITY;
+      l = 0.f;
+      const __nv_bfloat16* qrow = qb + (size_t)t_row * c.q_dim + (size_t)(cc.g * NREP + (live ? gq : 0)) * HD;
 #pragma unroll
-      for (int h = 0; h < NREP; ++h) {
-        m[h] = -INFINITY;
-        l[h] = 0.f;
-        const __nv_bfloat16* qrow = qb + (size_t)t_row * c.q_dim + (size_t)(cc.g * NREP + h) * HD;
-        const uint4 qr = *reinterpret_cast<const uint4*>(qrow + dc * 8);
-        const uint32_t qw[4] = {qr.x, qr.y, qr.z, qr.w};
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const unsigned long long f2 = bf2_to_f2(qw[i]);
-          q2[h][i] = pack2(lo2(f2) * qscale, hi2(f2) * qscale);
-          acc2[h][i] = 0ull;
-        }
+      for (int ks = 0; ks < KS; ++ks) {
+        qf[ks][0] = live ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 2 * tq) : 0u;
+        qf[ks][1] = live ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 8 + 2 * tq) : 0u;
       }
+#pragma unroll
+      for (int i = 0; i < HD / 8; ++i) { o[i][0] = 0.f; o[i][1] = 0.f; }
     }
     const int s = n_consumed % ATT_NS;
     if (!__all_sync(FULL, mbar_wait(c, &bars[s], (as.par >> s) & 1u, dead))) break;  // uniform exit
     as.par ^= 1u << s;
-    const char* kt = ring + s * STAGE;
-    const char* vt = kt + TILE;
+    const uint32_t kt = ring_s + s * STAGE, vt = kt + TILE;
     const int key0 = cc.kb * 16;
-
-    // scores: partial dot products over this lane's 8 dims
-    float part[NV];
+    const int n_valid = min(16, n_ctx - key0);   // >= 1
+    if (n_valid < 16) {
+      // the tail of the last block holds whatever the pool held: clear those V rows (0 x NaN)
+      uint4* vg = reinterpret_cast<uint4*>(ring + s * STAGE + TILE + n_valid * RB);
+      for (int i = lane; i < (16 - n_valid) * RB / 16; i += 32) vg[i] = make_uint4(0u, 0u, 0u, 0u);
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // before TMA refills this stage
+      __syncwarp();
+    }
+    // The matrix loads and MMAs below are issued in program order, so all loads of an operand are
+    // issued before the MMAs that use them, and V is fetched before the softmax arithmetic.
+    uint32_t kf[KS][4];
 #pragma unroll
-    for (int p = 0; p < NP; ++p) {
-      const uint4 kr = *reinterpret_cast<const uint4*>(kt + (KG * p + kg) * RB + dc * 16);
-      const uint32_t kw[4] = {kr.x, kr.y, kr.z, kr.w};
-      unsigned long long a2[NREP];
+    for (int ks = 0; ks < KS; ++ks) {
+      const int key = (lane & 7) + ((lane >> 4) & 1) * 8;
+      const int ck = ks * 2 + ((lane >> 3) & 1);
+      const int line = key * NBOX + (ck >> 3);   // 128-byte line of the tile; chunks are swizzled with the line index
+      ldsm_x4(kt + line * 128 + (((ck & 7) ^ (line & 7)) << 4), kf[ks][0], kf[ks][1], kf[ks][2], kf[ks][3]);
+    }
+    uint32_t vf[HD / 16][4];
 #pragma unroll
-      for (int h = 0; h < NREP; ++h) a2[h] = 0ull;
+    for (int dp = 0; dp < HD / 16; ++dp) {
+      const int key = (lane & 7) + ((lane >> 3) & 1) * 8;
+      const int ck = dp * 2 + (lane >> 4);
+      const int line = key * NBOX + (ck >> 3);
+      ldsm_x4_t(vt + line * 128 + (((ck & 7) ^ (line & 7)) << 4), vf[dp][0], vf[dp][1], vf[dp][2], vf[dp][3]);
+    }
+    // scores of the group's heads against the 16 keys: two n-tiles of 8 keys, two accumulators
+    // each (even and odd k-steps) to halve the dependent chain
+    float sacc[4][4];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const unsigned long long k2 = bf2_to_f2(kw[i]);
+    for (int i = 0; i < 4; ++i) { sacc[i][0] = sacc[i][1] = sacc[i][2] = sacc[i][3] = 0.f; }
 #pragma unroll
-        for (int h = 0; h < NREP; ++h) a2[h] = ffma2(q2[h][i], k2, a2[h]);
+    for (int ks = 0; ks < KS; ++ks) {
+      const uint32_t a[4] = {qf[ks][0], 0u, qf[ks][1], 0u};
+      mma_bf16_16816(sacc[(ks & 1) * 2], a, kf[ks][0], kf[ks][1]);
+      mma_bf16_16816(sacc[(ks & 1) * 2 + 1], a, kf[ks][2], kf[ks][3]);
+    }
+    sacc[0][0] += sacc[2][0]; sacc[0][1] += sacc[2][1];
+    sacc[1][0] += sacc[3][0]; sacc[1][1] += sacc[3][1];
+    // online softmax of operand row gq over this lane's four keys (2 tq, 2 tq + 1, 8 + 2 tq, 9 + 2 tq)
+    float sv[4];
+#pragma unroll
+    for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const int key = nt * 8 + 2 * tq + e;
+        sv[nt * 2 + e] = key < n_valid ? sacc[nt][e] * qscale : -INFINITY;
       }
+    float mx = fmaxf(fmaxf(sv[0], sv[1]), fmaxf(sv[2], sv[3]));
+    mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, 1));
+    mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, 2));
+    const float mn = fmaxf(m, mx);          // finite: key 0 of the tile is always valid
+    if (__any_sync(FULL, mn > m)) {
+      const float corr = fast_ex2(m - mn);
+      l *= corr;
 #pragma unroll
-      for (int h = 0; h < NREP; ++h) part[p * NREP + h] = lo2(a2[h]) + hi2(a2[h]);
+      for (int i = 0; i < HD / 8; ++i) { o[i][0] *= corr; o[i][1] *= corr; }
     }
-    // reduce over the LPK lanes of a key; each lane ends up owning OC complete scores
-    if constexpr (LPK == 16) {
-      reduce_step<NV, 8>(part, (dc & 8) != 0);
-      reduce_step<NV / 2, 4>(part, (dc & 4) != 0);
-      reduce_step<NV / 4, 2>(part, (dc & 2) != 0);
-      reduce_step<NV / 8, 1>(part, (dc & 1) != 0);
-    } else {
-      reduce_step<NV, 4>(part, (dc & 4) != 0);
-      reduce_step<NV / 2, 2>(part, (dc & 2) != 0);
-      reduce_step<NV / 4, 1>(part, (dc & 1) != 0);
+    m = mn;
+    const float p0 = fast_ex2(sv[0] - mn), p1 = fast_ex2(sv[1] - mn), p2 = fast_ex2(sv[2] - mn), p3 = fast_ex2(sv[3] - mn);
+    l += (p0 + p1) + (p2 + p3);
+    const uint32_t pa[4] = {pack_bf2(p0, p1), 0u, pack_bf2(p2, p3), 0u};
+    // out += P V: n-tiles of 8 dims, one k-step of 16 keys
+#pragma unroll
+    for (int dp = 0; dp < HD / 16; ++dp) {
+      float d0[4] = {o[2 * dp][0], o[2 * dp][1], 0.f, 0.f};
+      float d1[4] = {o[2 * dp + 1][0], o[2 * dp + 1][1], 0.f, 0.f};
+      mma_bf16_16816(d0, pa, vf[dp][0], vf[dp][1]);
+      mma_bf16_16816(d1, pa, vf[dp][2], vf[dp][3]);
+      o[2 * dp][0] = d0[0]; o[2 * dp][1] = d0[1];
+      o[2 * dp + 1][0] = d1[0]; o[2 * dp + 1][1] = d1[1];
     }
-    {
-      const int v_base = NV >= LPK ? dc * OC : dc / (LPK / NV);
-#pragma unroll
-      for (int o = 0; o < OC; ++o) {
-        const int v = v_base + o;
-        const int p = v / NREP, h = v % NREP;
-        const int key = KG * p + kg;
-        sc[key * NREP + h] = (key0 + key < n_ctx) ? part[o] : -INFINITY;
-      }
-    }
-    __syncwarp();
-    float sp[NP][NREP];
-    float tmax[NREP];
-#pragma unroll
-    for (int h = 0; h < NREP; ++h) tmax[h] = -INFINITY;
-#pragma unroll
-    for (int p = 0; p < NP; ++p)
-#pragma unroll
-      for (int h = 0; h < NREP; ++h) {
-        sp[p][h] = sc[(KG * p + kg) * NREP + h];
-        tmax[h] = fmaxf(tmax[h], sp[p][h]);
-      }
-    bool changed = false;
-#pragma unroll
-    for (int h = 0; h < NREP; ++h) {
-      tmax[h] = fmaxf(tmax[h], __shfl_xor_sync(FULL, tmax[h], 16));
-      if constexpr (KG == 4) tmax[h] = fmaxf(tmax[h], __shfl_xor_sync(FULL, tmax[h], 8));
-      changed |= tmax[h] > m[h];
-    }
-    if (changed) {  // warp-uniform: every lane holds the same m and tmax
-#pragma unroll
-      for (int h = 0; h < NREP; ++h) {
-        const float mn = fmaxf(m[h], tmax[h]);
-        const float corr = fast_ex2(m[h] - mn);
-        m[h] = mn;
-        l[h] *= corr;
-        const unsigned long long c2 = pack2(corr, corr);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) acc2[h][i] = fmul2(acc2[h][i], c2);
-      }
-    }
-    // probabilities and P.V
-#pragma unroll
-    for (int p = 0; p < NP; ++p) {
-      const int key = KG * p + kg;
-      if (key0 + key < n_ctx) {   // keys past the context hold whatever the pool held
-        const uint4 vr = *reinterpret_cast<const uint4*>(vt + key * RB + dc * 16);
-        const uint32_t vw[4] = {vr.x, vr.y, vr.z, vr.w};
-        unsigned long long pp[NREP];
-#pragma unroll
-        for (int h = 0; h < NREP; ++h) {
-          const float pv = fast_ex2(sp[p][h] - m[h]);
-          l[h] += pv;
-          pp[h] = pack2(pv, pv);
-        }
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const unsigned long long v2 = bf2_to_f2(vw[i]);
-#pragma unroll
-          for (int h = 0; h < NREP; ++h) acc2[h][i] = ffma2(pp[h], v2, acc2[h][i]);
-        }
-      }
-    }
-    __syncwarp();  // all reads of this stage and of sc are done before they are refilled
+    __syncwarp();  // all reads of this stage are done before it is refilled
     n_consumed += 1;
 
     const bool unit_ends = (cc.kb == cc.nkb - 1) || (cc.f + 1 == cc.f_end);
     if (unit_ends) {
       in_unit = false;
-      // sum over the key groups: the lane ends up owning OWN accumulator values
-      float a[NA];
-#pragma unroll
-      for (int h = 0; h < NREP; ++h)
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          a[h * 8 + 2 * i] = lo2(acc2[h][i]);
-          a[h * 8 + 2 * i + 1] = hi2(acc2[h][i]);
-        }
-      int a_base;
-      if constexpr (KG == 2) {
-        halve_step<NA, 16>(a, (lane & 16) != 0);
-        a_base = (lane & 16) ? OWN : 0;
-      } else {
-        halve_step<NA, 8>(a, (lane & 8) != 0);
-        halve_step<NA / 2, 16>(a, (lane & 16) != 0);
-        a_base = (((lane >> 3) & 1) * 2 + ((lane >> 4) & 1)) * OWN;
-      }
-#pragma unroll
-      for (int h = 0; h < NREP; ++h) {
-        l[h] += __shfl_xor_sync(FULL, l[h], 16);
-        if constexpr (KG == 4) l[h] += __shfl_xor_sync(FULL, l[h], 8);
-      }
+      float lt = l;
+      lt += __shfl_xor_sync(FULL, lt, 1);
+      lt += __shfl_xor_sync(FULL, lt, 2);
       const int us = Hkv * g_att_pre[cc.d] + cc.g * cc.nkb, ue = us + cc.nkb;
       const int j_first = us / S, j_last = (ue - 1) / S;
-      if (j_first == j_last) {
+      if ((ATT_SNAP && cc.nkb <= 2 * S) || j_first == j_last) {   // the whole unit was handled here
+        if (live) {
+          const float inv = 1.0f / lt;
+          __nv_bfloat16* orow = out + (size_t)t_row * c.q_dim + (size_t)(cc.g * NREP + gq) * HD;
 #pragma unroll
-        for (int o = 0; o < OWN; ++o) {
-          const int ai = a_base + o;
-          const int h = ai >> 3, dim = dc * 8 + (ai & 7);
-          float lh = l[0];
-#pragma unroll
-          for (int hh = 1; hh < NREP; ++hh) lh = (h == hh) ? l[hh] : lh;
-          out[(size_t)t_row * c.q_dim + (size_t)(cc.g * NREP + h) * HD + dim] = __float2bfloat16_rn(a[o] / lh);
+          for (int i = 0; i < HD / 8; ++i)
+            *reinterpret_cast<uint32_t*>(orow + i * 8 + 2 * tq) = pack_bf2(o[i][0] * inv, o[i][1] * inv);
         }
       } else {
         // partial record: [NREP][HD] accumulators, then m[NREP], then l[NREP]
         const int unit = cc.d * Hkv + cc.g;
         float* rec = c.att_part + (size_t)(2 * sub_id + (us <= sub_start ? 0 : 1)) * REC;
+        if (live) {
 #pragma unroll
-        for (int o = 0; o < OWN; ++o) {
-          const int ai = a_base + o;
-          rec[(ai >> 3) * HD + dc * 8 + (ai & 7)] = a[o];
-        }
-        if (lane == 0) {
-#pragma unroll
-          for (int h = 0; h < NREP; ++h) { rec[NREP * HD + h] = m[h]; rec[NREP * HD + NREP + h] = l[h]; }
+          for (int i = 0; i < HD / 8; ++i)
+            *reinterpret_cast<float2*>(rec + gq * HD + i * 8 + 2 * tq) = make_float2(o[i][0], o[i][1]);
+          if (tq == 0) { rec[NREP * HD + gq] = m; rec[NREP * HD + NREP + gq] = lt; }
         }
         __threadfence();
         __syncwarp();
@@ -443,20 +392,6 @@ __device__ __forceinline__ void attn_decode_stream(const DevCtx& c, int layer, c
 }
 
 // ---- prefill-chunk rows: tensor-core tile kernel ---------------------------------------------------
-__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
-}
-__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
-}
-__device__ __forceinline__ void mma_bf16_16816(float* d, const uint32_t* a, uint32_t b0, uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
 }
@@ -466,7 +401,7 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32
 // Shared memory: Q [128][HD] then two stages of K [64][HD], V [64][HD]; 16-byte chunks of a row
 // are XOR-swizzled with the row index so that ldmatrix reads are conflict-free.
 template <int HD, int NREP>
-__device__ __forceinline__ void attn_prefill_tile(const DevCtx& c, int layer, int item, int qblk, int g, char* smem) {
+__device__ __noinline__ void attn_prefill_tile(const DevCtx& c, int layer, int item, int qblk, int g, char* smem) {
   constexpr int QROWS = 128 / NREP;
   constexpr int RB = HD * 2;          // bytes per row
   constexpr int CPR = RB / 16;        // 16-byte chunks per row
@@ -544,14 +479,17 @@ __device__ __forceinline__ void attn_prefill_tile(const DevCtx& c, int layer, in
     for (int i = 0; i < 8; ++i) { sacc[i][0] = sacc[i][1] = sacc[i][2] = sacc[i][3] = 0.f; }
 #pragma unroll
     for (int ks = 0; ks < HD / 16; ++ks) {
+      uint32_t bf[4][4];   // all loads of the k-step first, then its MMAs (both are issued in program order)
 #pragma unroll
       for (int np = 0; np < 4; ++np) {
         const int key = np * 16 + (lane & 7) + (lane >> 4) * 8;
         const int ck = ks * 2 + ((lane >> 3) & 1);
-        uint32_t b0, b1, b2, b3;
-        ldsm_x4(sk + key * RB + ((ck ^ (key & 7)) << 4), b0, b1, b2, b3);
-        mma_bf16_16816(sacc[2 * np], qf[ks], b0, b1);
-        mma_bf16_16816(sacc[2 * np + 1], qf[ks], b2, b3);
+        ldsm_x4(sk + key * RB + ((ck ^ (key & 7)) << 4), bf[np][0], bf[np][1], bf[np][2], bf[np][3]);
+      }
+#pragma unroll
+      for (int np = 0; np < 4; ++np) {
+        mma_bf16_16816(sacc[2 * np], qf[ks], bf[np][0], bf[np][1]);
+        mma_bf16_16816(sacc[2 * np + 1], qf[ks], bf[np][2], bf[np][3]);
       }
     }
     // scale, causal mask, online softmax (rows gq and gq + 8 of the warp's 16)
@@ -591,13 +529,19 @@ __device__ __forceinline__ void attn_prefill_tile(const DevCtx& c, int layer, in
 #pragma unroll
     for (int kk = 0; kk < 4; ++kk) {
 #pragma unroll
-      for (int dp = 0; dp < HD / 16; ++dp) {
-        const int key = kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
-        const int ck = dp * 2 + (lane >> 4);
-        uint32_t b0, b1, b2, b3;
-        ldsm_x4_t(sv + key * RB + ((ck ^ (key & 7)) << 4), b0, b1, b2, b3);
-        mma_bf16_16816(o[2 * dp], pf[kk], b0, b1);
-        mma_bf16_16816(o[2 * dp + 1], pf[kk], b2, b3);
+      for (int d4 = 0; d4 < HD / 16; d4 += 4) {
+        uint32_t bf[4][4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int key = kk * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+          const int ck = (d4 + j) * 2 + (lane >> 4);
+          ldsm_x4_t(sv + key * RB + ((ck ^ (key & 7)) << 4), bf[j][0], bf[j][1], bf[j][2], bf[j][3]);
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          mma_bf16_16816(o[2 * (d4 + j)], pf[kk], bf[j][0], bf[j][1]);
+          mma_bf16_16816(o[2 * (d4 + j) + 1], pf[kk], bf[j][2], bf[j][3]);
+        }
       }
     }
     __syncthreads();  // everyone is done with this stage before it is refilled
@@ -621,10 +565,9 @@ __device__ __forceinline__ void attn_prefill_tile(const DevCtx& c, int layer, in
 }
 
 // ---- the phase ---------------------------------------------------------------------------------------
-constexpr int ATT_SC_BYTES = ATT_WARPS * 16 * 8 * 4;   // per-warp score buffers, up to 8 heads per group
 template <int HD>
 constexpr int att_smem_bytes() {
-  constexpr int ring = ATT_WARPS * ATT_NS * 2 * 16 * HD * 2 + ATT_SC_BYTES;
+  constexpr int ring = ATT_WARPS * ATT_NS * 2 * 16 * HD * 2 + 1024;   // + alignment slack
   constexpr int tile = 128 * HD * 2 + 2 * 2 * 64 * HD * 2;
   return ring > tile ? ring : tile;
 }
@@ -648,9 +591,8 @@ __device__ __forceinline__ void phase_attention_bf16(const DevCtx& c, int layer,
     __syncthreads();
     const int w = threadIdx.x >> 5;
     constexpr int STAGE = 2 * 16 * HD * 2;
-    char* ring = smem + w * ATT_NS * STAGE;
-    float* sc = reinterpret_cast<float*>(smem + ATT_WARPS * ATT_NS * STAGE) + w * 16 * 8;
-    attn_decode_stream<HD, NREP>(c, layer, ring, sc, as);
+    char* ring = tc_tiles(smem_f) + w * ATT_NS * STAGE;   // 1024-byte aligned: the tiles are swizzled
+    attn_decode_stream<HD, NREP>(c, layer, ring, as);
   }
 }
 

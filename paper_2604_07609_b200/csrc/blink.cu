@@ -546,6 +546,24 @@ int blink_create(const blink_model_cfg* model, const blink_sched_cfg* sched, con
       TRY(dev_alloc(x, &c.dec_kbpre, MB + 1));
       TRY(dev_alloc(x, &c.pf_item, TM / 16 + MB + 1)); TRY(dev_alloc(x, &c.pf_qb, TM / 16 + MB + 1));
       TRY(dev_alloc(x, &c.att_ctr, (size_t)c.L)); TRY(dev_alloc(x, &c.att_cnt, MB * c.Hkv));
+      {  // the KV pool as a rank-5 tensor {64 dims, hd/64 halves, n_blocks*Hkv*16 keys, K|V, L}; one box = the
+         // K and V tiles of a (layer, block, kv head): {64, hd/64, 16, 2, 1}, 128-byte swizzle
+        EncodeTiledFn enc = tc_encode_fn();
+        const uint64_t rows = (uint64_t)c.n_blocks * c.Hkv * 16, rb = (uint64_t)c.hd * 2;
+        if (!enc || rows > 0x7fffffffull) return fail(BLINK_EINVAL);
+        CUtensorMap hm;
+        cuuint64_t dims[5] = {64, (cuuint64_t)(c.hd / 64), rows, 2, (cuuint64_t)c.L};
+        cuuint64_t strides[4] = {128, rb, rows * rb, 2 * rows * rb};
+        cuuint32_t box[5] = {64, (cuuint32_t)(c.hd / 64), 16, 2, 1};
+        cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+        if (enc(&hm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, c.kv_base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+          return fail(BLINK_ECUDA);
+        void* dm = nullptr;
+        TRY(dev_alloc(x, reinterpret_cast<char**>(&dm), sizeof(CUtensorMap), false));
+        if (cudaMemcpy(dm, &hm, sizeof(CUtensorMap), cudaMemcpyHostToDevice) != cudaSuccess) return fail(BLINK_ECUDA);
+        c.kv_map = dm;
+      }
       TRY(dev_alloc(x, &c.att_part, (size_t)(2 * c.att_sub_max) * (c.n_rep * c.hd + ((2 * c.n_rep + 3) & ~3)), false));
     }
     TRY(dev_alloc(x, &p, TM * c.q_dim * esz)); c.attn = p;

@@ -187,6 +187,7 @@ struct DevCtx {
   float *rope_cos, *rope_sin;  // [max_pos][hd/2]
   void* kv_base;               // [L][2][n_blocks][Hkv][bs][hd] operand type
   const void* tc_maps;         // TMA descriptors of the tensor-core path (device memory)
+  const void* kv_map;          // TMA descriptor of the KV pool seen as [rows][head_dim], box 16 x 64 (device memory)
   // diagnostics
   int32_t* trace;
   long long trace_cap;

@@ -430,6 +430,7 @@ static __device__ void phase_silu_mul(const DevCtx& c) {
   WT* out = reinterpret_cast<WT*>(c.act);
   const int F4 = c.F / 4;
   const long long total = (long long)T * F4;
+#pragma unroll 4
   for (long long idx = (long long)blockIdx.x * FWD_THREADS + threadIdx.x; idx < total;
        idx += (long long)gridDim.x * FWD_THREADS) {
     const int t = (int)(idx / F4), j = (int)(idx % F4) * 4;
