@@ -97,7 +97,7 @@ typedef struct blink_ctx blink_ctx;
 typedef struct blink_model_cfg {
   uint32_t size;
   int32_t n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ff, vocab;
-  int32_t n_experts;     /* 0 = dense FFN */
+  int32_t n_experts;     /* 0 = dense FFN, else up to 16 routed experts */
   int32_t top_k_experts; /* experts per token when n_experts > 0 */
   float rope_theta;
   float rms_eps;
@@ -192,8 +192,8 @@ typedef struct blink_iter_stat {
   uint64_t phase_ns[16];  /* persistent / manual mode: device time per phase kind, summed over the
                              layers, each including the grid barrier that closes it.  Index:
                              0 norm1(+embedding) 1 QKV 2 RoPE+KV write 3 attention 4 O 5 norm2
-                             6 gate/up 7 SwiGLU 8 down 9 final norm 10 LM head 11 sampling;
-                             12..15 unused (zero)                                             */
+                             6 gate/up 7 SwiGLU 8 down 9 final norm 10 LM head 11 sampling
+                             12 expert grouping + gather (routed experts); 13..15 unused (zero)                                             */
 } blink_iter_stat;
 
 /* Bytes of the flat weight buffer for a model shape (dtype taken from cfg). */

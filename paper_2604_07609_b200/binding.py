@@ -81,7 +81,7 @@ ITER_STAT_DTYPE = np.dtype([("t_begin_ns", "<u8"), ("t_forward_ns", "<u8"), ("t_
                             ("n_items", "<i4"), ("ctx_tokens", "<i8"), ("kv_tokens", "<i8"),
                             ("phase_ns", "<u8", (16,))])
 PHASE_NAMES = ["norm1", "qkv", "rope_kv", "attention", "o", "norm2", "gate_up", "swiglu", "down", "final_norm",
-               "lm_head", "sample"]
+               "lm_head", "sample", "moe_group"]
 EVENT_DTYPE = np.dtype([("ticket", "<u8"), ("user_tag", "<u8"), ("index", "<i4"), ("token", "<i4"),
                         ("is_first", "<i4"), ("is_last", "<i4"), ("t_device_ns", "<u8"), ("t_host_ns", "<u8"),
                         ("t_submit_ns", "<u8")])

@@ -215,6 +215,8 @@ size_t phase_smem_bytes(const blink_ctx* x) {
   size_t s = sizeof(float) * (size_t)SAMPLE_SMEM_FLOATS;
   size_t m = a > s ? a : s;
   if (x->dc.gemm_tc && tc_smem_bytes() > m) m = tc_smem_bytes();
+  const size_t moe = x->dc.E > 0 ? (size_t)x->dc.Tmax * x->dc.topE * sizeof(int) : 0;   // routing lists of a step
+  if (moe > m) m = moe;
   if (x->dc.dtype == BLINK_DTYPE_BF16) {
     const size_t ab = x->dc.hd == 64 ? (size_t)att_smem_bytes<64>() : (size_t)att_smem_bytes<128>();
     if (ab > m) m = ab;
@@ -253,8 +255,8 @@ int pump(blink_ctx* x) {
   return launch_loop(x);
 }
 
-void launch_phase(blink_ctx* x, int phase, int layer) {
-  void* args[] = {(void*)&x->dc, (void*)&phase, (void*)&layer};
+void launch_phase(blink_ctx* x, int phase, int layer, int sub = 0) {
+  void* args[] = {(void*)&x->dc, (void*)&phase, (void*)&layer, (void*)&sub};
   cudaLaunchKernel(x->ks.phase, dim3(x->grid), dim3(FWD_THREADS), args, x->smem_bytes, x->stream);
   x->launches += 1;
 }
@@ -264,7 +266,14 @@ int step_once(blink_ctx* x) {
   x->launches += 1;
   if (!x->dc.control_only) {
     for (int l = 0; l < x->dc.L; ++l)
-      for (int ph = PH_NORM1; ph <= PH_DOWN; ++ph) launch_phase(x, ph, l);
+      for (int ph = PH_NORM1; ph <= PH_DOWN; ++ph) {
+        if (x->dc.E > 0 && (ph == PH_GU || ph == PH_DOWN)) {
+          if (ph == PH_GU) launch_phase(x, PH_MOE_GROUP, l);
+          for (int e = 0; e < x->dc.E; ++e) launch_phase(x, ph, l, e);
+        } else {
+          launch_phase(x, ph, l);
+        }
+      }
     for (int ph = PH_FNORM; ph <= PH_SAMPLE; ++ph) launch_phase(x, ph, 0);
   }
   return cudaGetLastError() == cudaSuccess ? BLINK_OK : BLINK_ECUDA;
@@ -449,7 +458,7 @@ int blink_create(const blink_model_cfg* model, const blink_sched_cfg* sched, con
   if (kv->block_size != 16) return BLINK_EINVAL;
   if (!sched->control_only && (model->weights == nullptr || model->weights_bytes < blink_weights_bytes(model)))
     return BLINK_EINVAL;
-  if (model->n_experts > 0 && !sched->control_only) return BLINK_EINVAL;  // routed experts: not built yet
+  if (model->n_experts > MAX_EXPERTS) return BLINK_EINVAL;
   if (((uintptr_t)kv->base & 255) || ((uintptr_t)model->weights & 255)) return BLINK_EINVAL;
   int dev_count = 0;
   if (cudaGetDeviceCount(&dev_count) != cudaSuccess || dev_count < 1) return BLINK_ECUDA;
@@ -567,8 +576,14 @@ int blink_create(const blink_model_cfg* model, const blink_sched_cfg* sched, con
       TRY(dev_alloc(x, &c.att_part, (size_t)(2 * c.att_sub_max) * (c.n_rep * c.hd + ((2 * c.n_rep + 3) & ~3)), false));
     }
     TRY(dev_alloc(x, &p, TM * c.q_dim * esz)); c.attn = p;
-    TRY(dev_alloc(x, &c.gu, TM * 2 * c.F));
-    TRY(dev_alloc(x, &p, TM * c.F * esz)); c.act = p;
+    const size_t RA = TM * (c.E > 0 ? (size_t)c.topE : 1);   // routed experts: one FFN row per (token, expert)
+    TRY(dev_alloc(x, &c.gu, RA * 2 * c.F));
+    TRY(dev_alloc(x, &p, RA * c.F * esz)); c.act = p;
+    if (c.E > 0) {
+      TRY(dev_alloc(x, &p, RA * c.d * esz)); c.xg = p;
+      TRY(dev_alloc(x, &c.moe_sel, RA)); TRY(dev_alloc(x, &c.moe_wt, RA)); TRY(dev_alloc(x, &c.moe_off, (size_t)c.E + 1));
+      TRY(dev_alloc(x, &c.moe_tok, RA)); TRY(dev_alloc(x, &c.moe_gate, RA));
+    }
     TRY(dev_alloc(x, &p, MB * c.d * esz)); c.xs = p;
     TRY(dev_alloc(x, &c.logits, MB * c.V));
     TRY(dev_alloc(x, &c.rope_cos, (size_t)c.max_pos * (c.hd / 2), false));

@@ -123,6 +123,7 @@ constexpr int32_t TRACE_MAGIC = 0x424C4B31;
 constexpr int CTRL_THREADS = 256;
 constexpr int MAX_BATCH = 256;
 constexpr int MAX_TOPK = 64;
+constexpr int MAX_EXPERTS = 16;
 
 struct DevCtx {
   // model
@@ -183,6 +184,13 @@ struct DevCtx {
   float* gu;      // [Tmax][2F]
   void* act;      // [Tmax][F]      operand type
   void* xs;       // [MB][d]        operand type
+  // routed experts (E > 0): one row per (token, chosen expert); gu and act then have Tmax * topE rows
+  void* xg;            // [Tmax*topE][d] operand type: normed rows gathered per expert
+  int32_t* moe_sel;    // [Tmax][topE] chosen experts of a token, by descending router weight
+  float* moe_wt;       // [Tmax][topE] their weights (sum to 1)
+  int32_t* moe_off;    // [E+1] first gathered row of each expert
+  int32_t* moe_tok;    // [Tmax*topE] token of a gathered row
+  float* moe_gate;     // [Tmax*topE] its weight
   float* logits;  // [MB][V]
   float *rope_cos, *rope_sin;  // [max_pos][hd/2]
   void* kv_base;               // [L][2][n_blocks][Hkv][bs][hd] operand type

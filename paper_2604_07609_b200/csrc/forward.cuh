@@ -96,7 +96,7 @@ __device__ __forceinline__ float4 load4<__nv_bfloat16>(const __nv_bfloat16* p) {
 constexpr int NORM_MAXV = 8;
 template <typename WT>
 __device__ __forceinline__ void norm_row_cta(const DevCtx& c, float* hrow, const WT* src_embed, const float* g, WT* orow,
-                                             float* s_red) {
+                                             float* s_red, const float* wr = nullptr, int row_index = 0) {
   const int d = c.d;
   float4 v[NORM_MAXV];
   float ss = 0.f;
@@ -126,8 +126,55 @@ __device__ __forceinline__ void norm_row_cta(const DevCtx& c, float* hrow, const
     const int i = (k * FWD_THREADS + threadIdx.x) * 4;
     if (i < d) {
       const float4 gg = *reinterpret_cast<const float4*>(g + i);
-      store4<WT>(orow + i, v[k].x * inv * gg.x, v[k].y * inv * gg.y, v[k].z * inv * gg.z, v[k].w * inv * gg.w);
+      v[k] = make_float4(v[k].x * inv * gg.x, v[k].y * inv * gg.y, v[k].z * inv * gg.z, v[k].w * inv * gg.w);
+      store4<WT>(orow + i, v[k].x, v[k].y, v[k].z, v[k].w);
     }
+  }
+  if (wr != nullptr) {
+    // Router of the routed-expert FFN on the normed row in fp32 (not its 16-bit copy): logits over
+    // the E experts, top-k by (logit desc, expert id asc), weights = softmax restricted to the chosen.
+    __shared__ float s_rl[FWD_THREADS / 32][MAX_EXPERTS];
+    const int E = c.E;
+    for (int e = 0; e < E; ++e) {
+      float p = 0.f;
+#pragma unroll
+      for (int k = 0; k < NORM_MAXV; ++k) {
+        const int i = (k * FWD_THREADS + threadIdx.x) * 4;
+        if (i < d) {
+          const float4 w4 = *reinterpret_cast<const float4*>(wr + (size_t)e * d + i);
+          p = fmaf(v[k].x, w4.x, p); p = fmaf(v[k].y, w4.y, p); p = fmaf(v[k].z, w4.z, p); p = fmaf(v[k].w, w4.w, p);
+        }
+      }
+      p = warp_sum(p);
+      if ((threadIdx.x & 31) == 0) s_rl[threadIdx.x >> 5][e] = p;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      float lg[MAX_EXPERTS];
+      for (int e = 0; e < E; ++e) {
+        float t = 0.f;
+        for (int w = 0; w < FWD_THREADS / 32; ++w) t += s_rl[w][e];
+        lg[e] = t;
+      }
+      int sel[MAX_EXPERTS];
+      float den = 0.f, top = 0.f;
+      for (int j = 0; j < c.topE; ++j) {
+        int best = -1;
+        for (int e = 0; e < E; ++e) {
+          bool taken = false;
+          for (int q = 0; q < j; ++q) taken |= sel[q] == e;
+          if (!taken && (best < 0 || lg[e] > lg[best])) best = e;   // ties keep the lower id
+        }
+        sel[j] = best;
+        if (j == 0) top = lg[best];
+        den += expf(lg[best] - top);
+      }
+      for (int j = 0; j < c.topE; ++j) {
+        c.moe_sel[(size_t)row_index * c.topE + j] = sel[j];
+        c.moe_wt[(size_t)row_index * c.topE + j] = expf(lg[sel[j]] - top) / den;
+      }
+    }
+    __syncthreads();
   }
 }
 
@@ -140,10 +187,12 @@ static __device__ void phase_norm(const DevCtx& c, int layer, int which /*0: nor
   const float* g = wptr_f(c, which == 0 ? 6 : 7) + (size_t)layer * c.d;
   WT* out = reinterpret_cast<WT*>(c.xn);
   // the split-K tensor-core GEMM that follows adds partial sums into its output
-  if (c.gemm_tc) zero_floats(which == 0 ? c.qkv : c.gu, (long long)T * (which == 0 ? c.qkv_dim : 2 * c.F));
+  const int rows_gu = c.E > 0 ? T * c.topE : T;   // routed experts: one gate/up row per (token, expert)
+  if (c.gemm_tc) zero_floats(which == 0 ? c.qkv : c.gu, which == 0 ? (long long)T * c.qkv_dim : (long long)rows_gu * 2 * c.F);
+  const float* wr = (which == 1 && c.E > 0) ? wptr_f(c, 5) + (size_t)layer * c.E * c.d : nullptr;
   for (int t = blockIdx.x; t < T; t += gridDim.x) {
     const WT* e = (which == 0 && layer == 0) ? wptr<WT>(c, 0) + (size_t)c.tok_id[t] * c.d : nullptr;
-    norm_row_cta<WT>(c, c.h + (size_t)t * c.d, e, g, out + (size_t)t * c.d, s_red);
+    norm_row_cta<WT>(c, c.h + (size_t)t * c.d, e, g, out + (size_t)t * c.d, s_red, wr, t);
   }
 }
 
@@ -167,6 +216,13 @@ struct GemmArgs {
   float* out;      // [M][ldo]
   int M, N, K, ldo;
   int accumulate;  // 1: out += result (residual), 0: out = result
+  // routed experts: x rows start at row x_row0 of the activation buffer, the weights at row w_row0 of
+  // the stacked weight tensor; with row_map the result row t goes to out row row_map[t], scaled by
+  // row_scale[t], always added (several experts contribute to one token)
+  int x_row0 = 0;
+  long long w_row0 = 0;
+  const int32_t* row_map = nullptr;
+  const float* row_scale = nullptr;
 };
 
 template <typename WT>
@@ -220,8 +276,12 @@ static __device__ void phase_gemm_simt(const GemmArgs& a) {
       for (int j = 0; j < 4; ++j) {
         const int n = n0 + tx * 4 + j;
         if (n >= a.N) continue;
-        float* o = a.out + (size_t)m * a.ldo + n;
-        *o = a.accumulate ? (*o + acc[i][j]) : acc[i][j];
+        if (a.row_map != nullptr) {
+          atomicAdd(a.out + (size_t)a.row_map[m] * a.ldo + n, a.row_scale[m] * acc[i][j]);
+        } else {
+          float* o = a.out + (size_t)m * a.ldo + n;
+          *o = a.accumulate ? (*o + acc[i][j]) : acc[i][j];
+        }
       }
     }
   }
@@ -426,7 +486,7 @@ constexpr int ATTN_SMEM_FLOATS(int HD, int NREP) { return NREP * HD + 2 * 8 * NR
 // ---- SwiGLU gate: act = silu(gate) * up ------------------------------------------------
 template <typename WT>
 static __device__ void phase_silu_mul(const DevCtx& c) {
-  const int T = c.ss->cur_T;
+  const int T = c.E > 0 ? c.ss->cur_T * c.topE : c.ss->cur_T;   // rows of the gate/up buffer
   WT* out = reinterpret_cast<WT*>(c.act);
   const int F4 = c.F / 4;
   const long long total = (long long)T * F4;
@@ -438,6 +498,53 @@ static __device__ void phase_silu_mul(const DevCtx& c) {
     const float4 u = *reinterpret_cast<const float4*>(c.gu + (size_t)t * 2 * c.F + c.F + j);
     store4<WT>(out + (size_t)t * c.F + j, g.x / (1.0f + __expf(-g.x)) * u.x, g.y / (1.0f + __expf(-g.y)) * u.y,
                g.z / (1.0f + __expf(-g.z)) * u.z, g.w / (1.0f + __expf(-g.w)) * u.w);
+  }
+}
+
+// ---- routed experts: group the (token, expert) pairs by expert and gather their rows ---------
+// Every CTA builds the same lists in shared memory (stable: ascending token inside an expert, so
+// the order does not depend on timing), CTA 0 publishes them, and all CTAs copy the normed rows
+// of the tokens into expert-contiguous order for the per-expert GEMMs.
+template <typename WT>
+static __device__ void phase_moe_group(const DevCtx& c, float* smem) {
+  const int T = c.ss->cur_T, K = c.topE, E = c.E;
+  const int A = T * K;   // assignments
+  __shared__ int s_off[MAX_EXPERTS + 1];
+  int* s_tok = reinterpret_cast<int*>(smem);          // [A] token of each gathered row
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  // counts, then offsets
+  if (threadIdx.x <= E) s_off[threadIdx.x] = 0;
+  __syncthreads();
+  for (int a = threadIdx.x; a < A; a += FWD_THREADS) atomicAdd(&s_off[c.moe_sel[a] + 1], 1);
+  __syncthreads();
+  if (threadIdx.x == 0)
+    for (int e = 0; e < E; ++e) s_off[e + 1] += s_off[e];
+  __syncthreads();
+  // stable placement: a warp walks all assignments in order for each of its experts
+  for (int e = w; e < E; e += FWD_THREADS / 32) {
+    int base = s_off[e];
+    for (int a0 = 0; a0 < A; a0 += 32) {
+      const int a = a0 + lane;
+      const bool mine = a < A && c.moe_sel[a] == e;
+      const unsigned m = __ballot_sync(0xffffffffu, mine);
+      if (mine) {
+        const int pos = base + __popc(m & ((1u << lane) - 1u));
+        s_tok[pos] = a / K;
+        if (blockIdx.x == 0) { c.moe_tok[pos] = a / K; c.moe_gate[pos] = c.moe_wt[a]; }
+      }
+      base += __popc(m);
+    }
+  }
+  if (blockIdx.x == 0 && threadIdx.x <= E) c.moe_off[threadIdx.x] = s_off[threadIdx.x];
+  __syncthreads();
+  // gather: one warp per row, 16-byte vectors
+  const WT* xn = reinterpret_cast<const WT*>(c.xn);
+  WT* xg = reinterpret_cast<WT*>(c.xg);
+  const int vec_per_row = c.d * (int)sizeof(WT) / 16;
+  for (int r = blockIdx.x * (FWD_THREADS / 32) + w; r < A; r += gridDim.x * (FWD_THREADS / 32)) {
+    const uint4* src = reinterpret_cast<const uint4*>(xn + (size_t)s_tok[r] * c.d);
+    uint4* dst = reinterpret_cast<uint4*>(xg + (size_t)r * c.d);
+    for (int i = lane; i < vec_per_row; i += 32) dst[i] = src[i];
   }
 }
 

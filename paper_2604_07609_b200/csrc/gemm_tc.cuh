@@ -29,7 +29,7 @@
 namespace blink {
 
 enum GemmWhich : int { GEMM_QKV = 0, GEMM_O, GEMM_GU, GEMM_DOWN, GEMM_LMHEAD, GEMM_KINDS };
-enum ActBuf : int { ACT_XN = 0, ACT_ATTN, ACT_ACT, ACT_XS, ACT_BUFS };
+enum ActBuf : int { ACT_XN = 0, ACT_ATTN, ACT_ACT, ACT_XS, ACT_XG, ACT_BUFS };
 constexpr int TC_BOXES = 5;  // token-tile boxes of 16, 32, 64, 128, 256 rows
 constexpr int TC_MAX_STAGES = 8;
 constexpr int TC_A_BYTES = 128 * 128;  // 128 weight rows x 64 bf16
@@ -236,11 +236,11 @@ __device__ __forceinline__ char* tc_tiles(float* smem_f) {
 }
 
 // Weight producer (one thread): stream the weight tiles of this CTA's range through the ring.
-__device__ __forceinline__ void tc_produce_weights(const DevCtx& c, const void* w, int which, int layer, const TcGeom& g,
-                                                   char* tiles, TcState& tc) {
+__device__ __forceinline__ void tc_produce_weights(const DevCtx& c, const void* w, long long w_row0, int which,
+                                                   const TcGeom& g, char* tiles, TcState& tc) {
   const TcMaps* maps = reinterpret_cast<const TcMaps*>(c.tc_maps);
   const CUtensorMap* map_a = &maps->w[which];
-  const int row_a0 = which == GEMM_LMHEAD ? 0 : layer * (g.ntiles * 128);
+  const int row_a0 = (int)w_row0;
   volatile int* dead = &g_tc.dead;
   long long u = g.u0;
   int stage = 0;
@@ -272,7 +272,8 @@ static __device__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int whi
   const TcGeom g = tc_geom(c, T, N, K);
   const int kblocks = g.kblocks, ntiles = g.ntiles, KPS = g.KPS, S = g.S;
   const uint32_t b_bytes = g.b_bytes, stage_bytes = g.stage_bytes;
-  const int act_id = which == GEMM_O ? ACT_ATTN : which == GEMM_DOWN ? ACT_ACT : which == GEMM_LMHEAD ? ACT_XS : ACT_XN;
+  const int act_id = which == GEMM_O ? ACT_ATTN : which == GEMM_DOWN ? ACT_ACT : which == GEMM_LMHEAD ? ACT_XS
+                     : (which == GEMM_GU && c.E > 0) ? ACT_XG : ACT_XN;
   const CUtensorMap* map_b = &maps->act[act_id][g.box_id];
   char* tiles = tc_tiles(smem_f);
   const long long u0 = g.u0, u1 = g.u1;
@@ -281,7 +282,7 @@ static __device__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int whi
 
   if (warp == 0) {
     if (lane == 0) {
-      tc_produce_weights(c, a.w, which, layer, g, tiles, tc);
+      tc_produce_weights(c, a.w, a.w_row0, which, g, tiles, tc);
     }
   } else if (warp == 2) {
     // token-tile producer: walks the same sequence of stages (nk k-blocks of one segment each)
@@ -298,7 +299,7 @@ static __device__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int whi
         char* sa = tiles + (size_t)stage * stage_bytes;
         mbar_expect_tx(&g_tc.full[stage], (uint32_t)nk * b_bytes);
         for (int j = 0; j < nk; ++j)
-          tma_load_2d(sa + KPS * TC_A_BYTES + j * b_bytes, map_b, (kb + j) * 64, pass * 256, &g_tc.full[stage]);
+          tma_load_2d(sa + KPS * TC_A_BYTES + j * b_bytes, map_b, (kb + j) * 64, a.x_row0 + pass * 256, &g_tc.full[stage]);
         u += nk;
         if (++stage == S) stage = 0;
       }
@@ -371,9 +372,13 @@ static __device__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int whi
           for (int j = 0; j < 16; ++j) {
             const int t = pass * 256 + c0 + j;
             if (t < T) {
-              float* o = a.out + (size_t)t * a.ldo + n;
-              if (whole && !a.accumulate) *o = v[j];
-              else atomicAdd(o, v[j]);
+              if (a.row_map != nullptr) {
+                atomicAdd(a.out + (size_t)a.row_map[t] * a.ldo + n, a.row_scale[t] * v[j]);
+              } else {
+                float* o = a.out + (size_t)t * a.ldo + n;
+                if (whole && !a.accumulate) *o = v[j];
+                else atomicAdd(o, v[j]);
+              }
             }
           }
         }
@@ -420,7 +425,7 @@ inline bool tc_make_map(EncodeTiledFn enc, CUtensorMap* m, const void* base, uin
 // The tensor-core path needs every contraction length to be a multiple of 64 (one swizzled
 // smem row) and 16-byte aligned rows.
 inline int tc_shape_ok(const DevCtx& c) {
-  return c.dtype == 0 && c.d % 64 == 0 && c.q_dim % 64 == 0 && c.F % 64 == 0 && c.V % 4 == 0 && c.E == 0;
+  return c.dtype == 0 && c.d % 64 == 0 && c.q_dim % 64 == 0 && c.F % 64 == 0 && c.V % 4 == 0;
 }
 inline int tc_available() { return tc_encode_fn() != nullptr; }
 // The streaming layout needs whole 128-row panels per layer in every GEMM matrix.
@@ -437,12 +442,14 @@ inline int tc_host_setup(TcHost& h, DevCtx& c) {
   bool ok = true;
   ok &= tc_make_map(enc, &hm->w[GEMM_QKV], w + c.w_off[1], L * c.qkv_dim, c.d, 128, true);
   ok &= tc_make_map(enc, &hm->w[GEMM_O], w + c.w_off[2], L * c.d, c.q_dim, 128, true);
-  ok &= tc_make_map(enc, &hm->w[GEMM_GU], w + c.w_off[3], L * 2 * c.F, c.d, 128, true);
-  ok &= tc_make_map(enc, &hm->w[GEMM_DOWN], w + c.w_off[4], L * c.d, c.F, 128, true);
+  const uint64_t E1 = c.E > 0 ? c.E : 1;
+  ok &= tc_make_map(enc, &hm->w[GEMM_GU], w + c.w_off[3], L * E1 * 2 * c.F, c.d, 128, true);
+  ok &= tc_make_map(enc, &hm->w[GEMM_DOWN], w + c.w_off[4], L * E1 * c.d, c.F, 128, true);
   ok &= tc_make_map(enc, &hm->w[GEMM_LMHEAD], w + c.w_off[9], c.V, c.d, 128, true);
-  const void* bufs[ACT_BUFS] = {c.xn, c.attn, c.act, c.xs};
-  const uint64_t rows[ACT_BUFS] = {(uint64_t)c.Tmax, (uint64_t)c.Tmax, (uint64_t)c.Tmax, (uint64_t)c.MB};
-  const uint64_t cols[ACT_BUFS] = {(uint64_t)c.d, (uint64_t)c.q_dim, (uint64_t)c.F, (uint64_t)c.d};
+  const void* bufs[ACT_BUFS] = {c.xn, c.attn, c.act, c.xs, c.xg ? c.xg : c.xn};
+  const uint64_t RA = (uint64_t)c.Tmax * (c.E > 0 ? c.topE : 1);   // routed experts: one row per (token, expert)
+  const uint64_t rows[ACT_BUFS] = {(uint64_t)c.Tmax, (uint64_t)c.Tmax, RA, (uint64_t)c.MB, c.xg ? RA : (uint64_t)c.Tmax};
+  const uint64_t cols[ACT_BUFS] = {(uint64_t)c.d, (uint64_t)c.q_dim, (uint64_t)c.F, (uint64_t)c.d, (uint64_t)c.d};
   for (int b = 0; b < ACT_BUFS; ++b)
     for (int i = 0; i < TC_BOXES; ++i) ok &= tc_make_map(enc, &hm->act[b][i], bufs[b], rows[b], cols[b], 16u << i, false);
   int rc = 0;

@@ -22,7 +22,8 @@ __device__ __forceinline__ void gemm_dispatch(const DevCtx& c, const GemmArgs& a
 }
 
 template <typename WT, int HD, int NREP>
-__device__ __forceinline__ void run_phase(const DevCtx& c, int phase, int layer, float* smem, TcState& tc, AttState& as) {
+__device__ __forceinline__ void run_phase(const DevCtx& c, int phase, int layer, int sub, float* smem, TcState& tc,
+                                          AttState& as) {
   const int T = c.ss->cur_T;
   const size_t esz = sizeof(WT);
   switch (phase) {
@@ -32,6 +33,7 @@ __device__ __forceinline__ void run_phase(const DevCtx& c, int phase, int layer,
     case PH_QKV: {
       GemmArgs a{c.xn, c.w_base + c.w_off[1] + (size_t)layer * c.qkv_dim * c.d * esz, c.qkv, T, c.qkv_dim, c.d,
                  c.qkv_dim, 0};
+      a.w_row0 = (long long)layer * c.qkv_dim;
       gemm_dispatch<WT>(c, a, GEMM_QKV, layer, smem, tc);
     } break;
     case PH_ROPE: phase_rope_kv<WT>(c, layer); break;
@@ -42,22 +44,49 @@ __device__ __forceinline__ void run_phase(const DevCtx& c, int phase, int layer,
       break;
     case PH_O: {
       GemmArgs a{c.attn, c.w_base + c.w_off[2] + (size_t)layer * c.d * c.q_dim * esz, c.h, T, c.d, c.q_dim, c.d, 1};
+      a.w_row0 = (long long)layer * c.d;
       gemm_dispatch<WT>(c, a, GEMM_O, layer, smem, tc);
     } break;
     case PH_NORM2:
       phase_norm<WT>(c, layer, 1);
       break;
     case PH_GU: {
-      GemmArgs a{c.xn, c.w_base + c.w_off[3] + (size_t)layer * 2 * c.F * c.d * esz, c.gu, T, 2 * c.F, c.d, 2 * c.F, 0};
-      gemm_dispatch<WT>(c, a, GEMM_GU, layer, smem, tc);
+      if (c.E == 0) {
+        GemmArgs a{c.xn, c.w_base + c.w_off[3] + (size_t)layer * 2 * c.F * c.d * esz, c.gu, T, 2 * c.F, c.d, 2 * c.F, 0};
+        a.w_row0 = (long long)layer * 2 * c.F;
+        gemm_dispatch<WT>(c, a, GEMM_GU, layer, smem, tc);
+      } else {
+        // expert `sub` on the rows routed to it (gathered, contiguous from moe_off[sub])
+        const int off = c.moe_off[sub], cnt = c.moe_off[sub + 1] - off;
+        const long long we = (long long)layer * c.E + sub;
+        GemmArgs a{reinterpret_cast<const char*>(c.xg) + (size_t)off * c.d * esz, c.w_base + c.w_off[3] + (size_t)we * 2 * c.F * c.d * esz,
+                   c.gu + (size_t)off * 2 * c.F, cnt, 2 * c.F, c.d, 2 * c.F, 0};
+        a.x_row0 = off;
+        a.w_row0 = we * 2 * c.F;
+        gemm_dispatch<WT>(c, a, GEMM_GU, layer, smem, tc);
+      }
     } break;
     case PH_SILU:
       phase_silu_mul<WT>(c);
       break;
     case PH_DOWN: {
-      GemmArgs a{c.act, c.w_base + c.w_off[4] + (size_t)layer * c.d * c.F * esz, c.h, T, c.d, c.F, c.d, 1};
-      gemm_dispatch<WT>(c, a, GEMM_DOWN, layer, smem, tc);
+      if (c.E == 0) {
+        GemmArgs a{c.act, c.w_base + c.w_off[4] + (size_t)layer * c.d * c.F * esz, c.h, T, c.d, c.F, c.d, 1};
+        a.w_row0 = (long long)layer * c.d;
+        gemm_dispatch<WT>(c, a, GEMM_DOWN, layer, smem, tc);
+      } else {
+        const int off = c.moe_off[sub], cnt = c.moe_off[sub + 1] - off;
+        const long long we = (long long)layer * c.E + sub;
+        GemmArgs a{reinterpret_cast<const char*>(c.act) + (size_t)off * c.F * esz, c.w_base + c.w_off[4] + (size_t)we * c.d * c.F * esz,
+                   c.h, cnt, c.d, c.F, c.d, 1};
+        a.x_row0 = off;
+        a.w_row0 = we * c.d;
+        a.row_map = c.moe_tok + off;     // result row i belongs to token moe_tok[off + i], weighted by its gate
+        a.row_scale = c.moe_gate + off;
+        gemm_dispatch<WT>(c, a, GEMM_DOWN, layer, smem, tc);
+      }
     } break;
+    case PH_MOE_GROUP: phase_moe_group<WT>(c, smem); break;
     case PH_FNORM:
       phase_final_norm<WT>(c);
       break;
@@ -90,18 +119,22 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) blink_loop_kernel(const __grid
       // the barrier that closes it); recorded only when per-iteration statistics are kept
       const bool timed = c.stats_cap > 0 && blockIdx.x == 0 && threadIdx.x == 0;
       uint64_t t_prev = timed ? global_timer_ns() : 0;
-      for (int layer = 0; layer < c.L && ok; ++layer) {
-        for (int ph = PH_NORM1; ph <= PH_DOWN && ok; ++ph) {
-          run_phase<WT, HD, NREP>(c, ph, layer, smem, tc, as);
-          ok = grid_barrier(c, gen);
-          if (timed) { const uint64_t t = global_timer_ns(); c.ss->cur_phase_ns[ph] += t - t_prev; t_prev = t; }
-        }
-      }
-      for (int ph = PH_FNORM; ph <= PH_SAMPLE && ok; ++ph) {
-        run_phase<WT, HD, NREP>(c, ph, 0, smem, tc, as);
+      auto step_phase = [&](int ph, int layer, int sub) {
+        run_phase<WT, HD, NREP>(c, ph, layer, sub, smem, tc, as);
         ok = grid_barrier(c, gen);
         if (timed) { const uint64_t t = global_timer_ns(); c.ss->cur_phase_ns[ph] += t - t_prev; t_prev = t; }
+      };
+      for (int layer = 0; layer < c.L && ok; ++layer) {
+        for (int ph = PH_NORM1; ph <= PH_DOWN && ok; ++ph) {
+          if (c.E > 0 && (ph == PH_GU || ph == PH_DOWN)) {
+            if (ph == PH_GU) step_phase(PH_MOE_GROUP, layer, 0);   // routing lists and gathered rows first
+            for (int e = 0; e < c.E && ok; ++e) step_phase(ph, layer, e);
+          } else {
+            step_phase(ph, layer, 0);
+          }
+        }
       }
+      for (int ph = PH_FNORM; ph <= PH_SAMPLE && ok; ++ph) step_phase(ph, 0, 0);
       if (!ok) break;
     } else if (!grid_barrier(c, gen)) break;
   }
@@ -115,14 +148,14 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) blink_loop_kernel(const __grid
 }
 
 template <typename WT, int HD, int NREP>
-__global__ void __launch_bounds__(FWD_THREADS, 1) blink_phase_kernel(const __grid_constant__ DevCtx c, int phase, int layer) {
+__global__ void __launch_bounds__(FWD_THREADS, 1) blink_phase_kernel(const __grid_constant__ DevCtx c, int phase, int layer, int sub) {
   extern __shared__ __align__(1024) float smem[];
   if (c.ss->cmd != CMD_RUN) return;
   TcState tc;
   tc_init(c, smem, tc);
   AttState as;
   att_init(c, as);
-  run_phase<WT, HD, NREP>(c, phase, layer, smem, tc, as);
+  run_phase<WT, HD, NREP>(c, phase, layer, sub, smem, tc, as);
   tc_fini(c, tc);
 }
 

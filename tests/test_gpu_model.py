@@ -201,3 +201,24 @@ def test_streaming_weight_layout_round_trip_and_parity():
     # the SIMT path cannot read the streaming layout: refused, not misread
     with pytest.raises(B.BlinkError):
         gpu_run_forced(model, sched, reqs, w, ora["tokens"], gemm_impl=B.GEMM_SIMT, weights_layout=B.WEIGHTS_STREAMING)
+
+
+@pytest.mark.parametrize("dtype,tol,kw", [("fp32", TOL_FP32, {}),
+                                           ("bf16", TOL_BF16, dict(gemm_impl=B.GEMM_TC, weights_layout=B.WEIGHTS_STREAMING))],
+                         ids=["fp32-simt", "bf16-tensor-cores-streaming"])
+def test_routed_experts_match_oracle(dtype, tol, kw):
+    """Top-2 of 4 experts: router on the fp32 normed rows, stable grouping by expert, per-expert
+    GEMMs on gathered rows, gate-weighted sum into the residual stream."""
+    model = model_cfg(1, n_experts=4, top_k_experts=2, d_ff=512, dtype=dtype)
+    sched = sched_cfg(1, prefill_chunk_tokens=40, max_batch=6, n_blocks=128)
+    reqs = make_requests(1, n_requests=6)
+    for r in reqs:
+        r.max_new = 8
+    w = make_weights(model, 31, "cpu", random_gains=True)
+    ora = oracle_run(model, sched, reqs, w, O2.round_bf16 if dtype == "bf16" else None)
+    trace, toks, logits, _ = gpu_run_forced(model, sched, reqs, w, ora["tokens"], **kw)
+    lo = np.stack([row for (_, _, _, _, row) in ora["logits"]])
+    err = np.abs(logits.astype(np.float64) - lo).max()
+    print(f"routed experts {dtype}: max-abs logit error {err:.3e}")
+    assert err <= tol
+    assert_traces_equal([{**r, "sampled": []} for r in trace], [{**r, "sampled": []} for r in ora["trace"]])
