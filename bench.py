@@ -203,6 +203,35 @@ class Stressor:
         self.procs = []
 
 
+def decode_point(B, m, sched, wbuf, kv, wl, gemm_impl, n, in_len, out_len, steps, cfg_i):
+    """Fixed-batch decode steps (an N x I -> O closed batch past its prefill): the clean
+    bandwidth-bound operating point.  Returns ms/step and the HBM-roofline fractions."""
+    from synth.workload import closed_batch
+    reqs = closed_batch(n, in_len, out_len, m.vocab, seed=7, top_k=50 if cfg_i >= 3 else 0, temperature=0.8)
+    ramp = (n * in_len + sched.prefill_chunk_tokens - 1) // sched.prefill_chunk_tokens + 2
+    eng = B.Blink(m, sched, wbuf, kv, exec_mode=B.EXEC_MANUAL, gemm_impl=gemm_impl, stats_iters=ramp + steps + 16,
+                  idle_exit_us=200_000, weights_layout=wl)
+    try:
+        for r in reqs:
+            eng.submit_request(r)
+        eng.blink_run(ramp)
+        eng.blink_run(3)
+        while len(eng.blink_poll(4096, 0)):
+            pass
+        it0 = int(eng.blink_get_stats().iterations)
+        ms = eng.blink_run(steps)
+        its = eng.blink_get_iter_stats()[it0:it0 + steps]
+    finally:
+        eng.blink_destroy()
+    by, _ = step_bytes_flops(m, its)
+    pk = measured_peaks()
+    gbs = float(by.sum() / (ms / 1e3) / 1e9)
+    return dict(batch=float(its["n_decode"].mean()), ctx_mean=float(its["kv_tokens"].mean() / max(1.0, its["n_items"].mean())),
+                steps=int(len(its)), ms_per_step=ms / max(1, len(its)), algorithmic_gb_per_step=float(by.mean() / 1e9),
+                achieved_gbs=gbs, frac_of_measured_hbm=gbs / pk["hbm_gbs"], frac_of_8TBs_spec=gbs / 8000.0,
+                tok_s=float(its["n_sample_rows"].sum() / (ms / 1e3)))
+
+
 def percentiles(x):
     if len(x) == 0:
         return dict(p50=None, p99=None, mean=None)
@@ -287,6 +316,8 @@ def main():
     ap.add_argument("--closed-batch", default="", help="N,I,O: use an N x I -> O closed batch instead of the stream")
     ap.add_argument("--kv-fraction", type=float, default=0.8)
     ap.add_argument("--kv-blocks", type=int, default=0, help="cap the KV pool at this many blocks")
+    ap.add_argument("--decode-points", default="64,512,256;256,512,384",
+                    help="N,I,O closed batches whose decode steps are timed besides the stream ('' = none)")
     ap.add_argument("--layers", type=int, default=0,
                     help="profiling aid: keep only this many layers of the configuration's shape")
     ap.add_argument("--exec", default="manual", choices=["manual", "stepped"],
@@ -491,6 +522,16 @@ def main():
                 control_plane_us=dict(p50=float(np.median(ctrl_us)), max=float(ctrl_us.max())))
     if cpu_baseline is not None:
         line["cpu_baseline"] = cpu_baseline
+
+    # ---- decode-only operating points (fixed batch): the HBM-bound regime ---------------------
+    if args.decode_points and rank == 0 and world == 1 and not args.closed_batch:
+        pts = []
+        for spec in args.decode_points.split(";"):
+            n, i_len, o_len = (int(v) for v in spec.split(","))
+            pts.append(decode_point(B, m, sched, wbuf, kv, wl, gemm_impl, n, i_len, o_len, 20, cfg_i))
+            log(f"[bench] decode point {spec}: {pts[-1]['ms_per_step']:.2f} ms/step, "
+                f"{pts[-1]['frac_of_measured_hbm']:.3f} of measured HBM")
+        line["decode_steps"] = pts
 
     # ---- end to end through the public API with host buffers ------------------------------
     if not args.skip_e2e:
