@@ -302,12 +302,12 @@ static __device__ void phase_rope_kv(const DevCtx& c, int layer) {
   const int T = c.ss->cur_T;
   const int half = c.hd / 2, quads = half / 4;
   const int heads = c.Hq + 2 * c.Hkv;
-  const long long total = (long long)T * heads * quads;
-  for (long long idx = (long long)blockIdx.x * FWD_THREADS + threadIdx.x; idx < total;
-       idx += (long long)gridDim.x * FWD_THREADS) {
-    const int i = (int)(idx % quads) * 4;
-    const int hh = (int)((idx / quads) % heads);
-    const int t = (int)(idx / ((long long)quads * heads));
+  const int total = T * heads * quads;   // < 2^31
+#pragma unroll 2
+  for (int idx = blockIdx.x * FWD_THREADS + threadIdx.x; idx < total; idx += gridDim.x * FWD_THREADS) {
+    const int i = (idx % quads) * 4;
+    const int hh = (idx / quads) % heads;
+    const int t = idx / (quads * heads);
     float* row = c.qkv + (size_t)t * c.qkv_dim + (size_t)hh * c.hd;
     const float4 x1 = *reinterpret_cast<const float4*>(row + i), x2 = *reinterpret_cast<const float4*>(row + i + half);
     if (hh < c.Hq + c.Hkv) {
@@ -489,11 +489,10 @@ static __device__ void phase_silu_mul(const DevCtx& c) {
   const int T = c.E > 0 ? c.ss->cur_T * c.topE : c.ss->cur_T;   // rows of the gate/up buffer
   WT* out = reinterpret_cast<WT*>(c.act);
   const int F4 = c.F / 4;
-  const long long total = (long long)T * F4;
+  const int total = T * F4;   // < 2^31: at most a few thousand rows
 #pragma unroll 4
-  for (long long idx = (long long)blockIdx.x * FWD_THREADS + threadIdx.x; idx < total;
-       idx += (long long)gridDim.x * FWD_THREADS) {
-    const int t = (int)(idx / F4), j = (int)(idx % F4) * 4;
+  for (int idx = blockIdx.x * FWD_THREADS + threadIdx.x; idx < total; idx += gridDim.x * FWD_THREADS) {
+    const int t = idx / F4, j = (idx - t * F4) * 4;
     const float4 g = *reinterpret_cast<const float4*>(c.gu + (size_t)t * 2 * c.F + j);
     const float4 u = *reinterpret_cast<const float4*>(c.gu + (size_t)t * 2 * c.F + c.F + j);
     store4<WT>(out + (size_t)t * c.F + j, g.x / (1.0f + __expf(-g.x)) * u.x, g.y / (1.0f + __expf(-g.y)) * u.y,
