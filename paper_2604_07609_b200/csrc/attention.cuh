@@ -136,11 +136,11 @@ __device__ __forceinline__ void mma_bf16_16816(float* d, const uint32_t* a, uint
 // One warp owns a (row, kv head) unit at a time and walks its 16-key tiles.  A tile's K and V
 // ([16 keys][head_dim] each, contiguous in the pool) arrive through one TMA tile copy with the
 // 128-byte swizzle, so both can be read with ldmatrix (at most two-way bank conflicts).  The two small contractions
-// of a tile (scores = Q K^T for the query heads of the group, out += P V) run as m16n8k16 MMAs
-// with the group's heads in the first rows of the 16-row operand: written with CUDA-core FMAs
-// the same loop needs about 800 instructions per tile and the SM runs out of issue slots at
-// about half the HBM bandwidth; this form needs about 130.  Softmax statistics stay in fp32
-// registers and are combined with quad shuffles.
+// of a tile (scores and out += P V for the query heads of the group) run as m16n8k16 MMAs with
+// the 16 keys (or 16 output dims) as the rows and the group's heads as the columns: written with
+// CUDA-core FMAs the same loop needs about 800 instructions per tile and the SM runs out of issue
+// slots at about half the HBM bandwidth; this form needs about 110.  Softmax statistics stay in
+// fp32 registers and are combined with shuffles.
 template <int HD, int NREP>
 __device__ __noinline__ void attn_decode_stream(const DevCtx& c, int layer, char* ring, AttState& as) {
   constexpr int RB = HD * 2;         // bytes per key row
@@ -158,7 +158,7 @@ __device__ __noinline__ void attn_decode_stream(const DevCtx& c, int layer, char
   const int Hkv = c.Hkv;
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   const int gq = lane >> 2, tq = lane & 3;   // operand row (= head of the group) and column pair
-  const bool live = gq < NREP;
+  const bool live = gq < NREP;   // this lane loads the q of head gq
   uint64_t* bars = g_att.bar[w];
   volatile int* dead = &g_att.dead;
   int* ctr = c.att_ctr + layer;
@@ -175,9 +175,12 @@ __device__ __noinline__ void attn_decode_stream(const DevCtx& c, int layer, char
   int sub_start = 0, sub_id = 0;
   bool in_unit = false;
 
-  uint32_t qf[KS][2];     // operand rows 8..15 are zero, so only a0 and a2 of each k-step are kept
-  float o[HD / 8][2];     // out rows 0..7 (c0, c1 of each n-tile)
-  float m = -INFINITY, l = 0.f;
+  // Both contractions are written with the 16 keys (scores) or 16 dims (output) as the M rows of
+  // the MMA and the group's heads as the 8 columns, so a tile costs 8 + 8 MMAs.  Column pair
+  // (2 tq, 2 tq + 1) of every accumulator belongs to this lane: two heads, softmax state for each.
+  uint32_t qf[KS][2];     // B operand of the scores: q of head gq, dims 16 ks + 2 tq .. and + 8
+  float o[HD / 16][4];    // out^T: dims gq + 16 i (c0, c1) and gq + 8 + 16 i (c2, c3), heads 2 tq, 2 tq + 1
+  float m2[2] = {-INFINITY, -INFINITY}, l2[2] = {0.f, 0.f};
 
   while (true) {
     // ---- producer: keep up to ATT_NS tiles in flight ----
@@ -234,8 +237,8 @@ __device__ __noinline__ void attn_decode_stream(const DevCtx& c, int layer, char
     const int n_ctx = g_att_nctx[cc.d];
     if (!in_unit) {  // a unit (or this sub-range's part of it) starts here
       in_unit = true;
-      m = -INFINITY;
-      l = 0.f;
+      m2[0] = m2[1] = -INFINITY;
+      l2[0] = l2[1] = 0.f;
       const __nv_bfloat16* qrow = qb + (size_t)t_row * c.q_dim + (size_t)(cc.g * NREP + (live ? gq : 0)) * HD;
 #pragma unroll
       for (int ks = 0; ks < KS; ++ks) {
@@ -243,7 +246,7 @@ __device__ __noinline__ void attn_decode_stream(const DevCtx& c, int layer, char
         qf[ks][1] = live ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 8 + 2 * tq) : 0u;
       }
 #pragma unroll
-      for (int i = 0; i < HD / 8; ++i) { o[i][0] = 0.f; o[i][1] = 0.f; }
+      for (int i = 0; i < HD / 16; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
     }
     const int s = n_consumed % ATT_NS;
     if (!__all_sync(FULL, mbar_wait(c, &bars[s], (as.par >> s) & 1u, dead))) break;  // uniform exit
@@ -260,96 +263,104 @@ __device__ __noinline__ void attn_decode_stream(const DevCtx& c, int layer, char
     }
     // The matrix loads and MMAs below are issued in program order, so all loads of an operand are
     // issued before the MMAs that use them, and V is fetched before the softmax arithmetic.
-    uint32_t kf[KS][4];
+    uint32_t kf[KS][4];    // A operand of the scores: K tile, keys x dims
 #pragma unroll
     for (int ks = 0; ks < KS; ++ks) {
-      const int key = (lane & 7) + ((lane >> 4) & 1) * 8;
-      const int ck = ks * 2 + ((lane >> 3) & 1);
+      const int key = (lane & 7) + ((lane >> 3) & 1) * 8;
+      const int ck = ks * 2 + (lane >> 4);
       const int line = key * NBOX + (ck >> 3);   // 128-byte line of the tile; chunks are swizzled with the line index
       ldsm_x4(kt + line * 128 + (((ck & 7) ^ (line & 7)) << 4), kf[ks][0], kf[ks][1], kf[ks][2], kf[ks][3]);
     }
-    uint32_t vf[HD / 16][4];
+    uint32_t vf[HD / 16][4];   // A operand of the output: V tile transposed, dims x keys
 #pragma unroll
-    for (int dp = 0; dp < HD / 16; ++dp) {
-      const int key = (lane & 7) + ((lane >> 3) & 1) * 8;
-      const int ck = dp * 2 + (lane >> 4);
+    for (int i = 0; i < HD / 16; ++i) {
+      const int key = (lane & 7) + ((lane >> 4) & 1) * 8;
+      const int ck = i * 2 + ((lane >> 3) & 1);
       const int line = key * NBOX + (ck >> 3);
-      ldsm_x4_t(vt + line * 128 + (((ck & 7) ^ (line & 7)) << 4), vf[dp][0], vf[dp][1], vf[dp][2], vf[dp][3]);
+      ldsm_x4_t(vt + line * 128 + (((ck & 7) ^ (line & 7)) << 4), vf[i][0], vf[i][1], vf[i][2], vf[i][3]);
     }
-    // scores of the group's heads against the 16 keys: two n-tiles of 8 keys, two accumulators
-    // each (even and odd k-steps) to halve the dependent chain
+    // scores^T [16 keys][8 heads]: four accumulators (k-step mod 4) keep the dependent chains short
     float sacc[4][4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) { sacc[i][0] = sacc[i][1] = sacc[i][2] = sacc[i][3] = 0.f; }
 #pragma unroll
-    for (int ks = 0; ks < KS; ++ks) {
-      const uint32_t a[4] = {qf[ks][0], 0u, qf[ks][1], 0u};
-      mma_bf16_16816(sacc[(ks & 1) * 2], a, kf[ks][0], kf[ks][1]);
-      mma_bf16_16816(sacc[(ks & 1) * 2 + 1], a, kf[ks][2], kf[ks][3]);
+    for (int ks = 0; ks < KS; ++ks) mma_bf16_16816(sacc[ks & 3], kf[ks], qf[ks][0], qf[ks][1]);
+    float sv[4];   // keys gq (0, 1) and gq + 8 (2, 3), heads 2 tq (0, 2) and 2 tq + 1 (1, 3)
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const float v = (sacc[0][e] + sacc[1][e]) + (sacc[2][e] + sacc[3][e]);
+      sv[e] = (gq + (e >> 1) * 8 < n_valid) ? v * qscale : -INFINITY;
     }
-    sacc[0][0] += sacc[2][0]; sacc[0][1] += sacc[2][1];
-    sacc[1][0] += sacc[3][0]; sacc[1][1] += sacc[3][1];
-    // online softmax of operand row gq over this lane's four keys (2 tq, 2 tq + 1, 8 + 2 tq, 9 + 2 tq)
-    float sv[4];
+    // online softmax per head: maxima over the 16 keys live in the lanes with the same tq
+    float mx0 = fmaxf(sv[0], sv[2]), mx1 = fmaxf(sv[1], sv[3]);
 #pragma unroll
-    for (int nt = 0; nt < 2; ++nt)
-#pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        const int key = nt * 8 + 2 * tq + e;
-        sv[nt * 2 + e] = key < n_valid ? sacc[nt][e] * qscale : -INFINITY;
-      }
-    float mx = fmaxf(fmaxf(sv[0], sv[1]), fmaxf(sv[2], sv[3]));
-    mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, 1));
-    mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, 2));
-    const float mn = fmaxf(m, mx);          // finite: key 0 of the tile is always valid
-    if (__any_sync(FULL, mn > m)) {
-      const float corr = fast_ex2(m - mn);
-      l *= corr;
-#pragma unroll
-      for (int i = 0; i < HD / 8; ++i) { o[i][0] *= corr; o[i][1] *= corr; }
+    for (int sh = 4; sh <= 16; sh <<= 1) {
+      mx0 = fmaxf(mx0, __shfl_xor_sync(FULL, mx0, sh));
+      mx1 = fmaxf(mx1, __shfl_xor_sync(FULL, mx1, sh));
     }
-    m = mn;
-    const float p0 = fast_ex2(sv[0] - mn), p1 = fast_ex2(sv[1] - mn), p2 = fast_ex2(sv[2] - mn), p3 = fast_ex2(sv[3] - mn);
-    l += (p0 + p1) + (p2 + p3);
-    const uint32_t pa[4] = {pack_bf2(p0, p1), 0u, pack_bf2(p2, p3), 0u};
-    // out += P V: n-tiles of 8 dims, one k-step of 16 keys
+    const float mn0 = fmaxf(m2[0], mx0), mn1 = fmaxf(m2[1], mx1);   // finite: key 0 of the tile is always valid
+    if (__any_sync(FULL, mn0 > m2[0] || mn1 > m2[1])) {
+      const float c0 = fast_ex2(m2[0] - mn0), c1 = fast_ex2(m2[1] - mn1);
+      l2[0] *= c0; l2[1] *= c1;
 #pragma unroll
-    for (int dp = 0; dp < HD / 16; ++dp) {
-      float d0[4] = {o[2 * dp][0], o[2 * dp][1], 0.f, 0.f};
-      float d1[4] = {o[2 * dp + 1][0], o[2 * dp + 1][1], 0.f, 0.f};
-      mma_bf16_16816(d0, pa, vf[dp][0], vf[dp][1]);
-      mma_bf16_16816(d1, pa, vf[dp][2], vf[dp][3]);
-      o[2 * dp][0] = d0[0]; o[2 * dp][1] = d0[1];
-      o[2 * dp + 1][0] = d1[0]; o[2 * dp + 1][1] = d1[1];
+      for (int i = 0; i < HD / 16; ++i) { o[i][0] *= c0; o[i][1] *= c1; o[i][2] *= c0; o[i][3] *= c1; }
     }
+    m2[0] = mn0; m2[1] = mn1;
+    const float p0 = fast_ex2(sv[0] - mn0), p1 = fast_ex2(sv[1] - mn1), p2 = fast_ex2(sv[2] - mn0), p3 = fast_ex2(sv[3] - mn1);
+    l2[0] += p0 + p2;
+    l2[1] += p1 + p3;
+    // P^T as the B operand of the output: transpose the two 8 x 8 (key, head) blocks in registers
+    uint32_t pb0, pb1;
+    {
+      const uint32_t plo = pack_bf2(p0, p1), phi = pack_bf2(p2, p3);
+      asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(pb0) : "r"(plo));
+      asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(pb1) : "r"(phi));
+    }
+    // out^T += V^T P^T: 16 dims per MMA, one k-step of 16 keys
+#pragma unroll
+    for (int i = 0; i < HD / 16; ++i) mma_bf16_16816(o[i], vf[i], pb0, pb1);
     __syncwarp();  // all reads of this stage are done before it is refilled
     n_consumed += 1;
 
     const bool unit_ends = (cc.kb == cc.nkb - 1) || (cc.f + 1 == cc.f_end);
     if (unit_ends) {
       in_unit = false;
-      float lt = l;
-      lt += __shfl_xor_sync(FULL, lt, 1);
-      lt += __shfl_xor_sync(FULL, lt, 2);
+      float lt0 = l2[0], lt1 = l2[1];   // sums over the keys: lanes with the same tq
+#pragma unroll
+      for (int sh = 4; sh <= 16; sh <<= 1) {
+        lt0 += __shfl_xor_sync(FULL, lt0, sh);
+        lt1 += __shfl_xor_sync(FULL, lt1, sh);
+      }
       const int us = Hkv * g_att_pre[cc.d] + cc.g * cc.nkb, ue = us + cc.nkb;
       const int j_first = us / S, j_last = (ue - 1) / S;
+      const int h0 = 2 * tq;   // this lane's heads: h0, h0 + 1
       if ((ATT_SNAP && cc.nkb <= 2 * S) || j_first == j_last) {   // the whole unit was handled here
-        if (live) {
-          const float inv = 1.0f / lt;
-          __nv_bfloat16* orow = out + (size_t)t_row * c.q_dim + (size_t)(cc.g * NREP + gq) * HD;
+        __nv_bfloat16* obase = out + (size_t)t_row * c.q_dim + (size_t)(cc.g * NREP) * HD;
 #pragma unroll
-          for (int i = 0; i < HD / 8; ++i)
-            *reinterpret_cast<uint32_t*>(orow + i * 8 + 2 * tq) = pack_bf2(o[i][0] * inv, o[i][1] * inv);
+        for (int e = 0; e < 2; ++e) {
+          if (h0 + e < NREP) {
+            const float inv = 1.0f / (e ? lt1 : lt0);
+#pragma unroll
+            for (int i = 0; i < HD / 16; ++i) {
+              obase[(h0 + e) * HD + 16 * i + gq] = __float2bfloat16_rn(o[i][e] * inv);
+              obase[(h0 + e) * HD + 16 * i + 8 + gq] = __float2bfloat16_rn(o[i][2 + e] * inv);
+            }
+          }
         }
       } else {
         // partial record: [NREP][HD] accumulators, then m[NREP], then l[NREP]
         const int unit = cc.d * Hkv + cc.g;
         float* rec = c.att_part + (size_t)(2 * sub_id + (us <= sub_start ? 0 : 1)) * REC;
-        if (live) {
 #pragma unroll
-          for (int i = 0; i < HD / 8; ++i)
-            *reinterpret_cast<float2*>(rec + gq * HD + i * 8 + 2 * tq) = make_float2(o[i][0], o[i][1]);
-          if (tq == 0) { rec[NREP * HD + gq] = m; rec[NREP * HD + NREP + gq] = lt; }
+        for (int e = 0; e < 2; ++e) {
+          if (h0 + e < NREP) {
+#pragma unroll
+            for (int i = 0; i < HD / 16; ++i) {
+              rec[(h0 + e) * HD + 16 * i + gq] = o[i][e];
+              rec[(h0 + e) * HD + 16 * i + 8 + gq] = o[i][2 + e];
+            }
+            if (gq == 0) { rec[NREP * HD + h0 + e] = m2[e]; rec[NREP * HD + NREP + h0 + e] = e ? lt1 : lt0; }
+          }
         }
         __threadfence();
         __syncwarp();
