@@ -232,6 +232,19 @@ def decode_point(B, m, sched, wbuf, kv, wl, gemm_impl, n, in_len, out_len, steps
                 tok_s=float(its["n_sample_rows"].sum() / (ms / 1e3)))
 
 
+def reduce_over_ranks(ms, tokens, device, world):
+    """Replicas exchange nothing on the data path; only the report is combined: the job's time is the
+    slowest rank's, its tokens the sum over ranks.  Works on any backend (nccl on GPUs, gloo on CPU)."""
+    import torch
+    t_ms = torch.tensor([ms], dtype=torch.float64, device=device)
+    tok = torch.tensor([tokens], dtype=torch.float64, device=device)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t_ms, op=dist.ReduceOp.MAX)
+        dist.all_reduce(tok, op=dist.ReduceOp.SUM)
+    return float(t_ms.item()), float(tok.item())
+
+
 def percentiles(x):
     if len(x) == 0:
         return dict(p50=None, p99=None, mean=None)
@@ -352,7 +365,7 @@ def main():
             cb, res, dt = cpu_oracle_sample(m, sched, wbuf, n_req, cap, new, cfg_i)
             vals.append(cb["value"])
         cb["value"] = float(np.median(vals))
-        line = dict(impl="reference", metric="output tok/s", value=cb["value"], unit="tok/s", n_gpus=0,
+        line = dict(impl="reference", metric="output tok/s", value=cb["value"], unit="tok/s", n_gpus=args.gpus,
                     steps=args.steps, warmup=args.warmup, ms_per_step=dt * 1e3 / max(1, len(res["trace"])),
                     higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f32", data="synthetic",
                     config=dict(workload=workload + " (bounded sample, CPU oracle)"), cpu_baseline=cb,
@@ -478,12 +491,7 @@ def main():
     tokens_out = int(its["n_sample_rows"].sum())
     by, fl = step_bytes_flops(m, its)
     pk = measured_peaks()
-    t_ms = torch.tensor([ms], dtype=torch.float64, device=dev)
-    tok = torch.tensor([tokens_out], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t_ms, op=dist.ReduceOp.MAX)
-        dist.all_reduce(tok, op=dist.ReduceOp.SUM)
-    ms_max, tok_all = float(t_ms.item()), float(tok.item())
+    ms_max, tok_all = reduce_over_ranks(ms, tokens_out, dev, world)
     value = tok_all / (ms_max / 1e3)
 
     bound_hbm_s = by / (pk["hbm_gbs"] * 1e9)

@@ -20,7 +20,6 @@ namespace blink {
 
 constexpr int ATT_NS = 3;  // ring stages per warp (decode path)
 constexpr int ATT_WARPS = FWD_THREADS / 32;
-constexpr bool ATT_SNAP = false;  // keep units of at most 2 S tiles whole (see dec_bound)
 
 struct AttShared {
   uint64_t bar[ATT_WARPS][ATT_NS];
@@ -47,13 +46,6 @@ __device__ __forceinline__ void att_init(const DevCtx& c, AttState& s) {
   }
   if (threadIdx.x == 0) g_att.dead = 0;
   __syncthreads();
-}
-
-__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                   smem_u32(dst)),
-               "l"(src), "r"(bytes), "r"(smem_u32(bar))
-               : "memory");
 }
 
 __device__ __forceinline__ float fast_ex2(float x) {
@@ -104,16 +96,6 @@ __device__ __forceinline__ void dec_advance(DecCursor& cur, int n_dec, int Hkv) 
       if (cur.d < n_dec) cur.nkb = g_att_pre[cur.d + 1] - g_att_pre[cur.d];
     }
   }
-}
-
-// Sub-range j of the flat tile sequence is [dec_bound(j S), dec_bound((j + 1) S)): a boundary that
-// would cut a unit of at most 2 S tiles moves to the end of that unit, so only long units are
-// ever split (and leave partial records); short ones stay with the sub-range they start in.
-__device__ __forceinline__ int dec_bound(int x, int S, int TT, int n_dec, int Hkv) {
-  if (x >= TT) return TT;
-  DecCursor t;
-  dec_seek(t, x, x, n_dec, Hkv);
-  return (ATT_SNAP && t.kb > 0 && t.nkb <= 2 * S) ? x + (t.nkb - t.kb) : x;
 }
 
 // ---- tensor-core and matrix-load wrappers ---------------------------------------------------------
@@ -197,8 +179,8 @@ __device__ __noinline__ void attn_decode_stream(const DevCtx& c, int layer, char
             id = __shfl_sync(FULL, id, 0);
           }
           if (id >= n_sub) { p_done = true; break; }
-          b0 = dec_bound(id * S, S, TT, n_dec, Hkv);
-          b1 = dec_bound(id * S + S, S, TT, n_dec, Hkv);
+          b0 = id * S;
+          b1 = min(TT, id * S + S);
           if (b0 < b1) break;
         }
         if (p_done) break;
@@ -230,7 +212,7 @@ __device__ __noinline__ void attn_decode_stream(const DevCtx& c, int layer, char
       sub_id = g_att.ids[w][c_k & 7];
       c_k += 1;
       sub_start = sub_id * S;
-      dec_seek(cc, dec_bound(sub_start, S, TT, n_dec, Hkv), dec_bound(sub_start + S, S, TT, n_dec, Hkv), n_dec, Hkv);
+      dec_seek(cc, sub_start, min(TT, sub_start + S), n_dec, Hkv);
       in_unit = false;
     }
     const int t_row = g_att_row[cc.d];
@@ -334,7 +316,7 @@ __device__ __noinline__ void attn_decode_stream(const DevCtx& c, int layer, char
       const int us = Hkv * g_att_pre[cc.d] + cc.g * cc.nkb, ue = us + cc.nkb;
       const int j_first = us / S, j_last = (ue - 1) / S;
       const int h0 = 2 * tq;   // this lane's heads: h0, h0 + 1
-      if ((ATT_SNAP && cc.nkb <= 2 * S) || j_first == j_last) {   // the whole unit was handled here
+      if (j_first == j_last) {   // the whole unit was handled here
         __nv_bfloat16* obase = out + (size_t)t_row * c.q_dim + (size_t)(cc.g * NREP) * HD;
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
