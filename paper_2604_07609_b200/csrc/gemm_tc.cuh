@@ -8,7 +8,8 @@
 // steps have few tokens and stream every weight once, so the weight tile fills the fixed
 // 128-row dimension and the token count only sets the cheap N.
 //
-// Work split ("stream-K"): the (pass, n-tile, k-block) units of one GEMM are flattened and
+// Work split ("stream-K"): the (n-tile, token pass, k-block) units of one GEMM are flattened (the
+// passes of a weight tile follow each other, so the later ones can find it in L2) and
 // cut into gridDim.x equal contiguous ranges, so every SM streams the same number of weight
 // bytes whatever the shape.  A CTA's range is a handful of segments (one n-tile each); a
 // segment that covers the whole K of its tile stores its result, a partial one adds it
@@ -248,7 +249,7 @@ __device__ __forceinline__ void tc_produce_weights(const DevCtx& c, const void* 
     const long long seg_end = min(g.u1, (u / g.kblocks + 1) * (long long)g.kblocks);
     const int nk = (int)min((long long)g.KPS, seg_end - u);
     const int kb = (int)(u % g.kblocks);
-    const int nt = (int)((u / g.kblocks) % g.ntiles);
+    const int nt = (int)(u / ((long long)g.kblocks * g.passes));   // unit order: n-tile, token pass, k-block
     // the n-th fill of a stage waits for its (n-1)-th release
     if (!mbar_wait(c, &g_tc.empty[stage], ((tc.fill_bits >> stage) & 1u) ^ 1u, dead)) break;
     tc.fill_bits ^= 1u << stage;
@@ -293,7 +294,7 @@ static __device__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int whi
         const long long seg_end = min(u1, (u / kblocks + 1) * (long long)kblocks);
         const int nk = (int)min((long long)KPS, seg_end - u);
         const int kb = (int)(u % kblocks);
-        const int pass = (int)(u / ((long long)kblocks * ntiles));
+        const int pass = (int)((u / kblocks) % g.passes);
         if (!mbar_wait(c, &g_tc.empty[stage], ((tc.fill_bits >> stage) & 1u) ^ 1u, dead)) break;
         tc.fill_bits ^= 1u << stage;
         char* sa = tiles + (size_t)stage * stage_bytes;
@@ -311,7 +312,7 @@ static __device__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int whi
       long long u = u0;
       while (u < u1) {
         const long long seg_end = min(u1, (u / kblocks + 1) * (long long)kblocks);
-        const int pass = (int)(u / ((long long)kblocks * ntiles));
+        const int pass = (int)((u / kblocks) % g.passes);
         const int rows = min(256, T - pass * 256);
         const int n_mma = (rows + 15) & ~15;
         const uint32_t idesc = idesc_bf16(n_mma);
@@ -354,8 +355,8 @@ static __device__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int whi
       const long long seg_end = min(u1, (u / kblocks + 1) * (long long)kblocks);
       const int kb0 = (int)(u % kblocks);
       const int kb1 = kb0 + (int)(seg_end - u);
-      const int nt = (int)((u / kblocks) % ntiles);
-      const int pass = (int)(u / ((long long)kblocks * ntiles));
+      const int nt = (int)(u / ((long long)kblocks * g.passes));
+      const int pass = (int)((u / kblocks) % g.passes);
       const int rows = min(256, T - pass * 256);
       const int n_mma = (rows + 15) & ~15;
       const bool whole = (kb0 == 0 && kb1 == kblocks);
