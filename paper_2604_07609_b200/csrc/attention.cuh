@@ -59,11 +59,11 @@ __device__ __forceinline__ uint32_t pack_bf2(float lo, float hi) {
 }
 // one TMA tile copy from a rank-5 tensor map
 __device__ __forceinline__ void tma_load_5d(void* smem_dst, const CUtensorMap* map, int c0, int c1, int c2, int c3, int c4,
-                                            uint64_t* bar) {
+                                            uint64_t* bar, uint64_t policy) {
   asm volatile(
-      "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];" ::"r"(
-          smem_u32(smem_dst)),
-      "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(smem_u32(bar))
+      "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4, "
+      "%5, %6}], [%7], %8;" ::"r"(smem_u32(smem_dst)),
+      "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(smem_u32(bar)), "l"(policy)
       : "memory");
 }
 
@@ -149,6 +149,7 @@ __device__ __noinline__ void attn_decode_stream(const DevCtx& c, int layer, char
   __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(c.attn);
   const float qscale = c.attn_scale * 1.4426950408889634f;
   const uint32_t ring_s = smem_u32(ring);
+  const uint64_t kv_policy = l2_evict_first();   // the cache is read once per step
 
   int n_issued = 0, n_consumed = 0, p_k = 0, c_k = 0;
   bool p_done = false, first_fetch = true;
@@ -200,7 +201,7 @@ __device__ __noinline__ void attn_decode_stream(const DevCtx& c, int layer, char
         const int s = n_issued % ATT_NS;
         // one copy brings the K tile and the V tile: box {64 dims, NBOX halves, 16 keys, K and V, this layer}
         mbar_expect_tx(&bars[s], STAGE);
-        tma_load_5d(ring + s * STAGE, kv_map, 0, 0, (blk * Hkv + pc.g) * 16, 0, layer, &bars[s]);
+        tma_load_5d(ring + s * STAGE, kv_map, 0, 0, (blk * Hkv + pc.g) * 16, 0, layer, &bars[s], kv_policy);
       }
       dec_advance(pc, n_dec, Hkv);
       n_issued += 1;

@@ -108,6 +108,31 @@ __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* m
       : "memory");
 }
 
+// L2 policy for data that is read once per step (weights, the KV cache): evicted first, so that
+// the streams do not push the step's activations out of L2.  Reductions into an evicted output
+// line have to fetch it from HBM first and run several times slower.
+__device__ __forceinline__ uint64_t l2_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ void tma_load_2d_hint(void* smem_dst, const CUtensorMap* map, int x, int y, uint64_t* bar,
+                                                 uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], "
+      "[%4], %5;" ::"r"(smem_u32(smem_dst)),
+      "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)), "l"(policy)
+      : "memory");
+}
+__device__ __forceinline__ void tma_bulk_load_hint(void* smem_dst, const void* src, uint32_t bytes, uint64_t* bar,
+                                                   uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(
+          smem_u32(smem_dst)),
+      "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(policy)
+      : "memory");
+}
+
 __device__ __forceinline__ void tma_bulk_load(void* smem_dst, const void* src, uint32_t bytes, uint64_t* bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
                    smem_u32(smem_dst)),
@@ -243,6 +268,7 @@ __device__ __forceinline__ void tc_produce_weights(const DevCtx& c, const void* 
   const CUtensorMap* map_a = &maps->w[which];
   const int row_a0 = (int)w_row0;
   volatile int* dead = &g_tc.dead;
+  const uint64_t stream_policy = l2_evict_first();
   long long u = g.u0;
   int stage = 0;
   while (u < g.u1) {
@@ -256,10 +282,10 @@ __device__ __forceinline__ void tc_produce_weights(const DevCtx& c, const void* 
     char* sa = tiles + (size_t)stage * g.stage_bytes;
     mbar_expect_tx(&g_tc.full[stage], (uint32_t)nk * TC_A_BYTES);
     if (c.w_streaming) {  // contiguous tiles, already in the shared-memory operand image
-      tma_bulk_load(sa, reinterpret_cast<const char*>(w) + ((size_t)nt * g.kblocks + kb) * TC_A_BYTES,
-                    (uint32_t)nk * TC_A_BYTES, &g_tc.full[stage]);
+      tma_bulk_load_hint(sa, reinterpret_cast<const char*>(w) + ((size_t)nt * g.kblocks + kb) * TC_A_BYTES,
+                         (uint32_t)nk * TC_A_BYTES, &g_tc.full[stage], stream_policy);
     } else {
-      tma_load_2d(sa, map_a, kb * 64, row_a0 + nt * 128, &g_tc.full[stage]);
+      tma_load_2d_hint(sa, map_a, kb * 64, row_a0 + nt * 128, &g_tc.full[stage], stream_policy);
     }
     u += nk;
     if (++stage == g.S) stage = 0;
@@ -288,6 +314,7 @@ static __device__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int whi
   } else if (warp == 2) {
     // token-tile producer: walks the same sequence of stages (nk k-blocks of one segment each)
     if (lane == 0) {
+      const int x_row0 = a.x_row0;
       int stage = 0;
       long long u = u0;
       while (u < u1) {
@@ -300,7 +327,7 @@ static __device__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int whi
         char* sa = tiles + (size_t)stage * stage_bytes;
         mbar_expect_tx(&g_tc.full[stage], (uint32_t)nk * b_bytes);
         for (int j = 0; j < nk; ++j)
-          tma_load_2d(sa + KPS * TC_A_BYTES + j * b_bytes, map_b, (kb + j) * 64, a.x_row0 + pass * 256, &g_tc.full[stage]);
+          tma_load_2d(sa + KPS * TC_A_BYTES + j * b_bytes, map_b, (kb + j) * 64, x_row0 + pass * 256, &g_tc.full[stage]);
         u += nk;
         if (++stage == S) stage = 0;
       }
@@ -349,6 +376,13 @@ static __device__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int whi
     }
   } else if (warp >= 4) {
     const int q = warp & 3;  // TMEM lane quarter this warp may read
+    // the arguments live in the caller's frame: keep what the store loops need in registers, or
+    // every reduction is followed by reloads that the next one depends on
+    float* const out = a.out;
+    const size_t ldo = (size_t)a.ldo;
+    const int* const row_map = a.row_map;
+    const float* const row_scale = a.row_scale;
+    const bool accumulate = a.accumulate != 0;
     int abuf = 0;
     long long u = u0;
     while (u < u1) {
@@ -359,7 +393,7 @@ static __device__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int whi
       const int pass = (int)((u / kblocks) % g.passes);
       const int rows = min(256, T - pass * 256);
       const int n_mma = (rows + 15) & ~15;
-      const bool whole = (kb0 == 0 && kb1 == kblocks);
+      const bool plain = (kb0 == 0 && kb1 == kblocks) && !accumulate && row_map == nullptr;
       if (!mbar_wait(c, &g_tc.acc_full[abuf], (tc.acc_epi >> abuf) & 1u, dead)) break;
       tc.acc_epi ^= 1u << abuf;
       tc_fence_after();
@@ -369,17 +403,22 @@ static __device__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int whi
         float v[16];
         tmem_ld16(taddr + (uint32_t)c0, v);
         if (n < N) {
+          const int t0 = pass * 256 + c0;
+          const int nv = min(16, T - t0);   // token rows of this group that exist
+          if (row_map != nullptr) {
 #pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            const int t = pass * 256 + c0 + j;
-            if (t < T) {
-              if (a.row_map != nullptr) {
-                atomicAdd(a.out + (size_t)a.row_map[t] * a.ldo + n, a.row_scale[t] * v[j]);
-              } else {
-                float* o = a.out + (size_t)t * a.ldo + n;
-                if (whole && !a.accumulate) *o = v[j];
-                else atomicAdd(o, v[j]);
-              }
+            for (int j = 0; j < 16; ++j)
+              if (j < nv) atomicAdd(out + (size_t)row_map[t0 + j] * ldo + n, row_scale[t0 + j] * v[j]);
+          } else {
+            float* o = out + (size_t)t0 * ldo + n;
+            if (plain) {
+#pragma unroll
+              for (int j = 0; j < 16; ++j)
+                if (j < nv) o[(size_t)j * ldo] = v[j];
+            } else {
+#pragma unroll
+              for (int j = 0; j < 16; ++j)
+                if (j < nv) atomicAdd(o + (size_t)j * ldo, v[j]);
             }
           }
         }
