@@ -158,6 +158,10 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
                : "memory");
 }
+// fp32 reduction into global memory, no return value (the pointer is known to be global here)
+__device__ __forceinline__ void red_add_f32(float* p, float v) {
+  asm volatile("red.relaxed.gpu.global.add.f32 [%0], %1;" ::"l"(__cvta_generic_to_global(p)), "f"(v) : "memory");
+}
 // 32 lanes x 16 consecutive 32-bit columns -> 16 registers per thread
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
   uint32_t r[16];
@@ -408,7 +412,7 @@ static __device__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int whi
           if (row_map != nullptr) {
 #pragma unroll
             for (int j = 0; j < 16; ++j)
-              if (j < nv) atomicAdd(out + (size_t)row_map[t0 + j] * ldo + n, row_scale[t0 + j] * v[j]);
+              if (j < nv) red_add_f32(out + (size_t)row_map[t0 + j] * ldo + n, row_scale[t0 + j] * v[j]);
           } else {
             float* o = out + (size_t)t0 * ldo + n;
             if (plain) {
@@ -418,7 +422,7 @@ static __device__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int whi
             } else {
 #pragma unroll
               for (int j = 0; j < 16; ++j)
-                if (j < nv) atomicAdd(o + (size_t)j * ldo, v[j]);
+                if (j < nv) red_add_f32(o + (size_t)j * ldo, v[j]);
             }
           }
         }
