@@ -193,6 +193,22 @@ __device__ __forceinline__ uint32_t idesc_bf16(int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 }
 
+// The same wait for warps that have nothing else to do for most of a phase: sleep between polls.
+__device__ __forceinline__ bool mbar_wait_idle(const DevCtx& c, uint64_t* bar, uint32_t parity, volatile int* dead) {
+  if (*dead) return false;
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity)) {
+    __nanosleep(200);
+    if (*dead) return false;
+    if ((unsigned long long)(clock64() - t0) > c.barrier_timeout_cycles) {
+      *dead = 1;
+      dev_fail(c, DEV_ERR_PIPE_TIMEOUT);
+      return false;
+    }
+  }
+  return true;
+}
+
 // ---- TMEM allocation for the life of the kernel ---------------------------------------------
 __device__ __forceinline__ void tc_init(const DevCtx& c, float*, TcState& s) {
   s.tmem_base = 0;
@@ -229,6 +245,47 @@ struct TcMaps {
   CUtensorMap act[ACT_BUFS][TC_BOXES];
 };
 
+// Where the epilogue's results go; held in registers by the warps that store (the arguments live
+// in the caller's frame, and a reload after every reduction would serialise them).
+struct TcEpiOut {
+  float* out;
+  size_t ldo;
+  const int* row_map;
+  const float* row_scale;
+  int T, N;
+};
+// columns [c_begin, c_end) of an accumulator (token rows t_base + column) -> out; lane = weight row n
+__device__ __forceinline__ void tc_epi_columns(const TcEpiOut& e, uint32_t taddr, int n, int t_base, int c_begin, int c_end,
+                                               bool plain) {
+  for (int c0 = c_begin; c0 < c_end; c0 += 16) {
+    float v[16];
+    tmem_ld16(taddr + (uint32_t)c0, v);
+    if (n < e.N) {
+      const int t0 = t_base + c0;
+      const int nv = min(16, e.T - t0);   // token rows of this group that exist
+      if (e.row_map != nullptr) {
+#pragma unroll
+        for (int j = 0; j < 16; ++j)
+          if (j < nv) red_add_f32(e.out + (size_t)e.row_map[t0 + j] * e.ldo + n, e.row_scale[t0 + j] * v[j]);
+      } else {
+        float* o = e.out + (size_t)t0 * e.ldo + n;
+        if (plain) {
+#pragma unroll
+          for (int j = 0; j < 16; ++j)
+            if (j < nv) o[(size_t)j * e.ldo] = v[j];
+        } else {
+#pragma unroll
+          for (int j = 0; j < 16; ++j)
+            if (j < nv) red_add_f32(o + (size_t)j * e.ldo, v[j]);
+        }
+      }
+    }
+  }
+}
+// First column of a CTA's last accumulator that warps 0-3 store (they have no role left by
+// then).  Below 128 columns the reduction is short and the extra waiting warps cost more.
+__device__ __forceinline__ int tc_epi_half(int n_mma) { return n_mma >= 128 ? ((n_mma / 16 + 1) / 2) * 16 : n_mma; }
+
 // ---- the GEMM phase -----------------------------------------------------------------------------
 // Shape of one GEMM's pipeline for the current step; every role derives the same numbers.
 struct TcGeom {
@@ -257,6 +314,24 @@ __device__ __forceinline__ TcGeom tc_geom(const DevCtx& c, int T, int N, int K) 
   const long long total = (long long)g.passes * g.ntiles * g.kblocks;
   g.u0 = total * blockIdx.x / gridDim.x;
   g.u1 = total * (blockIdx.x + 1) / gridDim.x;
+  // Few weight tiles (QKV, O, down at decode sizes): give every tile the same whole number of
+  // CTAs, so that no CTA's range crosses a tile and each has one partial tile to reduce at the
+  // end instead of two.  The longest range grows by (per * grid - total) / grid k-blocks of about
+  // 0.4 us each; the saved reduction takes about 0.018 us per token row.
+  const int split = (int)gridDim.x / g.ntiles;
+  if (g.passes == 1 && split >= 2) {
+    const int per = (g.kblocks + split - 1) / split;
+    if (((long long)per * gridDim.x - total) * 23 < (long long)T * gridDim.x) {
+      const int b = (int)blockIdx.x;
+      if (b < g.ntiles * split) {
+        const int nt = b / split, part = b % split;
+        g.u0 = (long long)nt * g.kblocks + (long long)g.kblocks * part / split;
+        g.u1 = (long long)nt * g.kblocks + (long long)g.kblocks * (part + 1) / split;
+      } else {
+        g.u0 = g.u1 = 0;
+      }
+    }
+  }
   return g;
 }
 // tiles need 1024-byte alignment for the 128-byte swizzle
@@ -380,12 +455,7 @@ static __device__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int whi
     }
   } else if (warp >= 4) {
     const int q = warp & 3;  // TMEM lane quarter this warp may read
-    // the arguments live in the caller's frame: keep what the store loops need in registers, or
-    // every reduction is followed by reloads that the next one depends on
-    float* const out = a.out;
-    const size_t ldo = (size_t)a.ldo;
-    const int* const row_map = a.row_map;
-    const float* const row_scale = a.row_scale;
+    const TcEpiOut eo{a.out, (size_t)a.ldo, a.row_map, a.row_scale, T, N};
     const bool accumulate = a.accumulate != 0;
     int abuf = 0;
     long long u = u0;
@@ -397,41 +467,51 @@ static __device__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int whi
       const int pass = (int)((u / kblocks) % g.passes);
       const int rows = min(256, T - pass * 256);
       const int n_mma = (rows + 15) & ~15;
-      const bool plain = (kb0 == 0 && kb1 == kblocks) && !accumulate && row_map == nullptr;
+      const bool plain = (kb0 == 0 && kb1 == kblocks) && !accumulate && eo.row_map == nullptr;
       if (!mbar_wait(c, &g_tc.acc_full[abuf], (tc.acc_epi >> abuf) & 1u, dead)) break;
       tc.acc_epi ^= 1u << abuf;
       tc_fence_after();
-      const int n = nt * 128 + q * 32 + lane;
       const uint32_t taddr = tc.tmem_base + (uint32_t)abuf * 256u + ((uint32_t)(q * 32) << 16);
-      for (int c0 = 0; c0 < n_mma; c0 += 16) {
-        float v[16];
-        tmem_ld16(taddr + (uint32_t)c0, v);
-        if (n < N) {
-          const int t0 = pass * 256 + c0;
-          const int nv = min(16, T - t0);   // token rows of this group that exist
-          if (row_map != nullptr) {
-#pragma unroll
-            for (int j = 0; j < 16; ++j)
-              if (j < nv) red_add_f32(out + (size_t)row_map[t0 + j] * ldo + n, row_scale[t0 + j] * v[j]);
-          } else {
-            float* o = out + (size_t)t0 * ldo + n;
-            if (plain) {
-#pragma unroll
-              for (int j = 0; j < 16; ++j)
-                if (j < nv) o[(size_t)j * ldo] = v[j];
-            } else {
-#pragma unroll
-              for (int j = 0; j < 16; ++j)
-                if (j < nv) red_add_f32(o + (size_t)j * ldo, v[j]);
-            }
-          }
-        }
-      }
+      // the upper columns of the CTA's last accumulator are left to warps 0-3
+      const int c_end = (seg_end == u1) ? tc_epi_half(n_mma) : n_mma;
+      tc_epi_columns(eo, taddr, nt * 128 + q * 32 + lane, pass * 256, 0, c_end, plain);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&g_tc.acc_empty[abuf]);
       abuf ^= 1;
       u = seg_end;
+    }
+  }
+  if (warp < 4) {
+    // Producers and the MMA issuer are done once the last MMA is committed: their warps store
+    // the upper columns of the last accumulator.  Every thread walks the segments to keep its
+    // copy of the accumulator parities in step with the epilogue warps.
+    __syncwarp();
+    int abuf = 0, last_abuf = -1;
+    uint32_t last_par = 0;
+    long long last_u = 0;
+    for (long long u = u0; u < u1;) {
+      last_abuf = abuf;
+      last_par = (tc.acc_epi >> abuf) & 1u;
+      last_u = u;
+      tc.acc_epi ^= 1u << abuf;
+      abuf ^= 1;
+      u = min(u1, (u / kblocks + 1) * (long long)kblocks);
+    }
+    if (last_abuf >= 0) {
+      const int kb0 = (int)(last_u % kblocks);
+      const int nt = (int)(last_u / ((long long)kblocks * g.passes));
+      const int pass = (int)((last_u / kblocks) % g.passes);
+      const int n_mma = (min(256, T - pass * 256) + 15) & ~15;
+      const int c_begin = tc_epi_half(n_mma);
+      if (c_begin < n_mma && mbar_wait_idle(c, &g_tc.acc_full[last_abuf], last_par, dead)) {
+        tc_fence_after();
+        const TcEpiOut eo{a.out, (size_t)a.ldo, a.row_map, a.row_scale, T, N};
+        const bool plain = (kb0 == 0 && (long long)kb0 + (u1 - last_u) == kblocks) && a.accumulate == 0 && eo.row_map == nullptr;
+        const uint32_t taddr = tc.tmem_base + (uint32_t)last_abuf * 256u + ((uint32_t)(warp * 32) << 16);
+        tc_epi_columns(eo, taddr, nt * 128 + warp * 32 + lane, pass * 256, c_begin, n_mma, plain);
+        tc_fence_before();
+      }
     }
   }
   __syncthreads();
