@@ -8,16 +8,19 @@
 // steps have few tokens and stream every weight once, so the weight tile fills the fixed
 // 128-row dimension and the token count only sets the cheap N.
 //
-// Work split ("stream-K"): the (n-tile, token pass, k-block) units of one GEMM are flattened (the
-// passes of a weight tile follow each other, so the later ones can find it in L2) and
-// cut into gridDim.x equal contiguous ranges, so every SM streams the same number of weight
-// bytes whatever the shape.  A CTA's range is a handful of segments (one n-tile each); a
-// segment that covers the whole K of its tile stores its result, a partial one adds it
-// with red.global.add.f32 (the output is zeroed or already holds the residual).
+// Work split ("stream-K"): the (n-tile, k-block) units of one GEMM are flattened and cut into
+// equal contiguous ranges, one per CTA, so every SM streams the same number of weight bytes
+// whatever the shape.  A CTA's range is a handful of segments (one n-tile each); a segment that
+// covers the whole K of its tile stores its result, a partial one adds it with
+// red.global.add.f32 (the output is zeroed or already holds the residual).  With few n-tiles
+// every tile gets the same whole number of CTAs (one partial tile per CTA); with more than 256
+// token rows the passes of a weight tile go to neighbouring CTAs that walk the same range at the
+// same time (the tile comes from HBM once, from L2 for the other passes).
 //
-// Warp roles in the 256-thread CTA: warp 0 = TMA producer (one lane), warp 1 = MMA issuer
-// (one lane), warps 4..7 = epilogue (TMEM -> registers -> global), two accumulator buffers
-// of 256 TMEM columns so the epilogue of one segment overlaps the MMAs of the next.
+// Warp roles in the 256-thread CTA: warp 0 = weight producer (one lane), warp 2 = token-tile
+// producer (one lane), warp 1 = MMA issuer (one lane), warps 4..7 = epilogue (TMEM -> registers
+// -> global), two accumulator buffers of 256 TMEM columns so the epilogue of one segment
+// overlaps the MMAs of the next; warps 0..3 store half of the CTA's last accumulator.
 // Every wait is bounded: on a time-out the CTA records DEV_ERR_PIPE_TIMEOUT, raises the
 // loop's abort flag and skips all further waits.
 #pragma once
@@ -290,6 +293,7 @@ __device__ __forceinline__ int tc_epi_half(int n_mma) { return n_mma >= 128 ? ((
 // Shape of one GEMM's pipeline for the current step; every role derives the same numbers.
 struct TcGeom {
   int kblocks, ntiles, passes, box_id, box_rows, KPS, S;
+  int pass_fixed, pdiv;   // one token pass per CTA (or -1), and the passes interleaved in its unit order
   uint32_t b_bytes, stage_bytes;
   long long u0, u1;
 };
@@ -314,6 +318,27 @@ __device__ __forceinline__ TcGeom tc_geom(const DevCtx& c, int T, int N, int K) 
   const long long total = (long long)g.passes * g.ntiles * g.kblocks;
   g.u0 = total * blockIdx.x / gridDim.x;
   g.u1 = total * (blockIdx.x + 1) / gridDim.x;
+  g.pass_fixed = -1;
+  g.pdiv = g.passes;
+  // More than 256 token rows: the passes of a weight tile go to neighbouring CTAs, which walk the
+  // same (weight tile, k-block) range at the same time, so the tile comes from HBM once and from
+  // L2 for the others.  One CTA doing the passes in turn re-reads it after the whole grid has
+  // streamed more than L2 holds in between.
+  if (g.passes > 1 && (int)gridDim.x >= g.passes) {
+    const int groups = (int)gridDim.x / g.passes;
+    const int b = (int)blockIdx.x;
+    const long long units = (long long)g.ntiles * g.kblocks;
+    g.pdiv = 1;
+    if (b < groups * g.passes) {
+      const int grp = b / g.passes;
+      g.pass_fixed = b % g.passes;
+      g.u0 = units * grp / groups;
+      g.u1 = units * (grp + 1) / groups;
+    } else {
+      g.pass_fixed = 0;
+      g.u0 = g.u1 = 0;
+    }
+  }
   // Few weight tiles (QKV, O, down at decode sizes): give every tile the same whole number of
   // CTAs, so that no CTA's range crosses a tile and each has one partial tile to reduce at the
   // end instead of two.  The longest range grows by (per * grid - total) / grid k-blocks of about
@@ -333,6 +358,11 @@ __device__ __forceinline__ TcGeom tc_geom(const DevCtx& c, int T, int N, int K) 
     }
   }
   return g;
+}
+// position of unit u: weight tile and token pass (the k-block is u % kblocks)
+__device__ __forceinline__ int tc_unit_nt(const TcGeom& g, long long u) { return (int)(u / ((long long)g.kblocks * g.pdiv)); }
+__device__ __forceinline__ int tc_unit_pass(const TcGeom& g, long long u) {
+  return g.pass_fixed >= 0 ? g.pass_fixed : (int)((u / g.kblocks) % g.passes);
 }
 // tiles need 1024-byte alignment for the 128-byte swizzle
 __device__ __forceinline__ char* tc_tiles(float* smem_f) {
@@ -354,7 +384,7 @@ __device__ __forceinline__ void tc_produce_weights(const DevCtx& c, const void* 
     const long long seg_end = min(g.u1, (u / g.kblocks + 1) * (long long)g.kblocks);
     const int nk = (int)min((long long)g.KPS, seg_end - u);
     const int kb = (int)(u % g.kblocks);
-    const int nt = (int)(u / ((long long)g.kblocks * g.passes));   // unit order: n-tile, token pass, k-block
+    const int nt = tc_unit_nt(g, u);
     // the n-th fill of a stage waits for its (n-1)-th release
     if (!mbar_wait(c, &g_tc.empty[stage], ((tc.fill_bits >> stage) & 1u) ^ 1u, dead)) break;
     tc.fill_bits ^= 1u << stage;
@@ -400,7 +430,7 @@ static __device__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int whi
         const long long seg_end = min(u1, (u / kblocks + 1) * (long long)kblocks);
         const int nk = (int)min((long long)KPS, seg_end - u);
         const int kb = (int)(u % kblocks);
-        const int pass = (int)((u / kblocks) % g.passes);
+        const int pass = tc_unit_pass(g, u);
         if (!mbar_wait(c, &g_tc.empty[stage], ((tc.fill_bits >> stage) & 1u) ^ 1u, dead)) break;
         tc.fill_bits ^= 1u << stage;
         char* sa = tiles + (size_t)stage * stage_bytes;
@@ -418,7 +448,7 @@ static __device__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int whi
       long long u = u0;
       while (u < u1) {
         const long long seg_end = min(u1, (u / kblocks + 1) * (long long)kblocks);
-        const int pass = (int)((u / kblocks) % g.passes);
+        const int pass = tc_unit_pass(g, u);
         const int rows = min(256, T - pass * 256);
         const int n_mma = (rows + 15) & ~15;
         const uint32_t idesc = idesc_bf16(n_mma);
@@ -463,8 +493,8 @@ static __device__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int whi
       const long long seg_end = min(u1, (u / kblocks + 1) * (long long)kblocks);
       const int kb0 = (int)(u % kblocks);
       const int kb1 = kb0 + (int)(seg_end - u);
-      const int nt = (int)(u / ((long long)kblocks * g.passes));
-      const int pass = (int)((u / kblocks) % g.passes);
+      const int nt = tc_unit_nt(g, u);
+      const int pass = tc_unit_pass(g, u);
       const int rows = min(256, T - pass * 256);
       const int n_mma = (rows + 15) & ~15;
       const bool plain = (kb0 == 0 && kb1 == kblocks) && !accumulate && eo.row_map == nullptr;
@@ -500,8 +530,8 @@ static __device__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int whi
     }
     if (last_abuf >= 0) {
       const int kb0 = (int)(last_u % kblocks);
-      const int nt = (int)(last_u / ((long long)kblocks * g.passes));
-      const int pass = (int)((last_u / kblocks) % g.passes);
+      const int nt = tc_unit_nt(g, last_u);
+      const int pass = tc_unit_pass(g, last_u);
       const int n_mma = (min(256, T - pass * 256) + 15) & ~15;
       const int c_begin = tc_epi_half(n_mma);
       if (c_begin < n_mma && mbar_wait_idle(c, &g_tc.acc_full[last_abuf], last_par, dead)) {
