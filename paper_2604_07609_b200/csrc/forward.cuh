@@ -484,20 +484,41 @@ static __device__ void phase_attention(const DevCtx& c, int layer, float* smem) 
 constexpr int ATTN_SMEM_FLOATS(int HD, int NREP) { return NREP * HD + 2 * 8 * NREP + 8 * NREP * HD; }
 
 // ---- SwiGLU gate: act = silu(gate) * up ------------------------------------------------
+// The gate/up buffer comes from HBM (the weight stream of the GEMM before has pushed it out of L2)
+// and one CTA per SM leaves eight warps to cover that latency, so every thread has the loads of
+// SILU_U items in flight before it stores.  A function of its own: inlined into the loop kernel
+// the buffers of loaded values end up in local memory.
+template <typename WT>
+__device__ __noinline__ void silu_mul_rows(const float* __restrict__ gu, WT* __restrict__ out, int T, int F) {
+  constexpr int SILU_U = 4;
+  const int F4 = F / 4;
+  const int total = T * F4;   // < 2^31: at most a few thousand rows
+  const int stride = gridDim.x * FWD_THREADS;
+  for (int base = blockIdx.x * FWD_THREADS + threadIdx.x; base < total; base += SILU_U * stride) {
+    float4 g[SILU_U], u[SILU_U];
+#pragma unroll
+    for (int k = 0; k < SILU_U; ++k) {
+      const int idx = min(base + k * stride, total - 1);   // clamped: the tail loads a valid item twice
+      const int t = idx / F4, j = (idx - t * F4) * 4;
+      g[k] = __ldcg(reinterpret_cast<const float4*>(gu + (size_t)t * 2 * F + j));
+      u[k] = __ldcg(reinterpret_cast<const float4*>(gu + (size_t)t * 2 * F + F + j));
+    }
+#pragma unroll
+    for (int k = 0; k < SILU_U; ++k) {
+      const int idx = base + k * stride;
+      if (idx < total) {
+        const int t = idx / F4, j = (idx - t * F4) * 4;
+        store4<WT>(out + (size_t)t * F + j, g[k].x / (1.0f + __expf(-g[k].x)) * u[k].x,
+                   g[k].y / (1.0f + __expf(-g[k].y)) * u[k].y, g[k].z / (1.0f + __expf(-g[k].z)) * u[k].z,
+                   g[k].w / (1.0f + __expf(-g[k].w)) * u[k].w);
+      }
+    }
+  }
+}
 template <typename WT>
 static __device__ void phase_silu_mul(const DevCtx& c) {
   const int T = c.E > 0 ? c.ss->cur_T * c.topE : c.ss->cur_T;   // rows of the gate/up buffer
-  WT* out = reinterpret_cast<WT*>(c.act);
-  const int F4 = c.F / 4;
-  const int total = T * F4;   // < 2^31: at most a few thousand rows
-#pragma unroll 4
-  for (int idx = blockIdx.x * FWD_THREADS + threadIdx.x; idx < total; idx += gridDim.x * FWD_THREADS) {
-    const int t = idx / F4, j = (idx - t * F4) * 4;
-    const float4 g = *reinterpret_cast<const float4*>(c.gu + (size_t)t * 2 * c.F + j);
-    const float4 u = *reinterpret_cast<const float4*>(c.gu + (size_t)t * 2 * c.F + c.F + j);
-    store4<WT>(out + (size_t)t * c.F + j, g.x / (1.0f + __expf(-g.x)) * u.x, g.y / (1.0f + __expf(-g.y)) * u.y,
-               g.z / (1.0f + __expf(-g.z)) * u.z, g.w / (1.0f + __expf(-g.w)) * u.w);
-  }
+  if (T > 0) silu_mul_rows<WT>(c.gu, reinterpret_cast<WT*>(c.act), T, c.F);
 }
 
 // ---- routed experts: group the (token, expert) pairs by expert and gather their rows ---------
