@@ -186,9 +186,10 @@ static __device__ void phase_norm(const DevCtx& c, int layer, int which /*0: nor
   const int T = c.ss->cur_T;
   const float* g = wptr_f(c, which == 0 ? 6 : 7) + (size_t)layer * c.d;
   WT* out = reinterpret_cast<WT*>(c.xn);
-  // the split-K tensor-core GEMM that follows adds partial sums into its output
-  const int rows_gu = c.E > 0 ? T * c.topE : T;   // routed experts: one gate/up row per (token, expert)
-  if (c.gemm_tc) zero_floats(which == 0 ? c.qkv : c.gu, which == 0 ? (long long)T * c.qkv_dim : (long long)rows_gu * 2 * c.F);
+  // The split-K tensor-core GEMMs add partial sums into their outputs.  Those are cleared during
+  // the O GEMM by a warp that has no role there (the gate/up buffer of this layer and the QKV
+  // buffer of the next); only the first layer's QKV buffer is cleared here.
+  if (c.gemm_tc && which == 0 && layer == 0) zero_floats(c.qkv, (long long)T * c.qkv_dim);
   const float* wr = (which == 1 && c.E > 0) ? wptr_f(c, 5) + (size_t)layer * c.E * c.d : nullptr;
   for (int t = blockIdx.x; t < T; t += gridDim.x) {
     const WT* e = (which == 0 && layer == 0) ? wptr<WT>(c, 0) + (size_t)c.tok_id[t] * c.d : nullptr;
@@ -223,6 +224,10 @@ struct GemmArgs {
   long long w_row0 = 0;
   const int32_t* row_map = nullptr;
   const float* row_scale = nullptr;
+  // tensor-core path: buffers that an otherwise idle warp clears during this GEMM (outputs of later
+  // split-K GEMMs, which add partial sums into them); counts in floats, multiples of 4
+  float* zero_p[2] = {nullptr, nullptr};
+  long long zero_n[2] = {0, 0};
 };
 
 template <typename WT>

@@ -485,6 +485,15 @@ static __device__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int whi
     }
   } else if (warp >= 4) {
     const int q = warp & 3;  // TMEM lane quarter this warp may read
+    // nothing to store until the first accumulator is complete: clear the buffers the caller named
+    // (16-byte stores, grid-strided over the epilogue threads)
+    for (int z = 0; z < 2; ++z) {
+      float4* zq = reinterpret_cast<float4*>(a.zero_p[z]);
+      const long long n4 = a.zero_n[z] >> 2;
+      const long long step = (long long)gridDim.x * 128;
+      for (long long i = (long long)blockIdx.x * 128 + (threadIdx.x - 128); i < n4; i += step)
+        zq[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
     const TcEpiOut eo{a.out, (size_t)a.ldo, a.row_map, a.row_scale, T, N};
     const bool accumulate = a.accumulate != 0;
     int abuf = 0;

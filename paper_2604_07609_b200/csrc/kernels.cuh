@@ -45,6 +45,15 @@ __device__ __forceinline__ void run_phase(const DevCtx& c, int phase, int layer,
     case PH_O: {
       GemmArgs a{c.attn, c.w_base + c.w_off[2] + (size_t)layer * c.d * c.q_dim * esz, c.h, T, c.d, c.q_dim, c.d, 1};
       a.w_row0 = (long long)layer * c.d;
+      if (c.gemm_tc) {
+        const int rows_gu = c.E > 0 ? T * c.topE : T;   // routed experts: one gate/up row per (token, expert)
+        a.zero_p[0] = c.gu;
+        a.zero_n[0] = (long long)rows_gu * 2 * c.F;
+        if (layer + 1 < c.L) {
+          a.zero_p[1] = c.qkv;
+          a.zero_n[1] = (long long)T * c.qkv_dim;
+        }
+      }
       gemm_dispatch<WT>(c, a, GEMM_O, layer, smem, tc);
     } break;
     case PH_NORM2:
