@@ -533,9 +533,13 @@ static __device__ int schedule_step(const DevCtx& c, unsigned long long visible)
     ss->pending_post = 1;
     if (c.dec_row != nullptr) {
       const long long TT = (long long)tot_kb * c.Hkv;
-      // sub-ranges: k per warp of the grid, about 32 to 64 tiles each once there is that much work
+      // Sub-ranges: k per warp of the grid.  Every cut of a unit costs a partial record and a merge,
+      // so a pure decode step takes one sub-range per warp up to 96 tiles; with prefill tiles in the
+      // step the CTAs reach their decode share at different times and smaller sub-ranges (up to 48
+      // tiles, the later ones handed out by the counter) even that out.
       const long long NW = c.n_warps_grid;
-      const long long k = (TT + 48 * NW - 1) / (48 * NW) > 1 ? (TT + 48 * NW - 1) / (48 * NW) : 1;
+      const long long cap = n_pf > 0 ? 48 : 96;
+      const long long k = (TT + cap * NW - 1) / (cap * NW) > 1 ? (TT + cap * NW - 1) / (cap * NW) : 1;
       long long S = (TT + k * NW - 1) / (k * NW);
       if (S < 1) S = 1;
       while ((TT + S - 1) / S > c.att_sub_max) S *= 2;   // cannot happen with the sizes set at create

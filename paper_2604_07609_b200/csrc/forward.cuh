@@ -224,8 +224,8 @@ struct GemmArgs {
   long long w_row0 = 0;
   const int32_t* row_map = nullptr;
   const float* row_scale = nullptr;
-  // tensor-core path: buffers that an otherwise idle warp clears during this GEMM (outputs of later
-  // split-K GEMMs, which add partial sums into them); counts in floats, multiples of 4
+  // tensor-core path: buffers that the epilogue warps clear at the start of this GEMM (outputs of
+  // later split-K GEMMs, which add partial sums into them); counts in floats, multiples of 4
   float* zero_p[2] = {nullptr, nullptr};
   long long zero_n[2] = {0, 0};
 };
