@@ -301,9 +301,17 @@ int blink_sample(const float* logits, int rows, int vocab, const int32_t* top_k,
  * value is refused with BLINK_ETOOBIG before anything is touched; split the rows over
  * several calls instead.
  *
- * The first call on each device looks up the device address of the scratch array (one
- * runtime query, with that device current); make that first call before any stream capture
- * begins.  All calls on a device share the one scratch array and it keeps the previous call's
+ * The first call on each device does the set-up: it looks up the device address of the scratch
+ * array (one runtime query, with that device current) and creates the stream the call works on
+ * (a driver object, no device memory from the allocator); make that first call before any
+ * stream capture begins.  Every later call only enqueues copies and one kernel on that stream
+ * and waits for the stream: it neither uses the legacy default stream nor synchronises the
+ * device, so other streams keep running.  Consequences for the caller: `logits` must be
+ * complete before the call (synchronise the stream that produced it); and the kernel needs
+ * SMs like any other launch, so while a persistent serving loop of this library occupies every
+ * SM of the GPU the call waits until that loop leaves (stop it, or let it reach its idle exit).
+ *
+ * All calls on a device share the one scratch array and it keeps the previous call's
  * contents: every call overwrites the part it uses before the kernel reads it, nothing has
  * to start at zero.  Calls that overlap on the same GPU (from several threads or processes
  * sharing a context) would race on the array: the library serialises its own callers with a

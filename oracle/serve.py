@@ -15,14 +15,18 @@ from . import transformer as O2
 
 
 def run(model_cfg, sched, weights: O2.Weights, requests, watermarks=None, act_round=None,
-        keep_logits=True, max_iters=10_000_000):
-    """requests: objects with ticket, prompt, max_new, top_k, temperature, seed, eos_id.
-    Returns dict(trace, tokens {ticket: [..]}, logits [(iter, bslot, ticket, gen_index, row)])."""
+        keep_logits=True, max_iters=10_000_000, forced=None):
+    """requests: objects with ticket, prompt, max_new, top_k, temperature, seed, eos_id (and top_p, optional).
+    forced: optional {ticket: [tokens]}: teacher forcing, the given tokens are fed back instead of
+    the sampled ones (the sampled ones are still what `sampled` reports).
+    Returns dict(trace, tokens {ticket: [fed-back tokens]}, sampled {ticket: [sampled tokens]},
+    logits [(iter, bslot, ticket, gen_index, row)])."""
     sim = [O1.SimRequest(r.ticket, len(r.prompt), r.max_new, r.eos_id, r.prompt) for r in requests]
     byt = {r.ticket: r for r in requests}
     model = O2.PagedModel(model_cfg, weights, sched.n_blocks, sched.block_size, act_round)
     logs = []
     it_no = [0]
+    sampled = {r.ticket: [] for r in requests}
 
     def sample_fn(items):
         lg = model.step(items)
@@ -32,7 +36,9 @@ def run(model_cfg, sched, weights: O2.Weights, requests, watermarks=None, act_ro
                 continue
             r = byt[it.ticket]
             l32 = np.asarray(lg[row], dtype=np.float32)
-            toks.append(S.sample(l32, r.top_k, r.temperature, r.ticket, it.gen_index, r.seed))
+            tok = S.sample(l32, r.top_k, r.temperature, r.ticket, it.gen_index, r.seed, getattr(r, "top_p", 0.0))
+            sampled[it.ticket].append(tok)
+            toks.append(tok if forced is None else int(forced[it.ticket][it.gen_index]))
             if keep_logits:
                 logs.append((it_no[0], it.bslot, it.ticket, it.gen_index, np.array(lg[row])))
             row += 1
@@ -42,4 +48,4 @@ def run(model_cfg, sched, weights: O2.Weights, requests, watermarks=None, act_ro
     trace, tokens, sch = O1.simulate(sim, sched.max_batch, sched.prefill_chunk_tokens,
                                      sched.n_blocks, sched.block_size, watermarks, sample_fn,
                                      max_iters=max_iters)
-    return dict(trace=trace, tokens=tokens, logits=logs, scheduler=sch)
+    return dict(trace=trace, tokens=tokens, sampled=sampled, logits=logs, scheduler=sch)

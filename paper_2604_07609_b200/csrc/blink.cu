@@ -397,6 +397,7 @@ static __device__ __align__(256) unsigned char g_sample_scratch[BLINK_SAMPLE_NOA
 namespace {
 std::mutex g_noalloc_mu;
 void* g_noalloc_ptr[NOALLOC_MAX_DEVICES] = {nullptr};
+cudaStream_t g_noalloc_stream[NOALLOC_MAX_DEVICES] = {nullptr};
 }  // namespace
 
 int blink_sample_noalloc(const float* logits, int rows, int vocab, const int32_t* top_k, const float* temperature,
@@ -414,14 +415,20 @@ int blink_sample_noalloc(const float* logits, int rows, int vocab, const int32_t
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= NOALLOC_MAX_DEVICES) return BLINK_ECUDA;
   std::lock_guard<std::mutex> g(g_noalloc_mu);  // one user of the shared scratch at a time
   if (!g_noalloc_ptr[dev]) {
+    // first call on this device: the address of the scratch array, and a stream of the call's own so
+    // that it neither joins the legacy default stream nor synchronises the whole device
     void* p = nullptr;
     const cudaError_t e = cudaGetSymbolAddress(&p, g_sample_scratch);
     if (e != cudaSuccess || !p) {
       fprintf(stderr, "blink_sample_noalloc: cudaGetSymbolAddress failed: %s\n", cudaGetErrorString(e));
       return BLINK_ECUDA;
     }
+    cudaStream_t st = nullptr;
+    if (cudaStreamCreateWithFlags(&st, cudaStreamNonBlocking) != cudaSuccess) return BLINK_ECUDA;
+    g_noalloc_stream[dev] = st;
     g_noalloc_ptr[dev] = p;
   }
+  cudaStream_t st = g_noalloc_stream[dev];
   // carve the scratch with the capacity as stride, so every sub-array stays naturally aligned
   char* d = static_cast<char*>(g_noalloc_ptr[dev]);
   const size_t cap = BLINK_SAMPLE_NOALLOC_MAX_ROWS, n = (size_t)rows;
@@ -431,18 +438,19 @@ int blink_sample_noalloc(const float* logits, int rows, int vocab, const int32_t
   float* d_temp = reinterpret_cast<float*>(d_topk + cap);
   int* d_gen = reinterpret_cast<int*>(d_temp + cap);
   int* d_out = d_gen + cap;
-  if (cudaMemcpy(d_ticket, ticket, n * 8, cudaMemcpyHostToDevice) != cudaSuccess ||
-      cudaMemcpy(d_seed, seed, n * 8, cudaMemcpyHostToDevice) != cudaSuccess ||
-      cudaMemcpy(d_topk, top_k, n * 4, cudaMemcpyHostToDevice) != cudaSuccess ||
-      cudaMemcpy(d_temp, temperature, n * 4, cudaMemcpyHostToDevice) != cudaSuccess ||
-      cudaMemcpy(d_gen, gen_index, n * 4, cudaMemcpyHostToDevice) != cudaSuccess ||
-      cudaMemset(d_out, 0xff, n * 4) != cudaSuccess)  // results of an earlier call must not show through
+  if (cudaMemcpyAsync(d_ticket, ticket, n * 8, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaMemcpyAsync(d_seed, seed, n * 8, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaMemcpyAsync(d_topk, top_k, n * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaMemcpyAsync(d_temp, temperature, n * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaMemcpyAsync(d_gen, gen_index, n * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaMemsetAsync(d_out, 0xff, n * 4, st) != cudaSuccess)  // results of an earlier call must not show through
     return BLINK_ECUDA;
   const int grid = rows < 1184 ? rows : 1184;
-  blink_sample_kernel<<<grid, FWD_THREADS, SAMPLE_SMEM_FLOATS * sizeof(float)>>>(logits, rows, vocab, d_topk, d_temp,
-                                                                                 d_ticket, d_gen, d_seed, d_out);
-  if (cudaGetLastError() != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) return BLINK_ECUDA;
-  if (cudaMemcpy(out, d_out, n * 4, cudaMemcpyDeviceToHost) != cudaSuccess) return BLINK_ECUDA;
+  blink_sample_kernel<<<grid, FWD_THREADS, SAMPLE_SMEM_FLOATS * sizeof(float), st>>>(logits, rows, vocab, d_topk, d_temp,
+                                                                                     d_ticket, d_gen, d_seed, d_out);
+  if (cudaGetLastError() != cudaSuccess) return BLINK_ECUDA;
+  if (cudaMemcpyAsync(out, d_out, n * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) return BLINK_ECUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return BLINK_ECUDA;
   return BLINK_OK;
 }
 

@@ -55,8 +55,16 @@ __device__ __forceinline__ unsigned long long ld_acquire_gpu_u64(const unsigned 
 // host before each launch) and waits until it reaches the next multiple of the grid size.
 // Returns false when the loop must unwind (time-out here or abort raised elsewhere).  `target`
 // is the caller's private running total (thread 0 of each CTA keeps it).
+__device__ __forceinline__ void fence_proxy_async_global() {
+  asm volatile("fence.proxy.async.global;" ::: "memory");
+}
+
 __device__ __forceinline__ bool grid_barrier(const DevCtx& c, unsigned long long& target) {
   __shared__ int s_ok;
+  // Buffers written with ordinary stores in one phase (normed rows, K/V rows, attention output, ...)
+  // are read by TMA / bulk copies (the async proxy) in a later phase: every thread orders its
+  // stores against that proxy before it arrives, and again before it issues copies afterwards.
+  fence_proxy_async_global();
   __syncthreads();
   if (threadIdx.x == 0) {
     int ok = 1;
@@ -82,6 +90,7 @@ __device__ __forceinline__ bool grid_barrier(const DevCtx& c, unsigned long long
     s_ok = ok;
   }
   __syncthreads();
+  fence_proxy_async_global();
   return s_ok != 0;
 }
 
@@ -576,6 +585,7 @@ static __device__ void control_phase(const DevCtx& c, long long& launch_iters) {
   const int tid = threadIdx.x;
   __shared__ int s_cmd;
   __shared__ int s_started;
+  __shared__ int s_abort;
   __shared__ unsigned long long s_tail;
   if (ss->pending_post) post_step(c);
   long long idle_t0 = clock64();
@@ -610,7 +620,11 @@ static __device__ void control_phase(const DevCtx& c, long long& launch_iters) {
       __syncthreads();
       break;
     }
-    if (*(volatile int*)&ss->abort_flag) {
+    // one thread reads the flag (another CTA may raise it at any time) so that the whole CTA
+    // takes the same branch
+    if (tid == 0) s_abort = *(volatile int*)&ss->abort_flag;
+    __syncthreads();
+    if (s_abort) {
       if (tid == 0) { s_cmd = CMD_EXIT; ss->exit_reason = 5; }
       __syncthreads();
       break;

@@ -29,6 +29,7 @@ class Request:
     seed: int = 0
     eos_id: int = -1
     user_tag: int = 0
+    top_p: float = 0.0            # outside (0, 1) = no nucleus cut
     extra: dict = field(default_factory=dict)
 
     @property

@@ -91,3 +91,92 @@ def gpu_run_forced(model, sched, reqs, weights_cpu, forced, *, exec_mode=B.EXEC_
         return trace, B.tokens_by_ticket(ev), cap.cpu().numpy(), eng.blink_get_iter_stats()
     finally:
         assert eng.blink_destroy() == B.BLINK_OK
+
+
+# ---- token rules near ties (a decision that rounding inside the tolerance may flip) -----------------
+def acceptable_tokens(row, req, gen_index, tol):
+    """Tokens a correct implementation may emit for oracle logits `row` when its own logits are
+    within `tol` (max-abs) of them.  Greedy: every token within 2*tol of the maximum.  Top-k /
+    top-p: the oracle's token, plus the neighbouring candidates when the draw lies within the
+    distance by which a tol-perturbation can move an inverse-CDF boundary, plus the entries at a
+    candidate-set boundary that is itself inside the margin.  Returns (set, in_margin)."""
+    from oracle import sampler as S
+    row = np.asarray(row, dtype=np.float32)
+    top_p = getattr(req, "top_p", 0.0)
+    nucleus_on = 0.0 < top_p < 1.0
+    if req.top_k <= 0 and not nucleus_on:
+        mx = float(row.max())
+        ok = set(int(i) for i in np.flatnonzero(row >= mx - 2 * tol))
+        return ok, len(ok) > 1
+    want = S.sample(row, req.top_k, req.temperature, req.ticket, gen_index, req.seed, top_p)
+    T = float(req.temperature)
+    n = len(row)
+    k = n if req.top_k <= 0 else min(req.top_k, n)
+    idx, z = S.top_k_candidates(row, min(n, k + 1), T)
+    ok, in_margin = {want}, False
+    if k < n and float(z[k - 1]) - float(z[k]) < 2 * tol / T:       # the k-th and (k+1)-th candidates may swap
+        in_margin = True
+        ok.update(int(i) for i in idx[max(0, k - 2):k + 1])
+    idx, z = idx[:k], z[:k].astype(np.float64)
+    w = np.exp(z - z[0])
+    if nucleus_on:
+        nidx, _ = S.nucleus(row, req.top_k, T, top_p)
+        m = len(nidx)
+        cfrac = np.cumsum(w) / w.sum()
+        d = 4 * tol / T + 1e-7
+        if m < k and abs(cfrac[m - 1] - top_p) < d or (m >= 2 and abs(cfrac[m - 2] - top_p) < d):
+            in_margin = True                                           # the nucleus may gain or lose its last token
+            ok.update(int(i) for i in idx[:min(k, m + 1)])
+            return ok, in_margin
+        w, idx = w[:m], idx[:m]
+    cfrac = np.cumsum(w) / w.sum()
+    u = (S.philox_word(req.ticket, gen_index, req.seed) >> 8) / 2.0 ** 24
+    j = int(np.flatnonzero(idx == want)[0])
+    d = 4 * tol / T + 1e-7
+    if j > 0 and u - cfrac[j - 1] < d:
+        in_margin = True
+        ok.add(int(idx[j - 1]))
+    if j + 1 < len(idx) and cfrac[j] - u < d:
+        in_margin = True
+        ok.add(int(idx[j + 1]))
+    return ok, in_margin
+
+
+def assert_tokens_within_margin(ora, reqs, toks_gpu, tol):
+    """Under teacher forcing the sampled token of every (ticket, index) must be the oracle's, except
+    where the oracle's own decision margin is inside the tolerance; there it must be one of the
+    in-margin candidates.  Returns the number of in-margin decisions."""
+    by_ticket = {r.ticket: r for r in reqs}
+    n_margin = 0
+    for (_, _, ticket, gi, row) in ora["logits"]:
+        ok, im = acceptable_tokens(row, by_ticket[ticket], gi, tol)
+        n_margin += int(im)
+        got = toks_gpu[ticket][gi]
+        assert got in ok, f"ticket {ticket} index {gi}: token {got} not among the admissible {sorted(ok)[:8]}"
+        if not im:
+            assert got == ora["sampled"][ticket][gi]
+    return n_margin
+
+
+def compare_with_oracle(model, sched, reqs, weights_cpu, tol, *, oracle_dtype=np.float64, plain_too=True, **kw):
+    """The whole check of one configuration: the oracle in the data path's rounding mode runs free
+    (its own tokens fed back); the GPU is teacher-forced with those tokens; traces must be equal word
+    for word (sampled tokens apart), logits within `tol`, tokens by the margin rule.  For the bf16 data
+    path the plain high-precision oracle (no rounding hook) is run on the same forced tokens as well
+    and the error against it reported."""
+    matched_round = O2.round_bf16 if model.dtype == "bf16" else None
+    W = O2.Weights(model, weights_as_numpy(model, weights_cpu), dtype=oracle_dtype)
+    ora = OS.run(model, sched, W, reqs, act_round=matched_round)
+    trace, toks, logits, its = gpu_run_forced(model, sched, reqs, weights_cpu, ora["tokens"], **kw)
+    assert_traces_equal([{**r, "sampled": []} for r in trace], [{**r, "sampled": []} for r in ora["trace"]])
+    lo = np.stack([row for (_, _, _, _, row) in ora["logits"]])
+    assert logits.shape == lo.shape
+    err = float(np.abs(logits.astype(np.float64) - lo).max())
+    assert err <= tol, f"max-abs logit error {err:.3e} against the oracle exceeds {tol}"
+    n_margin = assert_tokens_within_margin(ora, reqs, toks, tol)
+    err_plain = err
+    if plain_too and matched_round is not None:
+        plain = OS.run(model, sched, W, reqs, act_round=None, forced=ora["tokens"])
+        lp = np.stack([row for (_, _, _, _, row) in plain["logits"]])
+        err_plain = float(np.abs(logits.astype(np.float64) - lp).max())
+    return dict(err=err, err_plain=err_plain, n_margin=n_margin, trace=trace, toks=toks, ora=ora, its=its, logits=logits)

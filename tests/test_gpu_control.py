@@ -125,3 +125,42 @@ def test_timestamps_and_event_order():
             assert -1_000_000 < ttft_ns < 2_000_000_000
     finally:
         assert eng.blink_destroy() == B.BLINK_OK
+
+
+def test_eos_retires_a_request_early_and_frees_its_blocks():
+    """A request whose eos_id is a token it emits before max_new: it is retired in that iteration
+    (blocks pushed back, reservation released, finished flag in the published count) and the trace
+    equals the oracle's, which is given the same eos ids."""
+    model = model_cfg(1)
+    sched = sched_cfg(1, max_batch=4, n_blocks=64)
+    reqs = make_requests(1)
+    # control-only tokens are a fixed function of (ticket, index): pick, for every other request, the
+    # token it will emit at index 5 (unless it shows up earlier, then that earlier index ends it)
+    for r in reqs[::2]:
+        r.eos_id = O1.fake_token(r.ticket, 5, model.vocab)
+    eng = B.Blink(model, sched, control_only=True, start_paused=True, trace_words=1 << 20, idle_exit_us=300_000)
+    try:
+        for r in reqs:
+            eng.submit_request(r)
+        eng.blink_start()
+        tr_o, toks_o, _ = O1.simulate([O1.SimRequest(r.ticket, r.n_prompt, r.max_new, r.eos_id, r.prompt) for r in reqs],
+                                      sched.max_batch, sched.prefill_chunk_tokens, sched.n_blocks, sched.block_size,
+                                      vocab=model.vocab)
+        total = sum(len(v) for v in toks_o.values())
+        assert total < sum(r.max_new for r in reqs)                  # some requests really ended early
+        ev = eng.drain(total, timeout_s=60)
+        eng.blink_stop(final=False)
+        st = eng.blink_get_stats()
+        trace = B.parse_trace(eng.blink_get_trace())
+    finally:
+        assert eng.blink_destroy() == B.BLINK_OK
+    assert st.device_status == 0
+    assert_traces_equal(trace, tr_o)
+    assert B.tokens_by_ticket(ev) == toks_o
+    assert st.free_blocks == sched.n_blocks and st.reserved_blocks == 0 and st.batch_live == 0
+    for r in reqs:
+        e = np.sort(ev[ev["ticket"] == r.ticket], order="index")
+        assert len(e) == len(toks_o[r.ticket])
+        assert e["is_last"][-1] == 1 and e["is_last"][:-1].sum() == 0
+        if r.eos_id >= 0:
+            assert len(e) <= 6 and int(e["token"][-1]) == r.eos_id

@@ -8,7 +8,7 @@ from oracle import transformer as O2
 from paper_2604_07609_b200 import binding as B
 from synth import make_requests, make_weights, model_cfg, sched_cfg
 
-from gpu_util import assert_traces_equal, gpu_run_forced, oracle_run
+from gpu_util import assert_tokens_within_margin, assert_traces_equal, compare_with_oracle, gpu_run_forced, oracle_run
 
 pytestmark = pytest.mark.gpu
 
@@ -17,27 +17,15 @@ TOL_BF16 = 2e-2     # max-abs logit error, bf16 mode
 
 
 def _compare(model, sched, reqs, weights, act_round, tol, **kw):
-    ora = oracle_run(model, sched, reqs, weights, act_round)
-    trace, toks, logits, _ = gpu_run_forced(model, sched, reqs, weights, ora["tokens"], **kw)
-    assert_traces_equal([{**r, "sampled": []} for r in trace], [{**r, "sampled": []} for r in ora["trace"]])
-    lo = np.stack([row for (_, _, _, _, row) in ora["logits"]])
-    assert logits.shape == lo.shape
-    err = np.abs(logits.astype(np.float64) - lo).max()
-    # tokens: identical wherever the oracle's decision margin exceeds twice the tolerance
-    n_in_margin = 0
-    k = 0
-    for (it, bslot, ticket, gi, row) in ora["logits"]:
-        r = reqs[ticket]
-        if r.top_k == 0:
-            srt = np.sort(row)
-            margin = srt[-1] - srt[-2]
-            if margin > 2 * tol:
-                assert toks[ticket][gi] == ora["tokens"][ticket][gi], (ticket, gi, margin)
-            else:
-                n_in_margin += 1
-                assert row[toks[ticket][gi]] >= srt[-1] - 2 * tol
-        k += 1
-    return err, n_in_margin, trace, toks, ora
+    """Oracle (in the data path's rounding mode) vs GPU under teacher forcing: traces, logits within
+    `tol`, tokens by the margin rule; for bf16 also the error against the plain high-precision oracle,
+    which must meet the same tolerance."""
+    r = compare_with_oracle(model, sched, reqs, weights, tol, **kw)
+    if model.dtype == "bf16":
+        print(f"  max-abs logit error: {r['err']:.3e} against the oracle rounding where the data path stores 16-bit "
+              f"values, {r['err_plain']:.3e} against the plain high-precision oracle")
+        assert r["err_plain"] <= tol, r["err_plain"]
+    return r["err"], r["n_margin"], r["trace"], r["toks"], r["ora"]
 
 
 def test_config1_fp32_reference_mode_logits_tokens_trace():
@@ -91,15 +79,13 @@ def test_topk_sampling_end_to_end_fp32():
     for r in reqs:
         r.top_k, r.temperature = 50, 0.8
     w = make_weights(model, 5, "cpu")
-    ora = oracle_run(model, sched, reqs, w, None)
-    trace, toks, logits, _ = gpu_run_forced(model, sched, reqs, w, ora["tokens"])
-    lo = np.stack([row for (_, _, _, _, row) in ora["logits"]])
-    assert np.abs(logits - lo).max() <= TOL_FP32
-    # the draw is identical on both sides; tokens agree unless a candidate boundary sits inside the tolerance
-    agree = sum(toks[t][i] == ora["tokens"][t][i] for t in toks for i in range(len(toks[t])))
+    # the draw is identical on both sides: tokens are the oracle's except where a candidate-set or
+    # inverse-CDF boundary lies inside the logit tolerance (checked by the margin rule in _compare)
+    err, n_margin, trace, toks, ora = _compare(model, sched, reqs, w, None, TOL_FP32)
+    agree = sum(toks[t][i] == ora["sampled"][t][i] for t in toks for i in range(len(toks[t])))
     total = sum(len(v) for v in toks.values())
-    print(f"top-k end to end: {agree}/{total} tokens identical")
-    assert agree >= total - 2
+    print(f"top-k end to end: {agree}/{total} tokens identical, {n_margin} decisions inside the margin")
+    assert total - agree <= n_margin
 
 
 def test_sampler_alone_bit_exact_on_oracle_logits():
@@ -190,14 +176,9 @@ def test_streaming_weight_layout_round_trip_and_parity():
     for r in (0, 1, 7, 8, 77, 127):
         for c8 in range(8):
             assert torch.equal(tile[r, c8 ^ (r & 7)], rm[r, c8])
-    ora = oracle_run(model, sched, reqs, w, O2.round_bf16)
-    trace, toks, logits, _ = gpu_run_forced(model, sched, reqs, w, ora["tokens"], gemm_impl=B.GEMM_TC,
-                                            weights_layout=B.WEIGHTS_STREAMING)
-    lo = np.stack([row for (_, _, _, _, row) in ora["logits"]])
-    err = np.abs(logits.astype(np.float64) - lo).max()
+    err, _, trace, toks, ora = _compare(model, sched, reqs, w, O2.round_bf16, TOL_BF16, gemm_impl=B.GEMM_TC,
+                                        weights_layout=B.WEIGHTS_STREAMING)
     print(f"streaming layout: max-abs logit error {err:.3e}")
-    assert err <= TOL_BF16
-    assert_traces_equal([{**r, "sampled": []} for r in trace], [{**r, "sampled": []} for r in ora["trace"]])
     # the SIMT path cannot read the streaming layout: refused, not misread
     with pytest.raises(B.BlinkError):
         gpu_run_forced(model, sched, reqs, w, ora["tokens"], gemm_impl=B.GEMM_SIMT, weights_layout=B.WEIGHTS_STREAMING)
@@ -215,13 +196,8 @@ def test_routed_experts_match_oracle(dtype, tol, kw):
     for r in reqs:
         r.max_new = 8
     w = make_weights(model, 31, "cpu", random_gains=True)
-    ora = oracle_run(model, sched, reqs, w, O2.round_bf16 if dtype == "bf16" else None)
-    trace, toks, logits, _ = gpu_run_forced(model, sched, reqs, w, ora["tokens"], **kw)
-    lo = np.stack([row for (_, _, _, _, row) in ora["logits"]])
-    err = np.abs(logits.astype(np.float64) - lo).max()
+    err, _, trace, toks, ora = _compare(model, sched, reqs, w, None, tol, **kw)
     print(f"routed experts {dtype}: max-abs logit error {err:.3e}")
-    assert err <= tol
-    assert_traces_equal([{**r, "sampled": []} for r in trace], [{**r, "sampled": []} for r in ora["trace"]])
 
 
 def test_decode_attention_many_rows_whole_and_split_units():
@@ -235,11 +211,6 @@ def test_decode_attention_many_rows_whole_and_split_units():
     reqs = [Request(t, 0.0, rng.integers(0, model.vocab, size=int(p)).astype(np.int32), 6)
             for t, p in enumerate(rng.integers(150, 400, size=64))]
     w = make_weights(model, 11, "cpu", random_gains=True)
-    ora = oracle_run(model, sched, reqs, w, O2.round_bf16)
-    trace, toks, logits, _ = gpu_run_forced(model, sched, reqs, w, ora["tokens"])
-    lo = np.stack([row for (_, _, _, _, row) in ora["logits"]])
-    err = np.abs(logits.astype(np.float64) - lo).max()
+    err, _, trace, toks, ora = _compare(model, sched, reqs, w, O2.round_bf16, TOL_BF16)
     print(f"64 rows, long contexts: max-abs logit error {err:.3e}; rows/step up to "
           f"{max(sum(s[4] for s in r['scheduled']) for r in trace)}")
-    assert err <= TOL_BF16
-    assert_traces_equal([{**r, "sampled": []} for r in trace], [{**r, "sampled": []} for r in ora["trace"]])

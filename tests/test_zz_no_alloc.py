@@ -26,7 +26,9 @@ def _inputs(rows, vocab, seed):
     ticket = (np.arange(rows, dtype=np.uint64) * 131 + seed).astype(np.uint64)
     gen = (np.arange(rows) * 3 % 211).astype(np.int32)
     sd = (np.arange(rows, dtype=np.uint64) * np.uint64(0x9E3779B97F4A7C15)) ^ np.uint64(seed)
-    return torch.from_numpy(logits).cuda(), top_k, temp, ticket, gen, sd
+    dev = torch.from_numpy(logits).cuda()
+    torch.cuda.synchronize()     # the entry point works on a stream of its own: the logits must be complete
+    return dev, top_k, temp, ticket, gen, sd
 
 
 def test_no_alloc_sampler_equals_allocating_sampler_on_two_calls_in_a_row():
@@ -38,6 +40,17 @@ def test_no_alloc_sampler_equals_allocating_sampler_on_two_calls_in_a_row():
         assert got.dtype == np.int32 and got.shape == want.shape
         assert np.array_equal(got, want)
         assert (got >= 0).all() and (got < args[0].shape[1]).all()
+
+
+def test_no_alloc_sampler_at_its_row_limit_uses_the_whole_scratch():
+    """Exactly the maximum number of rows (small vocabulary): the last entries of every carved
+    sub-array of the fixed scratch are written and read."""
+    args = _inputs(B.SAMPLE_NOALLOC_MAX_ROWS, 512, 13)
+    want = B.blink_sample(*args)
+    got = B.blink_sample_noalloc(*args)
+    assert np.array_equal(got, want)
+    again = B.blink_sample_noalloc(*_inputs(5, 512, 14))      # and a short call right after it
+    assert np.array_equal(again, B.blink_sample(*_inputs(5, 512, 14)))
 
 
 def test_no_alloc_sampler_refuses_more_rows_than_its_scratch_holds():
