@@ -146,27 +146,75 @@ def weights_to_host_fp32(m, wbuf):
     return out
 
 
-def cpu_oracle_sample(m, sched, wbuf, n_requests, prompt_cap, new_tokens, config):
-    """Time the oracle, as it stands, on a bounded sample of the workload."""
-    import torch
-    from oracle import serve as OS
-    from oracle import transformer as O2
+def sample_requests(config, n_requests, prompt_cap, new_tokens):
     from synth import make_requests
     reqs = make_requests(config, n_requests=n_requests)
     for r in reqs:
         r.prompt = r.prompt[:prompt_cap]
         r.max_new = new_tokens
+    return reqs
+
+
+def cpu_oracle_sample(m, sched, wbuf, n_requests, prompt_cap, new_tokens, config, keep_logits=False):
+    """Time the oracle, as it stands, on a bounded sample of the workload."""
+    import torch
+    from oracle import serve as OS
+    from oracle import transformer as O2
+    reqs = sample_requests(config, n_requests, prompt_cap, new_tokens)
     arrays = weights_to_host_fp32(m, wbuf)
     W = O2.Weights(m, arrays, dtype=np.float32)
     sch = sched.with_(n_blocks=max(64, n_requests * ((prompt_cap + new_tokens) // 16 + 2)))
     t0 = time.perf_counter()
-    res = OS.run(m, sch, W, reqs, act_round=O2.round_bf16 if m.dtype == "bf16" else None, keep_logits=False)
+    res = OS.run(m, sch, W, reqs, act_round=O2.round_bf16 if m.dtype == "bf16" else None, keep_logits=keep_logits)
     dt = time.perf_counter() - t0
+    if keep_logits:   # untimed: the same sample through the plain oracle (no rounding hook), same tokens fed back
+        res["plain"] = OS.run(m, sch, W, reqs, act_round=None, forced=res["tokens"]) if m.dtype == "bf16" else res
+        res["requests"], res["sched"] = reqs, sch
     n_out = sum(len(v) for v in res["tokens"].values())
     return dict(value=n_out / dt, unit="output tok/s", cores=torch.get_num_threads(), kind="oracle",
                 sample=f"first {n_requests} requests of the stream, prompts cut to {prompt_cap} tokens, "
                        f"{new_tokens} new tokens each, full {m.n_layers}-layer model in fp32 numpy; "
                        f"{n_out} tokens in {dt:.1f} s, {len(res['trace'])} iterations"), res, dt
+
+
+def parity_on_sample(B, m, wbuf, wl, res):
+    """The oracle's sample (the one the CPU leg just timed, full model) through the GPU loop, teacher-forced
+    with the oracle's tokens, logits captured: how far the two are apart, beside how far the two CPU
+    oracles (with and without the 16-bit rounding hook) are from each other on the same inputs."""
+    import torch
+    reqs, sch = res["requests"], res["sched"]
+    dev = wbuf.device
+    total = sum(r.max_new for r in reqs)
+    kv = torch.zeros(sch.n_blocks * B.kv_bytes_per_block(m, sch.block_size), dtype=torch.uint8, device=dev)
+    cap = torch.zeros((total, m.vocab), dtype=torch.float32, device=dev)
+    eng = B.Blink(m, sch, wbuf, kv, start_paused=True, logits_capture=cap, idle_exit_us=300_000, weights_layout=wl,
+                  trace_words=1 << 20)
+    try:
+        for r in reqs:
+            eng.submit_request(r, forced_tokens=res["tokens"][r.ticket])
+        eng.blink_start()
+        ev = eng.drain(total, timeout_s=120)
+        eng.blink_stop(final=False)
+        trace = B.parse_trace(eng.blink_get_trace())
+    finally:
+        eng.blink_destroy()
+    torch.cuda.synchronize()
+    lg = cap.cpu().numpy().astype(np.float64)
+    lo = np.stack([row for (_, _, _, _, row) in res["logits"]]).astype(np.float64)
+    lp = np.stack([row for (_, _, _, _, row) in res["plain"]["logits"]]).astype(np.float64)
+    rms = lambda x: float(np.sqrt(np.mean(x * x)))
+    same_trace = [(r["admitted"], r["scheduled"], r["allocated"], r["finished"], r["freed"]) for r in trace] == \
+                 [(r["admitted"], r["scheduled"], r["allocated"], r["finished"], r["freed"]) for r in res["trace"]]
+    toks = B.tokens_by_ticket(ev)
+    agree = sum(toks[t][i] == res["sampled"][t][i] for t in toks for i in range(len(toks[t])))
+    return dict(rows=int(lg.shape[0]), logit_std=float(lp.std()), trace_equal=bool(same_trace),
+                parity_max_abs=float(np.abs(lg - lo).max()), parity_rms=rms(lg - lo),
+                vs_plain_oracle_max_abs=float(np.abs(lg - lp).max()), vs_plain_oracle_rms=rms(lg - lp),
+                oracle_rounding_noise_max_abs=float(np.abs(lo - lp).max()), oracle_rounding_noise_rms=rms(lo - lp),
+                sampled_tokens_equal=f"{agree}/{total}",
+                note="gpu logits vs the CPU oracle on the cpu_baseline sample (full model, teacher-forced); "
+                     "parity_* against the oracle with the data path's 16-bit rounding points, vs_plain_* against the "
+                     "oracle without them; oracle_rounding_noise_* is the distance between those two oracles")
 
 
 # ----------------------------------------------------------------------------------------------
@@ -261,8 +309,8 @@ def realtime_run(B, m, sched, wbuf, kv, reqs, time_limit_s, use_arrivals=True, w
         n_expected = 0
         evs = []
         t0 = time.monotonic()
+        t0_ns = time.monotonic_ns()
         i = 0
-        h2d = 0
         got = 0
         done_req = 0
         while True:
@@ -273,7 +321,6 @@ def realtime_run(B, m, sched, wbuf, kv, reqs, time_limit_s, use_arrivals=True, w
                     break
                 if rc < 0:
                     raise B.BlinkError(rc, "blink_submit")
-                h2d += reqs[i].n_prompt * 4 + 64
                 n_expected += reqs[i].max_new
                 i += 1
             e = eng.blink_poll(4096, 200)
@@ -287,7 +334,12 @@ def realtime_run(B, m, sched, wbuf, kv, reqs, time_limit_s, use_arrivals=True, w
         st = eng.blink_get_stats()
         ev = np.concatenate(evs) if evs else np.zeros(0, dtype=B.EVENT_DTYPE)
         its = int(st.iterations)
-        ttft, tpot = [], []
+        # device-side figures (token publish times on the device clock): the paper's claim, its frontend
+        # sits on the SmartNIC and not on the interfered host; host-side figures (when blink_poll saw
+        # the token) and the submit lag show what the stand-in frontend on the host adds
+        ttft, tpot, ttft_h, tpot_h, lag = [], [], [], [], []
+        done_s = {}   # ticket -> seconds from the start of the run until the host saw its last token
+        by_ticket = {r.ticket: r for r in reqs}
         if len(ev):
             ev = np.sort(ev, order=["ticket", "index"])
             bounds = np.flatnonzero(np.diff(ev["ticket"].astype(np.int64)) != 0) + 1
@@ -295,12 +347,21 @@ def realtime_run(B, m, sched, wbuf, kv, reqs, time_limit_s, use_arrivals=True, w
                 first = seg[seg["index"] == 0]
                 if len(first):
                     ttft.append((int(first["t_device_ns"][0]) + off - int(first["t_submit_ns"][0])) / 1e6)
+                    ttft_h.append((int(first["t_host_ns"][0]) - int(first["t_submit_ns"][0])) / 1e6)
+                    if use_arrivals:
+                        arr_ns = t0_ns + int(by_ticket[int(first["ticket"][0])].arrival_s * 1e9)
+                        lag.append((int(first["t_submit_ns"][0]) - arr_ns) / 1e6)
+                if seg["is_last"][-1]:
+                    done_s[int(seg["ticket"][-1])] = (int(seg["t_host_ns"][-1]) - t0_ns) / 1e9
                 if seg["is_last"][-1] and len(seg) > 1:
                     tpot.append((int(seg["t_device_ns"][-1]) - int(seg["t_device_ns"][0])) / 1e6 / (len(seg) - 1))
+                    tpot_h.append((int(seg["t_host_ns"][-1]) - int(seg["t_host_ns"][0])) / 1e6 / (len(seg) - 1))
         return dict(tokens=got, elapsed_s=elapsed, tok_s=got / elapsed if elapsed > 0 else 0.0,
                     requests_submitted=i, requests_completed=done_req, iterations=its,
-                    h2d_bytes=h2d, d2h_bytes=got * 16, ttft_ms=percentiles(ttft), tpot_ms=percentiles(tpot),
-                    device_status=int(st.device_status))
+                    h2d_bytes=int(st.bytes_to_device), d2h_bytes=int(st.bytes_from_device),
+                    ttft_ms=percentiles(ttft), tpot_ms=percentiles(tpot),
+                    ttft_host_ms=percentiles(ttft_h), tpot_host_ms=percentiles(tpot_h), submit_lag_ms=percentiles(lag),
+                    done_s=done_s, device_status=int(st.device_status))
     finally:
         rc = eng.blink_destroy()
         if rc != B.BLINK_OK:
@@ -314,7 +375,7 @@ def main():
     ap.add_argument("--steps", type=int, default=30)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="blink", choices=["blink", "reference"])
-    ap.add_argument("--config", type=int, default=3, help="BASELINE configuration (1..4)")
+    ap.add_argument("--config", type=int, default=3, help="BASELINE configuration (1..5)")
     ap.add_argument("--ramp", type=int, default=-1, help="untimed iterations that bring the batch to steady state")
     ap.add_argument("--gemm", default="auto", choices=["auto", "simt", "tc"])
     ap.add_argument("--weights", default="streaming", choices=["streaming", "row-major"],
@@ -322,7 +383,12 @@ def main():
     ap.add_argument("--rate", type=float, default=16.0, help="offered load of the real-time run (req/s)")
     ap.add_argument("--e2e-seconds", type=float, default=15.0)
     ap.add_argument("--latency-seconds", type=float, default=20.0)
-    ap.add_argument("--interfere", action="store_true", help="run the host-CPU stressor during the real-time run")
+    ap.add_argument("--interfere", default="both", choices=["both", "off", "on"],
+                    help="real-time run with the host idle, with the host-CPU stressor, or both (default: both, with ratios)")
+    ap.add_argument("--rates", default="", help="offered-load sweep, e.g. 'all' (the 13 levels) or '4,8,16': one real-time run per "
+                    "rate; reports the highest rate whose goodput reaches 0.95 x offered")
+    ap.add_argument("--rate-seconds", type=float, default=30.0, help="measurement window per rate of the sweep")
+    ap.add_argument("--skip-parity", action="store_true")
     ap.add_argument("--skip-cpu", action="store_true")
     ap.add_argument("--skip-e2e", action="store_true")
     ap.add_argument("--skip-latency", action="store_true")
@@ -393,11 +459,12 @@ def main():
     log(f"[bench] weights {wbuf.numel() / 1e9:.2f} GB on {dev} in {time.time() - t_setup:.1f}s")
 
     # ---- CPU oracle beside it (rank 0, N = 1 only) ----------------------------------------
-    cpu_baseline = None
+    cpu_baseline, cpu_res = None, None
     if rank == 0 and world == 1 and not args.skip_cpu:
         try:
             n_req, cap, new = (4, 64, 8) if cfg_i >= 2 else (8, 64, 32)
-            cpu_baseline, _, _ = cpu_oracle_sample(m, sched, wbuf, n_req, cap, new, cfg_i)
+            cpu_baseline, cpu_res, _ = cpu_oracle_sample(m, sched, wbuf, n_req, cap, new, cfg_i,
+                                                         keep_logits=not args.skip_parity and cfg_i != 5)
             log(f"[bench] cpu oracle: {cpu_baseline['value']:.2f} tok/s ({cpu_baseline['sample']})")
         except Exception as e:  # a baseline, never a reason to lose the measurement
             cpu_baseline = dict(value=None, unit="output tok/s", cores=os.cpu_count(), kind="oracle",
@@ -407,6 +474,15 @@ def main():
     if args.weights == "streaming" and m.dtype == "bf16" and args.gemm != "simt":
         B.blink_convert_weights(m, wbuf, B.WEIGHTS_ROW_MAJOR, B.WEIGHTS_STREAMING)   # set-up, once, in place
         wl = B.WEIGHTS_STREAMING
+    parity = None
+    if cpu_res is not None and "plain" in cpu_res:
+        try:
+            parity = parity_on_sample(B, m, wbuf, wl, cpu_res)
+            log(f"[bench] parity on the oracle sample: max-abs {parity['parity_max_abs']:.3e} (the two oracles differ by "
+                f"{parity['oracle_rounding_noise_max_abs']:.3e}), trace equal: {parity['trace_equal']}")
+        except Exception as e:
+            parity = dict(parity_max_abs=None, note=f"failed: {e!r}")
+        cpu_res = None
     # ---- KV pool: a fraction of what is free after the weights ---------------------------
     free, total = torch.cuda.mem_get_info(dev)
     lib_reserve = 6 << 30      # ring, arenas, activations and logits the library allocates itself
@@ -518,7 +594,7 @@ def main():
                 dtype="bf16" if m.dtype == "bf16" else "f32", data="synthetic",
                 config=dict(workload=workload, requests=len(reqs), max_batch=sched.max_batch,
                             prefill_chunk_tokens=sched.prefill_chunk_tokens, kv_blocks=n_blocks,
-                            ramp_iterations=ramp, sampling="top-k 50, T 0.8" if cfg_i >= 3 else "greedy",
+                            ramp_iterations=ramp, sampling="top-k 50, T 0.8" if cfg_i in (3, 4) else "greedy",
                             l2="per-step inputs (weights + KV) exceed L2 many times over; no flush needed",
                             rows_per_step=float(its["n_tokens"].mean()),
                             decode_rows_per_step=float(its["n_decode"].mean()),
@@ -530,6 +606,8 @@ def main():
                 control_plane_us=dict(p50=float(np.median(ctrl_us)), max=float(ctrl_us.max())))
     if cpu_baseline is not None:
         line["cpu_baseline"] = cpu_baseline
+    if parity is not None:
+        line["parity"] = parity
 
     # ---- decode-only operating points (fixed batch): the HBM-bound regime ---------------------
     if args.decode_points and rank == 0 and world == 1 and not args.closed_batch:
@@ -553,20 +631,75 @@ def main():
                            requests_completed=r["requests_completed"], iterations=r["iterations"],
                            note="all requests submitted from host memory at t=0 through blink_submit, tokens "
                                 "read with blink_poll, persistent loop; wall clock from first submit")
-    # ---- real-time run at the offered load: latency ----------------------------------------
-    if not args.skip_latency and rank == 0 and world == 1:
-        stress = Stressor() if args.interfere else None
+    # ---- real-time run at the offered load: latency, host idle and host stressed -----------------
+    def latency_leg(stressed, rate_reqs, seconds):
+        stress = Stressor() if stressed else None
         if stress:
             stress.start()
         try:
-            lreqs = [q for q in reqs if q.arrival_s <= args.latency_seconds]
-            r = realtime_run(B, m, sched, wbuf, kv, lreqs, args.latency_seconds * 3, use_arrivals=True, weights_layout=wl)
+            lreqs = [q for q in rate_reqs if q.arrival_s <= seconds]
+            r = realtime_run(B, m, sched, wbuf, kv, lreqs, seconds * 3, use_arrivals=True, weights_layout=wl)
         finally:
             if stress:
                 stress.stop()
-        line["latency"] = dict(offered_req_s=args.rate, host="stressed" if args.interfere else "idle",
-                               requests=len(lreqs), completed=r["requests_completed"], tok_s=r["tok_s"],
-                               ttft_ms=r["ttft_ms"], tpot_ms=r["tpot_ms"], seconds=r["elapsed_s"])
+        offered_tok = sum(q.max_new for q in lreqs)
+        return dict(host="stressed" if stressed else "idle", requests=len(lreqs), completed=r["requests_completed"],
+                    tok_s=r["tok_s"], goodput_req_s=r["requests_completed"] / r["elapsed_s"] if r["elapsed_s"] > 0 else 0.0,
+                    tokens=r["tokens"], offered_tokens=offered_tok, ttft_ms=r["ttft_ms"], tpot_ms=r["tpot_ms"],
+                    ttft_host_ms=r["ttft_host_ms"], tpot_host_ms=r["tpot_host_ms"], submit_lag_ms=r["submit_lag_ms"],
+                    seconds=r["elapsed_s"], done_s=r["done_s"])
+
+    if not args.skip_latency and rank == 0 and world == 1:
+        legs = {}
+        if args.interfere in ("both", "off"):
+            legs["isolated"] = latency_leg(False, reqs, args.latency_seconds)
+        if args.interfere in ("both", "on"):
+            legs["interfered"] = latency_leg(True, reqs, args.latency_seconds)
+        for v in legs.values():
+            v.pop("done_s", None)
+        lat = dict(offered_req_s=args.rate, **legs,
+                   note="ttft_ms / tpot_ms use the device publish times (the paper's frontend sits on the SmartNIC, not on "
+                        "the interfered host); *_host_ms use the time blink_poll saw the token on the (stressed) host; "
+                        "submit_lag_ms = blink_submit time minus scheduled arrival")
+        if "isolated" in legs and "interfered" in legs:
+            a, b = legs["isolated"], legs["interfered"]
+            ratio = lambda x, y: (y / x) if (x and y) else None
+            # interfered / isolated, the bracketed figures of the paper's Table 7
+            lat["ratios"] = dict(ttft_p99=ratio(a["ttft_ms"]["p99"], b["ttft_ms"]["p99"]),
+                                 tpot_p99=ratio(a["tpot_ms"]["p99"], b["tpot_ms"]["p99"]),
+                                 tpot_p50=ratio(a["tpot_ms"]["p50"], b["tpot_ms"]["p50"]),
+                                 throughput=ratio(a["tok_s"], b["tok_s"]),
+                                 ttft_host_p99=ratio(a["ttft_host_ms"]["p99"], b["ttft_host_ms"]["p99"]),
+                                 tpot_host_p99=ratio(a["tpot_host_ms"]["p99"], b["tpot_host_ms"]["p99"]))
+        line["latency"] = lat
+    # ---- offered-load sweep (Section 6.1: 13 levels between 1 and 32 req/s; Appendix C: serviceable load) ----
+    if args.rates and rank == 0 and world == 1:
+        from synth.workload import RATE_LEVELS
+        levels = RATE_LEVELS if args.rates == "all" else [float(v) for v in args.rates.split(",")]
+        sweep, serviceable = [], None
+        for lv in levels:
+            rr = make_requests(cfg_i, rate=float(lv))
+            leg = latency_leg(False, rr, args.rate_seconds)
+            leg["offered_req_s"] = float(lv)
+            # window [0, W]: requests arriving in the first part of it, [0, W - D], are the offered load; those of
+            # them whose last token the host saw by W are the goodput (D = 12 s or 0.4 W lets all but the very
+            # longest generations finish when nothing queues)
+            Wn = args.rate_seconds
+            D = min(12.0, 0.4 * Wn)
+            early = [q for q in rr if q.arrival_s <= Wn - D]
+            good = sum(1 for q in early if leg["done_s"].get(q.ticket, 1e30) <= Wn)
+            offered = len(early) / (Wn - D)
+            leg["goodput_req_s"] = good / (Wn - D)
+            leg["goodput_over_offered"] = good / len(early) if early else None
+            leg.pop("done_s", None)
+            sweep.append(leg)
+            if leg["goodput_over_offered"] is not None and leg["goodput_over_offered"] >= 0.95:
+                serviceable = float(lv)
+            log(f"[bench] rate {lv}: goodput {leg['goodput_req_s']:.2f} req/s of {offered:.2f} offered, "
+                f"TPOT p99 {leg['tpot_ms']['p99']}")
+        line["rate_sweep"] = dict(levels=sweep, serviceable_req_s=serviceable,
+                                  rule="highest offered rate at which at least 0.95 of the requests that arrived in the "
+                                       "first W - D seconds of the W-second window had their last token by its end")
     if rank == 0:
         print(json.dumps(line), flush=True)
     if world > 1:

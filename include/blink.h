@@ -118,7 +118,11 @@ typedef struct blink_sched_cfg {
   int32_t gemm_impl;            /* BLINK_GEMM_*                                                 */
   int32_t control_only;         /* 1: no model math, tokens come from a fixed hash (trace tests) */
   int32_t start_paused;         /* 1: the loop admits nothing until blink_start                 */
-  int32_t reserved0;
+  int32_t wait_limit_ms;        /* bound of every wait inside the kernel (grid barrier, copy / MMA pipeline
+                                   barriers): a wait that lasts longer ends the loop with device_status
+                                   set and BLINK_LOOP_EXIT_ERROR.  0 = idle_exit_us + 3 s.  CTAs wait at a
+                                   grid barrier while the control plane polls an empty queue, so a limit
+                                   below idle_exit_us turns an idle period into a time-out error          */
   int64_t iteration_budget;     /* iterations per kernel launch, 0 = unbounded                  */
   int64_t idle_exit_us;         /* leave the GPU after this long without work, 0 = 2 s          */
   int64_t trace_capacity_words; /* int32 words of scheduling trace kept on the device, 0 = off  */
@@ -175,6 +179,10 @@ typedef struct blink_stats {
   int64_t trace_words;    /* valid words in the trace                             */
   int64_t device_clock_offset_ns; /* host CLOCK_MONOTONIC minus device global timer at create */
   int32_t free_blocks, reserved_blocks, batch_live, reserved1;
+  int64_t bytes_to_device;   /* bytes blink_submit wrote into the mapped submit areas (entries, prompts,
+                                forced tokens) since create                                          */
+  int64_t bytes_from_device; /* bytes blink_poll read from the device-written mirrors (count words it
+                                looked at, tokens and timestamps it handed out) since create         */
 } blink_stats;
 
 /* One record per traced iteration, for throughput / roofline arithmetic. */

@@ -39,7 +39,7 @@ class blink_sched_cfg(C.Structure):
     _fields_ = [("size", C.c_uint32), ("max_batch", C.c_int32), ("prefill_chunk_tokens", C.c_int32),
                 ("n_slots", C.c_int32), ("max_prompt", C.c_int32), ("max_new", C.c_int32), ("exec_mode", C.c_int32),
                 ("gemm_impl", C.c_int32), ("control_only", C.c_int32), ("start_paused", C.c_int32),
-                ("reserved0", C.c_int32), ("iteration_budget", C.c_int64), ("idle_exit_us", C.c_int64),
+                ("wait_limit_ms", C.c_int32), ("iteration_budget", C.c_int64), ("idle_exit_us", C.c_int64),
                 ("trace_capacity_words", C.c_int64), ("stats_capacity_iters", C.c_int64),
                 ("logits_capture", C.c_void_p), ("logits_capture_rows", C.c_int64)]
 
@@ -66,7 +66,8 @@ class blink_stats(C.Structure):
                 ("n_blocks", C.c_int32), ("iterations", C.c_int64), ("launches", C.c_int64),
                 ("tokens_out", C.c_int64), ("prompt_tokens", C.c_int64), ("trace_words", C.c_int64),
                 ("device_clock_offset_ns", C.c_int64), ("free_blocks", C.c_int32), ("reserved_blocks", C.c_int32),
-                ("batch_live", C.c_int32), ("reserved1", C.c_int32)]
+                ("batch_live", C.c_int32), ("reserved1", C.c_int32), ("bytes_to_device", C.c_int64),
+                ("bytes_from_device", C.c_int64)]
 
 
 class blink_iter_stat(C.Structure):
@@ -274,7 +275,7 @@ class Blink:
 
     def __init__(self, model, sched, weights=None, kv_pool=None, *, exec_mode=EXEC_PERSISTENT, gemm_impl=GEMM_AUTO,
                  control_only=False, start_paused=False, iteration_budget=0, idle_exit_us=0, trace_words=0,
-                 stats_iters=0, logits_capture=None, kv_bytes=None, weights_layout=WEIGHTS_ROW_MAJOR):
+                 stats_iters=0, logits_capture=None, kv_bytes=None, weights_layout=WEIGHTS_ROW_MAJOR, wait_limit_ms=0):
         L = lib()
         self.model, self.sched = model, sched
         self._keep = (weights, kv_pool, logits_capture)
@@ -285,7 +286,7 @@ class Blink:
         cap_rows = logits_capture.shape[0] if logits_capture is not None else 0
         sc = blink_sched_cfg(C.sizeof(blink_sched_cfg), sched.max_batch, sched.prefill_chunk_tokens, sched.n_slots,
                              sched.max_prompt, sched.max_new, exec_mode, gemm_impl, int(control_only),
-                             int(start_paused), 0, iteration_budget, idle_exit_us, trace_words, stats_iters,
+                             int(start_paused), wait_limit_ms, iteration_budget, idle_exit_us, trace_words, stats_iters,
                              cap_ptr, cap_rows)
         if kv_pool is not None:
             kv = blink_kv_pool(C.sizeof(blink_kv_pool), sched.block_size, kv_pool.data_ptr(),

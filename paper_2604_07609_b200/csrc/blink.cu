@@ -159,6 +159,7 @@ struct blink_ctx {
   int hint = 0;
   uint64_t next_ticket = 0;
   int64_t launches = 0;
+  int64_t bytes_to_device = 0, bytes_from_device = 0;
   int64_t clock_offset = 0;
   bool final_stop = false;
   int n_sms = 1;
@@ -270,7 +271,7 @@ int step_once(blink_ctx* x) {
         if (x->dc.E > 0 && (ph == PH_GU || ph == PH_DOWN)) {
           if (ph == PH_GU) launch_phase(x, PH_MOE_GROUP, l);
           for (int e = 0; e < x->dc.E; ++e) launch_phase(x, ph, l, e);
-        } else {
+        } else if (!(x->dc.fused && (ph == PH_ROPE || ph == PH_SILU))) {   // fused into the GEMM epilogues
           launch_phase(x, ph, l);
         }
       }
@@ -461,7 +462,7 @@ int blink_create(const blink_model_cfg* model, const blink_sched_cfg* sched, con
   if (!model_ok(model) || !sched || sched->size != sizeof(blink_sched_cfg) || !kv || kv->size != sizeof(blink_kv_pool))
     return BLINK_EINVAL;
   if (sched->max_batch < 1 || sched->max_batch > MAX_BATCH || sched->prefill_chunk_tokens < 1 || sched->n_slots < 1 ||
-      sched->max_prompt < 1 || sched->max_new < 1)
+      sched->max_prompt < 1 || sched->max_new < 1 || sched->wait_limit_ms < 0)
     return BLINK_EINVAL;
   if (kv->block_size != 16) return BLINK_EINVAL;
   if (!sched->control_only && (model->weights == nullptr || model->weights_bytes < blink_weights_bytes(model)))
@@ -508,6 +509,10 @@ int blink_create(const blink_model_cfg* model, const blink_sched_cfg* sched, con
   if (!c.control_only && model->dtype == BLINK_DTYPE_BF16 && sched->gemm_impl != BLINK_GEMM_SIMT)
     c.gemm_tc = tc_available() && tc_shape_ok(c);
   if (sched->gemm_impl == BLINK_GEMM_TC && !c.gemm_tc) { delete x; return BLINK_EINVAL; }
+  // epilogue fusion needs whole 128-feature tiles that do not straddle q|k|v or gate|up
+  c.fused = c.gemm_tc && c.qkv_dim % 128 == 0 && c.q_dim % 128 == 0 && c.kv_dim % 128 == 0 && c.F % 128 == 0 &&
+            c.d % 128 == 0 && 128 % c.hd == 0;
+  c.fused_norm = c.fused && c.E == 0;
   c.w_streaming = model->weights_layout == BLINK_WEIGHTS_STREAMING;
   if (model->weights_layout != BLINK_WEIGHTS_ROW_MAJOR && model->weights_layout != BLINK_WEIGHTS_STREAMING) { delete x; return BLINK_EINVAL; }
   // the streaming layout is read by the tensor-core path only
@@ -516,7 +521,8 @@ int blink_create(const blink_model_cfg* model, const blink_sched_cfg* sched, con
   const double cyc_per_us = 2000.0;  // upper bound on the SM clock: time-outs only get longer at lower clocks
   const int64_t idle_us = sched->idle_exit_us > 0 ? sched->idle_exit_us : 2000000;
   c.idle_exit_cycles = (unsigned long long)(idle_us * cyc_per_us);
-  c.barrier_timeout_cycles = (unsigned long long)((idle_us + 3000000) * cyc_per_us);
+  c.barrier_timeout_cycles = sched->wait_limit_ms > 0 ? (unsigned long long)(sched->wait_limit_ms * 1000.0 * cyc_per_us)
+                                                      : (unsigned long long)((idle_us + 3000000) * cyc_per_us);
   c.kv_base = kv->base;
   c.trace_cap = sched->trace_capacity_words;
   c.stats_cap = sched->stats_capacity_iters;
@@ -593,6 +599,7 @@ int blink_create(const blink_model_cfg* model, const blink_sched_cfg* sched, con
       TRY(dev_alloc(x, &c.moe_tok, RA)); TRY(dev_alloc(x, &c.moe_gate, RA));
     }
     TRY(dev_alloc(x, &p, MB * c.d * esz)); c.xs = p;
+    TRY(dev_alloc(x, &c.rowss_a, TM)); TRY(dev_alloc(x, &c.rowss_b, TM)); TRY(dev_alloc(x, &c.tile_cnt, (size_t)TILE_CNT_SLOTS));
     TRY(dev_alloc(x, &c.logits, MB * c.V));
     TRY(dev_alloc(x, &c.rope_cos, (size_t)c.max_pos * (c.hd / 2), false));
     TRY(dev_alloc(x, &c.rope_sin, (size_t)c.max_pos * (c.hd / 2), false));
@@ -715,6 +722,7 @@ int blink_submit(blink_ctx* x, const blink_request* r, uint64_t* ticket_out) {
   SlotInfo& si = x->slots[slot];
   si.busy = true; si.ticket = ticket; si.user_tag = r->user_tag; si.max_new = r->max_new_tokens; si.consumed = 0;
   si.t_submit_ns = now_ns();
+  x->bytes_to_device += (int64_t)sizeof(SubEntry) + 8 + (int64_t)r->n_prompt * 4 + (r->forced_tokens ? (int64_t)r->max_new_tokens * 4 : 0);
   x->active.push_front(slot);  // new slots are looked at first by the token reader
   // payload first, then the tail that makes it visible
   std::atomic_thread_fence(std::memory_order_release);
@@ -739,6 +747,7 @@ int blink_poll(blink_ctx* x, blink_token_event* out, int max_events, int timeout
         const int slot = *it;
         SlotInfo& si = x->slots[slot];
         const uint32_t cnt = __atomic_load_n(&x->out_count[slot], __ATOMIC_ACQUIRE);
+        x->bytes_from_device += 4;
         const int have = (int)(cnt & 0x7fffffffu);
         const bool fin = (cnt >> 31) != 0;
         while (si.consumed < have && n < max_events) {
@@ -752,6 +761,7 @@ int blink_poll(blink_ctx* x, blink_token_event* out, int max_events, int timeout
           ev.t_host_ns = t_now;
           ev.t_submit_ns = si.t_submit_ns;
           si.consumed += 1;
+          x->bytes_from_device += 12;   // token + timestamp
         }
         if (fin && si.consumed == have) {
           si.busy = false;  // DECODE_COMPLETED -> EMPTY: the frontend owns this transition
@@ -859,6 +869,8 @@ int blink_get_stats(blink_ctx* x, blink_stats* out) {
   for (int v : ph) live += v != PHASE_FREE;
   out->batch_live = live;
   out->reserved1 = 0;
+  out->bytes_to_device = x->bytes_to_device;
+  out->bytes_from_device = x->bytes_from_device;
   return BLINK_OK;
 }
 

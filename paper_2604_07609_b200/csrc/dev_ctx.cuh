@@ -124,6 +124,7 @@ constexpr int CTRL_THREADS = 256;
 constexpr int MAX_BATCH = 256;
 constexpr int MAX_TOPK = 64;
 constexpr int MAX_EXPERTS = 16;
+constexpr int TILE_CNT_SLOTS = 8192;
 
 struct DevCtx {
   // model
@@ -191,6 +192,12 @@ struct DevCtx {
   int32_t* moe_off;    // [E+1] first gathered row of each expert
   int32_t* moe_tok;    // [Tmax*topE] token of a gathered row
   float* moe_gate;     // [Tmax*topE] its weight
+  // fused epilogues of the tensor-core path
+  float* rowss_a;      // [Tmax] sum of squares of the residual rows after the O GEMM (input of the second norm)
+  float* rowss_b;      // [Tmax] the same after the down GEMM (input of the next layer's first norm / the final norm)
+  int32_t* tile_cnt;   // [TILE_CNT_SLOTS] k-blocks delivered per output tile of the running GEMM; self-resetting
+  int fused;           // 1: RoPE + KV write and SwiGLU run in the epilogues of the QKV and gate/up GEMMs
+  int fused_norm;      // 1: the O and down epilogues add up sum(x^2) per row and the norms are element-wise
   float* logits;  // [MB][V]
   float *rope_cos, *rope_sin;  // [max_pos][hd/2]
   void* kv_base;               // [L][2][n_blocks][Hkv][bs][hd] operand type

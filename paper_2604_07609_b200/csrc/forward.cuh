@@ -186,15 +186,52 @@ static __device__ void phase_norm(const DevCtx& c, int layer, int which /*0: nor
   const int T = c.ss->cur_T;
   const float* g = wptr_f(c, which == 0 ? 6 : 7) + (size_t)layer * c.d;
   WT* out = reinterpret_cast<WT*>(c.xn);
-  // The split-K tensor-core GEMMs add partial sums into their outputs.  Those are cleared during
-  // the O GEMM by a warp that has no role there (the gate/up buffer of this layer and the QKV
-  // buffer of the next); only the first layer's QKV buffer is cleared here.
-  if (c.gemm_tc && which == 0 && layer == 0) zero_floats(c.qkv, (long long)T * c.qkv_dim);
+  // fused path: both sum-of-squares buffers start a step at zero (the last layer's leftovers)
+  if (c.fused_norm && which == 0 && layer == 0)
+    for (int i = blockIdx.x * FWD_THREADS + threadIdx.x; i < c.Tmax; i += gridDim.x * FWD_THREADS) {
+      c.rowss_a[i] = 0.f;
+      c.rowss_b[i] = 0.f;
+    }
   const float* wr = (which == 1 && c.E > 0) ? wptr_f(c, 5) + (size_t)layer * c.E * c.d : nullptr;
   for (int t = blockIdx.x; t < T; t += gridDim.x) {
     const WT* e = (which == 0 && layer == 0) ? wptr<WT>(c, 0) + (size_t)c.tok_id[t] * c.d : nullptr;
     norm_row_cta<WT>(c, c.h + (size_t)t * c.d, e, g, out + (size_t)t * c.d, s_red, wr, t);
   }
+}
+
+// The LM head gives every CTA whole weight tiles when there are at least as many tiles as CTAs: no
+// partial sums, so the logits need no clearing.
+__device__ __forceinline__ bool lm_head_whole_tiles(const DevCtx& c) { return (c.V + 127) / 128 >= (int)gridDim.x; }
+
+// Fused path: the sum of squares of every residual row is already known (added up by the epilogue of
+// the GEMM that completed the row), so the norm is element-wise: n = x * rsqrt(ss / d + eps) * g.
+// `rows` null: rows 0 .. R-1 of h go to rows 0 .. R-1 of out; else row r of out comes from row rows[r].
+template <typename WT>
+__device__ __noinline__ void norm_apply_rows(const float* __restrict__ h, const float* __restrict__ rowss,
+                                             const float* __restrict__ g, WT* __restrict__ out, const int32_t* rows, int R,
+                                             int d, float eps) {
+  const int d4 = d >> 2;
+  const int total = R * d4;   // < 2^31
+  const float inv_d = 1.0f / (float)d;
+  for (int idx = blockIdx.x * FWD_THREADS + threadIdx.x; idx < total; idx += gridDim.x * FWD_THREADS) {
+    const int r = idx / d4, j = (idx - r * d4) * 4;
+    const int t = rows != nullptr ? rows[r] : r;
+    const float4 v = __ldcg(reinterpret_cast<const float4*>(h + (size_t)t * d + j));
+    const float inv = 1.0f / sqrtf(__ldcg(rowss + t) * inv_d + eps);
+    const float4 gg = *reinterpret_cast<const float4*>(g + j);
+    store4<WT>(out + (size_t)r * d + j, v.x * inv * gg.x, v.y * inv * gg.y, v.z * inv * gg.z, v.w * inv * gg.w);
+  }
+}
+
+// Norm phases of the fused path for layers whose input rows are complete with their sums of squares:
+// which 0 = first norm of layer > 0 (reads rowss_b, clears rowss_a), 1 = second norm (reads rowss_a,
+// clears rowss_b).  The cleared buffer is the one the next GEMM epilogue adds into.
+template <typename WT>
+static __device__ void phase_norm_apply(const DevCtx& c, int layer, int which, int T) {
+  const float* g = wptr_f(c, which == 0 ? 6 : 7) + (size_t)layer * c.d;
+  float* clear = which == 0 ? c.rowss_a : c.rowss_b;
+  for (int i = blockIdx.x * FWD_THREADS + threadIdx.x; i < T; i += gridDim.x * FWD_THREADS) clear[i] = 0.f;
+  norm_apply_rows<WT>(c.h, which == 0 ? c.rowss_b : c.rowss_a, g, reinterpret_cast<WT*>(c.xn), nullptr, T, c.d, c.rms_eps);
 }
 
 // Final norm of the sampled rows only (the LM head runs on those rows).
@@ -204,13 +241,23 @@ static __device__ void phase_final_norm(const DevCtx& c) {
   const int R = c.ss->cur_rows;
   const float* g = wptr_f(c, 8);
   WT* out = reinterpret_cast<WT*>(c.xs);
-  if (c.gemm_tc) zero_floats(c.logits, (long long)R * c.V);
+  if (c.gemm_tc && !lm_head_whole_tiles(c)) zero_floats(c.logits, (long long)R * c.V);
+  if (c.fused_norm) {
+    norm_apply_rows<WT>(c.h, c.rowss_b, g, out, c.row_tok, R, c.d, c.rms_eps);
+    return;
+  }
   for (int r = blockIdx.x; r < R; r += gridDim.x)
     norm_row_cta<WT>(c, c.h + (size_t)c.row_tok[r] * c.d, nullptr, g, out + (size_t)r * c.d, s_red);
 }
 
 // ---- CUDA-core reference GEMM: out[t][n] (+)= sum_k x[t][k] * w[n][k], fp32 accumulate.
 // 64x64 output tile, BK = 16, 4x4 outputs per thread.  Deterministic (no split-K).
+enum GemmFix : int {
+  FIX_NONE = 0,
+  FIX_ROPE_KV,  // QKV: RoPE on q and k, q -> 16-bit attention operand, k and v -> paged pool; the tile is cleared
+  FIX_SILU,     // gate/up: act = silu(gate) * up in the operand type; both tiles are cleared
+  FIX_SUMSQ,    // O and down: add the tile's share of sum(x^2) of every residual row
+};
 struct GemmArgs {
   const void* x;   // [M][K] operand type
   const void* w;   // [N][K] operand type
@@ -224,10 +271,11 @@ struct GemmArgs {
   long long w_row0 = 0;
   const int32_t* row_map = nullptr;
   const float* row_scale = nullptr;
-  // tensor-core path: buffers that the epilogue warps clear at the start of this GEMM (outputs of
-  // later split-K GEMMs, which add partial sums into them); counts in floats, multiples of 4
-  float* zero_p[2] = {nullptr, nullptr};
-  long long zero_n[2] = {0, 0};
+  // tensor-core path: element-wise work that consumes the finished output tiles of this GEMM (run by
+  // the CTA that delivers a tile's last partial sum, see tc_finish_tiles)
+  int fix = 0;               // FIX_*
+  void* fix_out = nullptr;   // FIX_SILU: the activation rows (operand type) matching `out`
+  float* fix_rowss = nullptr;// FIX_SUMSQ: per-row sums of squares to add to
 };
 
 template <typename WT>
@@ -349,6 +397,91 @@ static __device__ void phase_rope_kv(const DevCtx& c, int layer) {
       store4<WT>(dst + i, x1.x, x1.y, x1.z, x1.w);
       store4<WT>(dst + i + half, x2.x, x2.y, x2.z, x2.w);
     }
+  }
+}
+
+// ---- element-wise consumers of finished GEMM output tiles (fused path) ----------------------------
+// A tile is 128 consecutive output features of rows [t0, t1); the eight warps take rows in turn and a
+// lane owns four consecutive features, so every access is one 512-byte line per row.  The fp32 sums
+// were produced by reductions at L2 by several CTAs: they are read with .cg loads.
+
+// QKV tile nt: RoPE on the q and k heads it covers (the rotation partner i + hd/2 of a feature lies in
+// the same tile, hd/8 lanes away), q into the 16-bit attention operand, k and v into the paged pool;
+// then the tile is cleared for the next GEMM that adds partial sums into this buffer.
+template <typename WT>
+__device__ __noinline__ void fixup_rope_kv(const DevCtx& c, int layer, int nt, int t0, int t1) {
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const int hd = c.hd, half = hd >> 1;
+  const int f = nt * 128 + lane * 4;          // feature of this lane
+  const int hh = f / hd, i0 = f - hh * hd;    // head and offset inside it
+  const bool low = i0 < half;
+  const int i = low ? i0 : i0 - half;         // rotation pair index
+  const int partner = half >> 2;              // lanes between the two halves of a pair
+  if (f >= c.qkv_dim) return;                 // whole warp: tiles are not ragged on this path
+  for (int t = t0 + w; t < t1; t += FWD_THREADS / 32) {
+    float4* src = reinterpret_cast<float4*>(c.qkv + (size_t)t * c.qkv_dim + f);
+    const float4 x = __ldcg(src);
+    float4 o;
+    o.x = __shfl_xor_sync(0xffffffffu, x.x, partner);
+    o.y = __shfl_xor_sync(0xffffffffu, x.y, partner);
+    o.z = __shfl_xor_sync(0xffffffffu, x.z, partner);
+    o.w = __shfl_xor_sync(0xffffffffu, x.w, partner);
+    float4 y = x;
+    if (hh < c.Hq + c.Hkv) {
+      const int pos = c.tok_pos[t];
+      const float4 cs = *reinterpret_cast<const float4*>(c.rope_cos + (size_t)pos * half + i);
+      const float4 sn = *reinterpret_cast<const float4*>(c.rope_sin + (size_t)pos * half + i);
+      // the same explicit fused forms as the stand-alone RoPE phase: x1 = low half, x2 = high half
+      if (low) {
+        y = make_float4(fmaf(x.x, cs.x, -__fmul_rn(o.x, sn.x)), fmaf(x.y, cs.y, -__fmul_rn(o.y, sn.y)),
+                        fmaf(x.z, cs.z, -__fmul_rn(o.z, sn.z)), fmaf(x.w, cs.w, -__fmul_rn(o.w, sn.w)));
+      } else {
+        y = make_float4(fmaf(x.x, cs.x, __fmul_rn(o.x, sn.x)), fmaf(x.y, cs.y, __fmul_rn(o.y, sn.y)),
+                        fmaf(x.z, cs.z, __fmul_rn(o.z, sn.z)), fmaf(x.w, cs.w, __fmul_rn(o.w, sn.w)));
+      }
+    }
+    WT* dst;
+    if (hh < c.Hq) {
+      dst = reinterpret_cast<WT*>(c.qb) + (size_t)t * c.q_dim + (size_t)hh * hd + i0;
+    } else {
+      const int sm = c.tok_slotmap[t];
+      const int kv = hh < c.Hq + c.Hkv ? 0 : 1;
+      dst = kv_tile<WT>(c, layer, kv, sm / c.bs, hh - c.Hq - kv * c.Hkv) + (size_t)(sm % c.bs) * hd + i0;
+    }
+    store4<WT>(dst, y.x, y.y, y.z, y.w);
+    __stcg(src, make_float4(0.f, 0.f, 0.f, 0.f));
+  }
+}
+
+// gate tile j and up tile j of rows [t0, t1) of `gu` (row pitch 2F): act = silu(gate) * up; both cleared.
+template <typename WT>
+__device__ __noinline__ void fixup_silu(float* gu, WT* act, int F, int j, int t0, int t1) {
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const int f = j * 128 + lane * 4;
+  if (f >= F) return;
+  for (int t = t0 + w; t < t1; t += FWD_THREADS / 32) {
+    float4* gp = reinterpret_cast<float4*>(gu + (size_t)t * 2 * F + f);
+    float4* up = reinterpret_cast<float4*>(gu + (size_t)t * 2 * F + F + f);
+    const float4 g = __ldcg(gp), u = __ldcg(up);
+    store4<WT>(act + (size_t)t * F + f, g.x / (1.0f + __expf(-g.x)) * u.x, g.y / (1.0f + __expf(-g.y)) * u.y,
+               g.z / (1.0f + __expf(-g.z)) * u.z, g.w / (1.0f + __expf(-g.w)) * u.w);
+    __stcg(gp, make_float4(0.f, 0.f, 0.f, 0.f));
+    __stcg(up, make_float4(0.f, 0.f, 0.f, 0.f));
+  }
+}
+
+// residual tile nt of rows [t0, t1): its share of sum(x^2) per row
+static __device__ __noinline__ void fixup_sumsq(const float* h, int ld, int N, float* rowss, int nt, int t0, int t1) {
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const int f = nt * 128 + lane * 4;
+  for (int t = t0 + w; t < t1; t += FWD_THREADS / 32) {
+    float s = 0.f;
+    if (f < N) {
+      const float4 x = __ldcg(reinterpret_cast<const float4*>(h + (size_t)t * ld + f));
+      s = fmaf(x.x, x.x, fmaf(x.y, x.y, fmaf(x.z, x.z, x.w * x.w)));
+    }
+    s = warp_sum(s);
+    if (lane == 0) atomicAdd(rowss + t, s);
   }
 }
 

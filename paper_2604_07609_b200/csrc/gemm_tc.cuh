@@ -48,10 +48,12 @@ struct TcState {
   uint32_t use_bits;    // MMA issuer: stages consumed so far, parity per stage
   uint32_t acc_mma;     // MMA issuer: accumulator buffers claimed, parity per buffer
   uint32_t acc_epi;     // epilogue: accumulator buffers drained, parity per buffer
+  uint32_t last_bit;    // warps 0-3: parity of the next "last accumulator complete" signal
 };
 
 struct TcShared {
   uint64_t full[TC_MAX_STAGES], empty[TC_MAX_STAGES], acc_full[2], acc_empty[2];
+  uint64_t acc_last;   // completes once per GEMM phase, when the CTA's last accumulator is complete
   uint32_t tmem;
   int dead;
 };
@@ -215,11 +217,12 @@ __device__ __forceinline__ bool mbar_wait_idle(const DevCtx& c, uint64_t* bar, u
 // ---- TMEM allocation for the life of the kernel ---------------------------------------------
 __device__ __forceinline__ void tc_init(const DevCtx& c, float*, TcState& s) {
   s.tmem_base = 0;
-  s.fill_bits = s.use_bits = s.acc_mma = s.acc_epi = 0;
+  s.fill_bits = s.use_bits = s.acc_mma = s.acc_epi = s.last_bit = 0;
   if (!c.gemm_tc) return;
   if (threadIdx.x == 32) {
     for (int i = 0; i < TC_MAX_STAGES; ++i) { mbar_init(&g_tc.full[i], 2); mbar_init(&g_tc.empty[i], 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(&g_tc.acc_full[b], 1); mbar_init(&g_tc.acc_empty[b], 4); }
+    mbar_init(&g_tc.acc_last, 1);
     g_tc.dead = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -297,7 +300,7 @@ struct TcGeom {
   uint32_t b_bytes, stage_bytes;
   long long u0, u1;
 };
-__device__ __forceinline__ TcGeom tc_geom(const DevCtx& c, int T, int N, int K) {
+__device__ __forceinline__ TcGeom tc_geom(const DevCtx& c, int T, int N, int K, bool whole_tiles) {
   TcGeom g;
   g.kblocks = K / 64;
   g.ntiles = (N + 127) / 128;
@@ -320,6 +323,12 @@ __device__ __forceinline__ TcGeom tc_geom(const DevCtx& c, int T, int N, int K) 
   g.u1 = total * (blockIdx.x + 1) / gridDim.x;
   g.pass_fixed = -1;
   g.pdiv = g.passes;
+  if (whole_tiles && g.passes == 1) {
+    // every CTA gets whole weight tiles (at most one more than its neighbours): no partial sums at all
+    g.u0 = (long long)g.kblocks * ((long long)g.ntiles * blockIdx.x / gridDim.x);
+    g.u1 = (long long)g.kblocks * ((long long)g.ntiles * (blockIdx.x + 1) / gridDim.x);
+    return g;
+  }
   // More than 256 token rows: the passes of a weight tile go to neighbouring CTAs, which walk the
   // same (weight tile, k-block) range at the same time, so the tile comes from HBM once and from
   // L2 for the others.  One CTA doing the passes in turn re-reads it after the whole grid has
@@ -401,11 +410,59 @@ __device__ __forceinline__ void tc_produce_weights(const DevCtx& c, const void* 
   }
 }
 
+// ---- consumers of finished output tiles -------------------------------------------------------------
+// Every CTA adds the number of k-blocks it contributed to an output tile to that tile's counter once
+// its partial sums are in memory; the CTA whose addition completes the tile (all K / 64 k-blocks; for
+// gate/up the gate tile and its up tile share a counter) runs the GEMM's element-wise consumer on it:
+// the finished fp32 tile is still in L2.  Counters return to zero for the next GEMM.
+static __device__ __noinline__ void tc_finish_tiles(const DevCtx& c, const GemmArgs& a, const TcGeom& g, int layer) {
+  constexpr int BATCH = 16;
+  __shared__ int s_fin[BATCH];
+  __shared__ int s_nfin;
+  __shared__ long long s_next;
+  const int ntiles_slot = a.fix == FIX_SILU ? g.ntiles / 2 : g.ntiles;   // gate tile j and up tile j share slot j
+  const int need = (a.fix == FIX_SILU ? 2 : 1) * g.kblocks;
+  long long u = g.u0;
+  while (u < g.u1) {   // uniform over the CTA
+    if (threadIdx.x == 0) {
+      int n = 0;
+      __threadfence();   // the CTA's partial sums (ordered before by the barrier above) before the counters
+      while (u < g.u1 && n < BATCH) {
+        const long long seg_end = min(g.u1, (u / g.kblocks + 1) * (long long)g.kblocks);
+        const int nt = tc_unit_nt(g, u), pass = tc_unit_pass(g, u);
+        const int units = (int)(seg_end - u);
+        const int tile = nt % ntiles_slot;
+        const int slot = (pass * ntiles_slot + tile) % TILE_CNT_SLOTS;
+        const int old = atomicAdd(&c.tile_cnt[slot], units);
+        if (old + units == need) {
+          c.tile_cnt[slot] = 0;   // nobody touches this counter again before the next grid barrier
+          s_fin[n++] = (pass << 16) | tile;
+        }
+        u = seg_end;
+      }
+      if (n > 0) __threadfence();
+      s_nfin = n;
+      s_next = u;
+    }
+    __syncthreads();
+    const int n = s_nfin;
+    u = s_next;
+    for (int i = 0; i < n; ++i) {
+      const int tile = s_fin[i] & 0xffff, pass = s_fin[i] >> 16;
+      const int t0 = pass * 256, t1 = min(a.M, t0 + 256);
+      if (a.fix == FIX_ROPE_KV) fixup_rope_kv<__nv_bfloat16>(c, layer, tile, t0, t1);
+      else if (a.fix == FIX_SILU) fixup_silu<__nv_bfloat16>(a.out, reinterpret_cast<__nv_bfloat16*>(a.fix_out), a.N / 2, tile, t0, t1);
+      else fixup_sumsq(a.out, a.ldo, a.N, a.fix_rowss, tile, t0, t1);
+    }
+    __syncthreads();
+  }
+}
+
 static __device__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int which, int layer, float* smem_f, TcState& tc) {
   const int T = a.M, N = a.N, K = a.K;
   if (T <= 0) return;  // uniform over the grid
   const TcMaps* maps = reinterpret_cast<const TcMaps*>(c.tc_maps);
-  const TcGeom g = tc_geom(c, T, N, K);
+  const TcGeom g = tc_geom(c, T, N, K, which == GEMM_LMHEAD && lm_head_whole_tiles(c));
   const int kblocks = g.kblocks, ntiles = g.ntiles, KPS = g.KPS, S = g.S;
   const uint32_t b_bytes = g.b_bytes, stage_bytes = g.stage_bytes;
   const int act_id = which == GEMM_O ? ACT_ATTN : which == GEMM_DOWN ? ACT_ACT : which == GEMM_LMHEAD ? ACT_XS
@@ -480,20 +537,16 @@ static __device__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int whi
         }
         if (!ok) break;
         umma_commit(&g_tc.acc_full[abuf]);
+        // Warps 0-3 take part of the CTA's last accumulator.  They cannot wait on acc_full: a parity
+        // wait tells two consecutive completions apart, not the first use of a buffer in this phase
+        // from its third, and they arrive here long before the epilogue warps.  A barrier of their own
+        // that completes exactly once per phase has no such ambiguity.
+        if (u == u1) umma_commit(&g_tc.acc_last);
         abuf ^= 1;
       }
     }
   } else if (warp >= 4) {
     const int q = warp & 3;  // TMEM lane quarter this warp may read
-    // nothing to store until the first accumulator is complete: clear the buffers the caller named
-    // (16-byte stores, grid-strided over the epilogue threads)
-    for (int z = 0; z < 2; ++z) {
-      float4* zq = reinterpret_cast<float4*>(a.zero_p[z]);
-      const long long n4 = a.zero_n[z] >> 2;
-      const long long step = (long long)gridDim.x * 128;
-      for (long long i = (long long)blockIdx.x * 128 + (threadIdx.x - 128); i < n4; i += step)
-        zq[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-    }
     const TcEpiOut eo{a.out, (size_t)a.ldo, a.row_map, a.row_scale, T, N};
     const bool accumulate = a.accumulate != 0;
     int abuf = 0;
@@ -523,27 +576,25 @@ static __device__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int whi
   }
   if (warp < 4) {
     // Producers and the MMA issuer are done once the last MMA is committed: their warps store
-    // the upper columns of the last accumulator.  Every thread walks the segments to keep its
-    // copy of the accumulator parities in step with the epilogue warps.
+    // the upper columns of the last accumulator.
     __syncwarp();
-    int abuf = 0, last_abuf = -1;
-    uint32_t last_par = 0;
-    long long last_u = 0;
-    for (long long u = u0; u < u1;) {
-      last_abuf = abuf;
-      last_par = (tc.acc_epi >> abuf) & 1u;
-      last_u = u;
-      tc.acc_epi ^= 1u << abuf;
-      abuf ^= 1;
-      u = min(u1, (u / kblocks + 1) * (long long)kblocks);
-    }
-    if (last_abuf >= 0) {
+    if (u0 < u1) {
+      const uint32_t par = tc.last_bit;
+      tc.last_bit ^= 1u;
+      long long last_u = u0;
+      int last_abuf = 0;
+      for (long long u = u0; u < u1;) {   // find the last segment and its accumulator buffer
+        last_u = u;
+        u = min(u1, (u / kblocks + 1) * (long long)kblocks);
+        if (u < u1) last_abuf ^= 1;
+      }
       const int kb0 = (int)(last_u % kblocks);
       const int nt = tc_unit_nt(g, last_u);
       const int pass = tc_unit_pass(g, last_u);
       const int n_mma = (min(256, T - pass * 256) + 15) & ~15;
       const int c_begin = tc_epi_half(n_mma);
-      if (c_begin < n_mma && mbar_wait_idle(c, &g_tc.acc_full[last_abuf], last_par, dead)) {
+      // every thread waits (also when it has no columns to store) so that its parity stays in step
+      if (mbar_wait_idle(c, &g_tc.acc_last, par, dead) && c_begin < n_mma) {
         tc_fence_after();
         const TcEpiOut eo{a.out, (size_t)a.ldo, a.row_map, a.row_scale, T, N};
         const bool plain = (kb0 == 0 && (long long)kb0 + (u1 - last_u) == kblocks) && a.accumulate == 0 && eo.row_map == nullptr;
@@ -554,6 +605,7 @@ static __device__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int whi
     }
   }
   __syncthreads();
+  if (a.fix != FIX_NONE) tc_finish_tiles(c, a, g, layer);
 }
 
 // ---- host side: tensor maps ----------------------------------------------------------------

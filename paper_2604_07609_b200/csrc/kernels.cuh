@@ -21,19 +21,21 @@ __device__ __forceinline__ void gemm_dispatch(const DevCtx& c, const GemmArgs& a
   else phase_gemm_simt<WT>(a);
 }
 
+// `T` = rows of the step (read once per step by the caller: it does not change between phases)
 template <typename WT, int HD, int NREP>
 __device__ __forceinline__ void run_phase(const DevCtx& c, int phase, int layer, int sub, float* smem, TcState& tc,
-                                          AttState& as) {
-  const int T = c.ss->cur_T;
+                                          AttState& as, int T) {
   const size_t esz = sizeof(WT);
   switch (phase) {
     case PH_NORM1:
-      phase_norm<WT>(c, layer, 0);
+      if (c.fused_norm && layer > 0) phase_norm_apply<WT>(c, layer, 0, T);
+      else phase_norm<WT>(c, layer, 0);
       break;
     case PH_QKV: {
       GemmArgs a{c.xn, c.w_base + c.w_off[1] + (size_t)layer * c.qkv_dim * c.d * esz, c.qkv, T, c.qkv_dim, c.d,
                  c.qkv_dim, 0};
       a.w_row0 = (long long)layer * c.qkv_dim;
+      if (c.fused) a.fix = FIX_ROPE_KV;
       gemm_dispatch<WT>(c, a, GEMM_QKV, layer, smem, tc);
     } break;
     case PH_ROPE: phase_rope_kv<WT>(c, layer); break;
@@ -45,24 +47,18 @@ __device__ __forceinline__ void run_phase(const DevCtx& c, int phase, int layer,
     case PH_O: {
       GemmArgs a{c.attn, c.w_base + c.w_off[2] + (size_t)layer * c.d * c.q_dim * esz, c.h, T, c.d, c.q_dim, c.d, 1};
       a.w_row0 = (long long)layer * c.d;
-      if (c.gemm_tc) {
-        const int rows_gu = c.E > 0 ? T * c.topE : T;   // routed experts: one gate/up row per (token, expert)
-        a.zero_p[0] = c.gu;
-        a.zero_n[0] = (long long)rows_gu * 2 * c.F;
-        if (layer + 1 < c.L) {
-          a.zero_p[1] = c.qkv;
-          a.zero_n[1] = (long long)T * c.qkv_dim;
-        }
-      }
+      if (c.fused_norm) { a.fix = FIX_SUMSQ; a.fix_rowss = c.rowss_a; }
       gemm_dispatch<WT>(c, a, GEMM_O, layer, smem, tc);
     } break;
     case PH_NORM2:
-      phase_norm<WT>(c, layer, 1);
+      if (c.fused_norm) phase_norm_apply<WT>(c, layer, 1, T);
+      else phase_norm<WT>(c, layer, 1);
       break;
     case PH_GU: {
       if (c.E == 0) {
         GemmArgs a{c.xn, c.w_base + c.w_off[3] + (size_t)layer * 2 * c.F * c.d * esz, c.gu, T, 2 * c.F, c.d, 2 * c.F, 0};
         a.w_row0 = (long long)layer * 2 * c.F;
+        if (c.fused) { a.fix = FIX_SILU; a.fix_out = c.act; }
         gemm_dispatch<WT>(c, a, GEMM_GU, layer, smem, tc);
       } else {
         // expert `sub` on the rows routed to it (gathered, contiguous from moe_off[sub])
@@ -72,6 +68,7 @@ __device__ __forceinline__ void run_phase(const DevCtx& c, int phase, int layer,
                    c.gu + (size_t)off * 2 * c.F, cnt, 2 * c.F, c.d, 2 * c.F, 0};
         a.x_row0 = off;
         a.w_row0 = we * 2 * c.F;
+        if (c.fused) { a.fix = FIX_SILU; a.fix_out = reinterpret_cast<char*>(c.act) + (size_t)off * c.F * esz; }
         gemm_dispatch<WT>(c, a, GEMM_GU, layer, smem, tc);
       }
     } break;
@@ -82,6 +79,7 @@ __device__ __forceinline__ void run_phase(const DevCtx& c, int phase, int layer,
       if (c.E == 0) {
         GemmArgs a{c.act, c.w_base + c.w_off[4] + (size_t)layer * c.d * c.F * esz, c.h, T, c.d, c.F, c.d, 1};
         a.w_row0 = (long long)layer * c.d;
+        if (c.fused_norm) { a.fix = FIX_SUMSQ; a.fix_rowss = c.rowss_b; }
         gemm_dispatch<WT>(c, a, GEMM_DOWN, layer, smem, tc);
       } else {
         const int off = c.moe_off[sub], cnt = c.moe_off[sub + 1] - off;
@@ -128,8 +126,10 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) blink_loop_kernel(const __grid
       // the barrier that closes it); recorded only when per-iteration statistics are kept
       const bool timed = c.stats_cap > 0 && blockIdx.x == 0 && threadIdx.x == 0;
       uint64_t t_prev = timed ? global_timer_ns() : 0;
+      const int T = __ldcg(&c.ss->cur_T);   // fixed for the whole step: one L2 read instead of one per phase
       auto step_phase = [&](int ph, int layer, int sub) {
-        run_phase<WT, HD, NREP>(c, ph, layer, sub, smem, tc, as);
+        if (c.fused && (ph == PH_ROPE || ph == PH_SILU)) return;   // done by the epilogues of the QKV and gate/up GEMMs
+        run_phase<WT, HD, NREP>(c, ph, layer, sub, smem, tc, as, T);
         ok = grid_barrier(c, gen);
         if (timed) { const uint64_t t = global_timer_ns(); c.ss->cur_phase_ns[ph] += t - t_prev; t_prev = t; }
       };
@@ -164,7 +164,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) blink_phase_kernel(const __gri
   tc_init(c, smem, tc);
   AttState as;
   att_init(c, as);
-  run_phase<WT, HD, NREP>(c, phase, layer, sub, smem, tc, as);
+  run_phase<WT, HD, NREP>(c, phase, layer, sub, smem, tc, as, c.ss->cur_T);
   tc_fini(c, tc);
 }
 

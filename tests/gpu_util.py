@@ -112,34 +112,41 @@ def acceptable_tokens(row, req, gen_index, tol):
     T = float(req.temperature)
     n = len(row)
     k = n if req.top_k <= 0 else min(req.top_k, n)
-    idx, z = S.top_k_candidates(row, min(n, k + 1), T)
-    ok, in_margin = {want}, False
-    if k < n and float(z[k - 1]) - float(z[k]) < 2 * tol / T:       # the k-th and (k+1)-th candidates may swap
-        in_margin = True
-        ok.update(int(i) for i in idx[max(0, k - 2):k + 1])
-    idx, z = idx[:k], z[:k].astype(np.float64)
-    w = np.exp(z - z[0])
-    if nucleus_on:
-        nidx, _ = S.nucleus(row, req.top_k, T, top_p)
-        m = len(nidx)
-        cfrac = np.cumsum(w) / w.sum()
-        d = 4 * tol / T + 1e-7
-        if m < k and abs(cfrac[m - 1] - top_p) < d or (m >= 2 and abs(cfrac[m - 2] - top_p) < d):
-            in_margin = True                                           # the nucleus may gain or lose its last token
-            ok.update(int(i) for i in idx[:min(k, m + 1)])
-            return ok, in_margin
-        w, idx = w[:m], idx[:m]
-    cfrac = np.cumsum(w) / w.sum()
+    z_all = (row / np.float32(T)).astype(np.float32)
+    idx, z = S.top_k_candidates(row, k, T)
+    zs = z.astype(np.float64)
+    tail_pool, p0, d_set = None, k, 0.0
+    if k < n:
+        # candidate set: a token whose z is within the margin of the k-th largest may be a member of the
+        # other side's top k.  Then the positions from the first oracle member that may drop out (p0) to
+        # the end may hold any of those members or of the outsiders that may come in, and the total mass
+        # is uncertain by the mass of those positions.
+        wide = np.flatnonzero(z_all >= z[k - 1] - 2 * tol / T)
+        if len(wide) > k:
+            p0 = int(np.argmax(zs < zs[k - 1] + 2 * tol / T))
+            tail_pool = set(int(i) for i in wide if z_all[i] < zs[k - 1] + 2 * tol / T)
+    w = np.exp(zs - zs[0])
+    idx_all, zs_all = idx, zs
+    d = float(np.expm1(2 * tol / T)) + 1e-7      # how far a tol-perturbation can move a normalised cumulative sum
+    if tail_pool is not None:
+        d += float(w[p0:].sum() / w.sum())
+    cf = np.cumsum(w) / w.sum()
+    prev = np.concatenate([[0.0], cf[:-1]])
+    m_lo = m_hi = len(cf)
+    if nucleus_on:   # the nucleus ends at the first prefix reaching top_p; the other side's may end a little earlier or later
+        m_lo = min(len(cf), int(np.argmax(cf >= top_p - d)) + 1) if (cf >= top_p - d).any() else len(cf)
+        m_hi = min(len(cf), int(np.argmax(cf >= top_p + d)) + 1) if (cf >= top_p + d).any() else len(cf)
     u = (S.philox_word(req.ticket, gen_index, req.seed) >> 8) / 2.0 ** 24
-    j = int(np.flatnonzero(idx == want)[0])
-    d = 4 * tol / T + 1e-7
-    if j > 0 and u - cfrac[j - 1] < d:
-        in_margin = True
-        ok.add(int(idx[j - 1]))
-    if j + 1 < len(idx) and cfrac[j] - u < d:
-        in_margin = True
-        ok.add(int(idx[j + 1]))
-    return ok, in_margin
+    # the draw lands at u * (mass of the nucleus); masses and boundaries each move by at most d
+    t_lo, t_hi = u * (cf[m_lo - 1] - d), u * (cf[m_hi - 1] + d)
+    pos = np.arange(len(cf))
+    hit = np.flatnonzero((pos < m_hi) & (prev - d <= t_hi) & (cf + d >= t_lo))
+    ok = {want}
+    for j in hit:   # the candidate at an admissible position, and whatever may trade places with it in the order
+        if j >= p0:
+            ok.update(tail_pool)
+        ok.update(int(i) for i in idx_all[np.abs(zs_all - zs_all[j]) < 2 * tol / T + 1e-7])
+    return ok, len(ok) > 1
 
 
 def assert_tokens_within_margin(ora, reqs, toks_gpu, tol):
@@ -158,25 +165,57 @@ def assert_tokens_within_margin(ora, reqs, toks_gpu, tol):
     return n_margin
 
 
-def compare_with_oracle(model, sched, reqs, weights_cpu, tol, *, oracle_dtype=np.float64, plain_too=True, **kw):
+def compare_with_oracle(model, sched, reqs, weights_cpu, tol, *, oracle_dtype=np.float64, plain_too=True,
+                        noise_relative=False, **kw):
     """The whole check of one configuration: the oracle in the data path's rounding mode runs free
     (its own tokens fed back); the GPU is teacher-forced with those tokens; traces must be equal word
-    for word (sampled tokens apart), logits within `tol`, tokens by the margin rule.  For the bf16 data
-    path the plain high-precision oracle (no rounding hook) is run on the same forced tokens as well
-    and the error against it reported."""
+    for word (sampled tokens apart), logits within the tolerance, tokens by the margin rule.  For the
+    bf16 data path the plain high-precision oracle (no rounding hook) runs on the same forced tokens.
+
+    Tolerance.  `tol` is the absolute max-abs bound (2e-2 for bf16, 1e-4 for the fp32 mode).  With
+    `noise_relative` (the large layer shapes) the bound is taken from the arithmetic instead: two
+    evaluations that are both correct and differ only in where values are rounded to 16 bits (the two
+    oracles) differ by max-abs N_max and rms N_rms on these very inputs; an implementation cannot be
+    asked to be closer to either of them than they are to each other.  Then the GPU must satisfy
+      max|gpu - rounding oracle| <= max(tol, 1.5 N_max), rms(gpu - rounding oracle) <= N_rms,
+      max|gpu - plain oracle|    <= max(tol, 1.5 N_max), rms(gpu - plain oracle)  <= 1.25 N_rms
+    (the rms bounds are the sharp ones: a maximum over 10^7 to 10^8 entries fluctuates by tens of per
+    cent from one realisation of the rounding to the next), and the token rule uses the max bound as
+    the logit tolerance."""
     matched_round = O2.round_bf16 if model.dtype == "bf16" else None
     W = O2.Weights(model, weights_as_numpy(model, weights_cpu), dtype=oracle_dtype)
     ora = OS.run(model, sched, W, reqs, act_round=matched_round)
     trace, toks, logits, its = gpu_run_forced(model, sched, reqs, weights_cpu, ora["tokens"], **kw)
     assert_traces_equal([{**r, "sampled": []} for r in trace], [{**r, "sampled": []} for r in ora["trace"]])
-    lo = np.stack([row for (_, _, _, _, row) in ora["logits"]])
+    lo = np.stack([np.asarray(row, dtype=np.float32) for (_, _, _, _, row) in ora["logits"]])
     assert logits.shape == lo.shape
-    err = float(np.abs(logits.astype(np.float64) - lo).max())
-    assert err <= tol, f"max-abs logit error {err:.3e} against the oracle exceeds {tol}"
-    n_margin = assert_tokens_within_margin(ora, reqs, toks, tol)
-    err_plain = err
-    if plain_too and matched_round is not None:
+    lg = logits
+
+    def dist(a, b):   # (max-abs, rms) of a - b, row by row to bound temporary memory
+        mx, ss = 0.0, 0.0
+        for i in range(a.shape[0]):
+            dd = a[i].astype(np.float64) - b[i]
+            mx = max(mx, float(np.abs(dd).max()))
+            ss += float(np.dot(dd, dd))
+        return mx, float(np.sqrt(ss / a.size))
+
+    err, err_rms = dist(lg, lo)
+    out = dict(err=err, err_rms=err_rms, err_plain=err, err_plain_rms=err_rms, noise_max=0.0, noise_rms=0.0,
+               logit_std=float(lo[: min(64, lo.shape[0])].std()), trace=trace, toks=toks, ora=ora, its=its, logits=logits)
+    tol_eff = tol
+    if matched_round is not None and (plain_too or noise_relative):
         plain = OS.run(model, sched, W, reqs, act_round=None, forced=ora["tokens"])
-        lp = np.stack([row for (_, _, _, _, row) in plain["logits"]])
-        err_plain = float(np.abs(logits.astype(np.float64) - lp).max())
-    return dict(err=err, err_plain=err_plain, n_margin=n_margin, trace=trace, toks=toks, ora=ora, its=its, logits=logits)
+        lp = np.stack([np.asarray(row, dtype=np.float32) for (_, _, _, _, row) in plain["logits"]])
+        (ep, ep_rms), (nm, n_rms) = dist(lg, lp), dist(lo, lp)
+        out.update(err_plain=ep, err_plain_rms=ep_rms, noise_max=nm, noise_rms=n_rms)
+        if noise_relative:
+            tol_eff = max(tol, 1.5 * out["noise_max"])
+            msg = (f"gpu vs rounding oracle max {err:.3e} rms {err_rms:.3e}; gpu vs plain oracle max {out['err_plain']:.3e} "
+                   f"rms {out['err_plain_rms']:.3e}; rounding oracle vs plain oracle max {out['noise_max']:.3e} rms {out['noise_rms']:.3e}")
+            assert err_rms <= out["noise_rms"], msg
+            assert out["err_plain"] <= max(tol, 1.5 * out["noise_max"]), msg
+            assert out["err_plain_rms"] <= 1.25 * out["noise_rms"], msg
+    out["tol"] = tol_eff
+    assert err <= tol_eff, f"max-abs logit error {err:.3e} against the oracle exceeds {tol_eff:.3e}"
+    out["n_margin"] = assert_tokens_within_margin(ora, reqs, toks, tol_eff)
+    return out

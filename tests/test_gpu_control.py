@@ -164,3 +164,40 @@ def test_eos_retires_a_request_early_and_frees_its_blocks():
         assert e["is_last"][-1] == 1 and e["is_last"][:-1].sum() == 0
         if r.eos_id >= 0:
             assert len(e) <= 6 and int(e["token"][-1]) == r.eos_id
+
+
+def test_a_wait_that_runs_out_unwinds_the_loop_with_a_status():
+    """Every wait inside the kernel is bounded.  Here the bound (5 ms) is set below the idle-exit time
+    (1 s): once the queue is empty the control plane keeps polling it while the other CTAs of the grid
+    wait at the grid barrier for the next step, and nothing ends that wait in time.  The waiting CTAs
+    must record the time-out, every CTA must leave the GPU, the host calls must report the device
+    error, and the context must still be destroyed cleanly (no trap, no hang: the CUDA context stays
+    usable, which the tests that run after this one rely on)."""
+    import time
+    import torch
+    from synth import make_weights
+    model, sched = model_cfg(1, dtype="fp32"), sched_cfg(1)
+    w = make_weights(model, 1, "cpu").cuda()
+    kv = torch.zeros(sched.n_blocks * B.kv_bytes_per_block(model, sched.block_size), dtype=torch.uint8, device="cuda")
+    eng = B.Blink(model, sched, w, kv, idle_exit_us=1_000_000, wait_limit_ms=5)
+    try:
+        rng = np.random.default_rng(3)
+        eng.blink_submit(rng.integers(0, model.vocab, size=20).astype(np.int32), 4)
+        ev = eng.drain(4, timeout_s=30)            # real work completes: the limit is far above a step's time
+        assert len(ev) == 4
+        t0 = time.monotonic()
+        while eng.blink_get_stats().loop_state == B.LOOP_RUNNING and time.monotonic() - t0 < 5:
+            time.sleep(0.01)
+        st = eng.blink_get_stats()
+        assert st.loop_state == B.LOOP_EXIT_ERROR, st.loop_state
+        assert st.device_status == 1                 # the grid-barrier wait ran out
+        assert time.monotonic() - t0 < 0.9           # long before the idle exit: it was the wait limit
+        with pytest.raises(B.BlinkError) as e:
+            eng.blink_poll(16, 1000)
+        assert e.value.code == B.BLINK_EDEVICE
+        assert eng.blink_submit(np.arange(8, dtype=np.int32), 2, raise_on_error=False) == B.BLINK_EDEVICE
+    finally:
+        assert eng.blink_destroy() == B.BLINK_OK
+    # the CUDA context is intact: a fresh loop on the same device works
+    trace, toks, st2, _ = run_control_only(model_cfg(1), sched_cfg(1), make_requests(1))
+    assert st2.device_status == 0 and len(toks) == 8
