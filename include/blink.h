@@ -80,6 +80,13 @@ enum {
   BLINK_GEMM_TC = 2    /* tcgen05 / TMEM / TMA kernels (bf16 only)   */
 };
 
+/* where RoPE + KV write, SwiGLU and the norms' sums of squares run (tensor-core path only) */
+enum {
+  BLINK_FUSION_AUTO = 0, /* the faster of the two for the model shape (currently: separate phases)        */
+  BLINK_FUSION_OFF = 1,  /* phases of their own between grid barriers                                     */
+  BLINK_FUSION_ON = 2    /* in the GEMM epilogues: the CTA that completes an output tile consumes it      */
+};
+
 /* why the device loop is not running (blink_stats.loop_state) */
 enum {
   BLINK_LOOP_NOT_STARTED = 0,
@@ -130,6 +137,8 @@ typedef struct blink_sched_cfg {
   float* logits_capture;        /* DEVICE, caller-owned [logits_capture_rows][vocab] or NULL: row r
                                    receives the logits of the r-th sampled row since create      */
   int64_t logits_capture_rows;
+  int32_t epilogue_fusion;      /* BLINK_FUSION_*                                               */
+  int32_t reserved0;
 } blink_sched_cfg;
 
 /* Caller-owned DEVICE memory for the paged KV cache.  The library derives
@@ -154,6 +163,12 @@ typedef struct blink_request {
   const int32_t* forced_tokens; /* HOST or NULL.  Teacher forcing for tests: max_new_tokens ids
                                    that are fed back instead of the sampled ones; the sampled ones
                                    are still the ones reported.                                 */
+  float top_p;                  /* nucleus sampling (Section 4.2: Top-P with temperature): in (0, 1) the
+                                   draw is restricted to the smallest set of most likely tokens whose
+                                   probability reaches top_p (taken among the top_k largest when top_k > 0,
+                                   else over the whole vocabulary); 0 or >= 1 = no cut.  Needs
+                                   temperature > 0                                              */
+  int32_t reserved0;
 } blink_request;
 
 typedef struct blink_token_event {
@@ -293,6 +308,16 @@ int blink_get_iter_stats(blink_ctx* ctx, blink_iter_stat* out, int64_t capacity,
  * and frees a small device scratch. */
 int blink_sample(const float* logits, int rows, int vocab, const int32_t* top_k, const float* temperature,
                  const uint64_t* ticket, const int32_t* gen_index, const uint64_t* seed, int32_t* out);
+
+/* blink_sample with the nucleus cut of Section 4.2 ("Top-P with temperature"): `top_p` is a HOST array of
+ * length rows; row r is sampled as the loop samples a request with top_k[r], temperature[r] and
+ * top_p[r] (see blink_request.top_p).  Arithmetic, so that results do not depend on the order of a
+ * parallel sum: integer weights floor(exp(z - z_max) * 2^40), the nucleus is the shortest prefix of the
+ * order (z desc, index asc) whose weight times 2^24 reaches round(top_p * 2^24) times the total weight,
+ * and the 24-bit uniform draw is scaled to the nucleus' weight. */
+int blink_sample_top_p(const float* logits, int rows, int vocab, const int32_t* top_k, const float* temperature,
+                       const float* top_p, const uint64_t* ticket, const int32_t* gen_index, const uint64_t* seed,
+                       int32_t* out);
 
 /* blink_sample for callers that cannot allocate.  The paper has no counterpart: this is a
  * convenience of this library.  Some callers must not call cudaMalloc / cudaFree once they

@@ -22,6 +22,7 @@ DTYPE_BF16, DTYPE_FP32 = 0, 1
 EXEC_PERSISTENT, EXEC_STEPPED, EXEC_MANUAL = 0, 1, 2
 GEMM_AUTO, GEMM_SIMT, GEMM_TC = 0, 1, 2
 WEIGHTS_ROW_MAJOR, WEIGHTS_STREAMING = 0, 1
+FUSION_AUTO, FUSION_OFF, FUSION_ON = 0, 1, 2
 LOOP_NOT_STARTED, LOOP_RUNNING, LOOP_EXIT_STOP, LOOP_EXIT_BUDGET, LOOP_EXIT_IDLE, LOOP_EXIT_ERROR = range(6)
 TRACE_MAGIC = 0x424C4B31
 TRACE_HDR_WORDS = 12
@@ -41,7 +42,8 @@ class blink_sched_cfg(C.Structure):
                 ("gemm_impl", C.c_int32), ("control_only", C.c_int32), ("start_paused", C.c_int32),
                 ("wait_limit_ms", C.c_int32), ("iteration_budget", C.c_int64), ("idle_exit_us", C.c_int64),
                 ("trace_capacity_words", C.c_int64), ("stats_capacity_iters", C.c_int64),
-                ("logits_capture", C.c_void_p), ("logits_capture_rows", C.c_int64)]
+                ("logits_capture", C.c_void_p), ("logits_capture_rows", C.c_int64), ("epilogue_fusion", C.c_int32),
+                ("reserved0", C.c_int32)]
 
 
 class blink_kv_pool(C.Structure):
@@ -52,7 +54,7 @@ class blink_request(C.Structure):
     _fields_ = [("size", C.c_uint32), ("n_prompt", C.c_int32), ("prompt", C.POINTER(C.c_int32)),
                 ("max_new_tokens", C.c_int32), ("top_k", C.c_int32), ("temperature", C.c_float),
                 ("eos_id", C.c_int32), ("seed", C.c_uint64), ("user_tag", C.c_uint64),
-                ("forced_tokens", C.POINTER(C.c_int32))]
+                ("forced_tokens", C.POINTER(C.c_int32)), ("top_p", C.c_float), ("reserved0", C.c_int32)]
 
 
 class blink_token_event(C.Structure):
@@ -89,7 +91,8 @@ EVENT_DTYPE = np.dtype([("ticket", "<u8"), ("user_tag", "<u8"), ("index", "<i4")
 
 EXPORTS = ["blink_weights_bytes", "blink_weight_offset", "blink_convert_weights", "blink_kv_blocks_for_bytes", "blink_create",
            "blink_start", "blink_submit", "blink_poll", "blink_step", "blink_run", "blink_stop", "blink_destroy",
-           "blink_get_stats", "blink_get_trace", "blink_get_iter_stats", "blink_sample", "blink_sample_noalloc",
+           "blink_get_stats", "blink_get_trace", "blink_get_iter_stats", "blink_sample", "blink_sample_top_p",
+           "blink_sample_noalloc",
            "blink_strerror"]
 
 _lib = None
@@ -137,6 +140,8 @@ def lib():
     L.blink_get_iter_stats.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, P(C.c_int64)]
     L.blink_sample.restype = C.c_int
     L.blink_sample.argtypes = [C.c_void_p, C.c_int, C.c_int] + [C.c_void_p] * 6
+    L.blink_sample_top_p.restype = C.c_int
+    L.blink_sample_top_p.argtypes = [C.c_void_p, C.c_int, C.c_int] + [C.c_void_p] * 7
     L.blink_sample_noalloc.restype = C.c_int
     L.blink_sample_noalloc.argtypes = [C.c_void_p, C.c_int, C.c_int] + [C.c_void_p] * 6
     L.blink_strerror.restype = C.c_char_p
@@ -194,6 +199,21 @@ def blink_sample(logits, top_k, temperature, ticket, gen_index, seed) -> np.ndar
                             gi.ctypes.data, sd.ctypes.data, out.ctypes.data)
     if rc != BLINK_OK:
         raise BlinkError(rc, "blink_sample")
+    return out
+
+
+def blink_sample_top_p(logits, top_k, temperature, top_p, ticket, gen_index, seed) -> np.ndarray:
+    """blink_sample with a per-row nucleus cut (top_p in (0, 1); 0 or >= 1 = off)."""
+    rows, vocab = logits.shape
+    assert logits.is_cuda and logits.is_contiguous() and logits.dtype.is_floating_point and logits.element_size() == 4
+    a = lambda v, dt: np.ascontiguousarray(v, dtype=dt)
+    tk, tp, pp, ti, gi, sd = a(top_k, np.int32), a(temperature, np.float32), a(top_p, np.float32), a(ticket, np.uint64), \
+        a(gen_index, np.int32), a(seed, np.uint64)
+    out = np.zeros(rows, dtype=np.int32)
+    rc = lib().blink_sample_top_p(logits.data_ptr(), rows, vocab, tk.ctypes.data, tp.ctypes.data, pp.ctypes.data,
+                                  ti.ctypes.data, gi.ctypes.data, sd.ctypes.data, out.ctypes.data)
+    if rc != BLINK_OK:
+        raise BlinkError(rc, "blink_sample_top_p")
     return out
 
 
@@ -275,7 +295,8 @@ class Blink:
 
     def __init__(self, model, sched, weights=None, kv_pool=None, *, exec_mode=EXEC_PERSISTENT, gemm_impl=GEMM_AUTO,
                  control_only=False, start_paused=False, iteration_budget=0, idle_exit_us=0, trace_words=0,
-                 stats_iters=0, logits_capture=None, kv_bytes=None, weights_layout=WEIGHTS_ROW_MAJOR, wait_limit_ms=0):
+                 stats_iters=0, logits_capture=None, kv_bytes=None, weights_layout=WEIGHTS_ROW_MAJOR, wait_limit_ms=0,
+                 epilogue_fusion=FUSION_AUTO):
         L = lib()
         self.model, self.sched = model, sched
         self._keep = (weights, kv_pool, logits_capture)
@@ -287,7 +308,7 @@ class Blink:
         sc = blink_sched_cfg(C.sizeof(blink_sched_cfg), sched.max_batch, sched.prefill_chunk_tokens, sched.n_slots,
                              sched.max_prompt, sched.max_new, exec_mode, gemm_impl, int(control_only),
                              int(start_paused), wait_limit_ms, iteration_budget, idle_exit_us, trace_words, stats_iters,
-                             cap_ptr, cap_rows)
+                             cap_ptr, cap_rows, epilogue_fusion, 0)
         if kv_pool is not None:
             kv = blink_kv_pool(C.sizeof(blink_kv_pool), sched.block_size, kv_pool.data_ptr(),
                                kv_pool.numel() * kv_pool.element_size())
@@ -308,12 +329,12 @@ class Blink:
             raise BlinkError(rc, "blink_start")
 
     def blink_submit(self, prompt, max_new_tokens, top_k=0, temperature=1.0, eos_id=-1, seed=0, user_tag=0,
-                     forced_tokens=None, raise_on_error=True):
+                     forced_tokens=None, raise_on_error=True, top_p=0.0):
         p = np.ascontiguousarray(prompt, dtype=np.int32)
         f = None if forced_tokens is None else np.ascontiguousarray(forced_tokens, dtype=np.int32)
         r = blink_request(C.sizeof(blink_request), p.shape[0], p.ctypes.data_as(C.POINTER(C.c_int32)),
                           max_new_tokens, top_k, temperature, eos_id, seed, user_tag,
-                          f.ctypes.data_as(C.POINTER(C.c_int32)) if f is not None else None)
+                          f.ctypes.data_as(C.POINTER(C.c_int32)) if f is not None else None, top_p, 0)
         t = C.c_uint64()
         rc = lib().blink_submit(self._h, C.byref(r), C.byref(t))
         if rc != BLINK_OK:
@@ -387,7 +408,7 @@ class Blink:
     # -- conveniences built only from the calls above ---------------------------------------
     def submit_request(self, r, forced_tokens=None, **kw):
         return self.blink_submit(r.prompt, r.max_new, r.top_k, r.temperature, r.eos_id, r.seed, r.user_tag,
-                                 forced_tokens, **kw)
+                                 forced_tokens, top_p=getattr(r, "top_p", 0.0), **kw)
 
     def drain(self, n_tokens_expected: int, timeout_s: float = 60.0, step_iters: int = 0):
         """Poll (persistent mode) or step+poll (stepped mode, step_iters per round) until

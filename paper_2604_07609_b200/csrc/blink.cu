@@ -42,11 +42,12 @@ __global__ void __launch_bounds__(CTRL_THREADS, 1) blink_control_kernel(const __
 // Sampler alone over caller-provided logits (one CTA per row).
 __global__ void __launch_bounds__(FWD_THREADS, 1)
 blink_sample_kernel(const float* logits, int rows, int V, const int* top_k, const float* temp,
-                    const unsigned long long* ticket, const int* gen_index, const unsigned long long* seed, int* out) {
+                    const unsigned long long* ticket, const int* gen_index, const unsigned long long* seed, int* out,
+                    const float* top_p) {
   extern __shared__ __align__(1024) float smem[];
   for (int r = blockIdx.x; r < rows; r += gridDim.x) {
-    const int tok = sample_row(logits + (size_t)r * V, V, min(top_k[r], MAX_TOPK), temp[r], ticket[r], gen_index[r],
-                               seed[r], smem);
+    const int tok = sample_row(logits + (size_t)r * V, V, min(top_k[r], MAX_TOPK), temp[r], top_p ? top_p[r] : 0.f, ticket[r],
+                               gen_index[r], seed[r], smem);
     if (threadIdx.x == 0) out[r] = tok;
   }
 }
@@ -352,15 +353,19 @@ int64_t blink_kv_blocks_for_bytes(const blink_model_cfg* cfg, int block_size, ui
   return (int64_t)(bytes / per);
 }
 
-int blink_sample(const float* logits, int rows, int vocab, const int32_t* top_k, const float* temperature,
-                 const uint64_t* ticket, const int32_t* gen_index, const uint64_t* seed, int32_t* out) {
+static int sample_impl(const float* logits, int rows, int vocab, const int32_t* top_k, const float* temperature,
+                       const float* top_p, const uint64_t* ticket, const int32_t* gen_index, const uint64_t* seed,
+                       int32_t* out) {
   if (!logits || rows < 1 || vocab < 2 || !top_k || !temperature || !ticket || !gen_index || !seed || !out)
     return BLINK_EINVAL;
-  for (int r = 0; r < rows; ++r)
-    if (top_k[r] < 0 || top_k[r] > MAX_TOPK || (top_k[r] > 0 && !(temperature[r] > 0.f))) return BLINK_EINVAL;
+  for (int r = 0; r < rows; ++r) {
+    const bool nucleus = top_p && top_p[r] > 0.f && top_p[r] < 1.f;
+    if (top_k[r] < 0 || top_k[r] > MAX_TOPK || ((top_k[r] > 0 || nucleus) && !(temperature[r] > 0.f))) return BLINK_EINVAL;
+    if (top_p && !(top_p[r] >= 0.f)) return BLINK_EINVAL;
+  }
   char* d = nullptr;
   const size_t n = (size_t)rows;
-  const size_t bytes = n * (4 + 4 + 8 + 4 + 8 + 4);
+  const size_t bytes = n * (4 + 4 + 8 + 4 + 8 + 4 + 4);
   if (cudaMalloc(&d, bytes) != cudaSuccess) return BLINK_ENOMEM;
   unsigned long long* d_ticket = (unsigned long long*)d;
   unsigned long long* d_seed = d_ticket + n;
@@ -368,7 +373,9 @@ int blink_sample(const float* logits, int rows, int vocab, const int32_t* top_k,
   float* d_temp = (float*)(d_topk + n);
   int* d_gen = (int*)(d_temp + n);
   int* d_out = d_gen + n;
+  float* d_topp = (float*)(d_out + n);
   int rc = BLINK_OK;
+  if (top_p && cudaMemcpy(d_topp, top_p, n * 4, cudaMemcpyHostToDevice) != cudaSuccess) rc = BLINK_ECUDA;
   if (cudaMemcpy(d_ticket, ticket, n * 8, cudaMemcpyHostToDevice) != cudaSuccess ||
       cudaMemcpy(d_seed, seed, n * 8, cudaMemcpyHostToDevice) != cudaSuccess ||
       cudaMemcpy(d_topk, top_k, n * 4, cudaMemcpyHostToDevice) != cudaSuccess ||
@@ -378,12 +385,24 @@ int blink_sample(const float* logits, int rows, int vocab, const int32_t* top_k,
   if (rc == BLINK_OK) {
     const int grid = rows < 1184 ? rows : 1184;
     blink_sample_kernel<<<grid, FWD_THREADS, SAMPLE_SMEM_FLOATS * sizeof(float)>>>(
-        logits, rows, vocab, d_topk, d_temp, d_ticket, d_gen, d_seed, d_out);
+        logits, rows, vocab, d_topk, d_temp, d_ticket, d_gen, d_seed, d_out, top_p ? d_topp : nullptr);
     if (cudaDeviceSynchronize() != cudaSuccess) rc = BLINK_ECUDA;
     else if (cudaMemcpy(out, d_out, n * 4, cudaMemcpyDeviceToHost) != cudaSuccess) rc = BLINK_ECUDA;
   }
   cudaFree(d);
   return rc;
+}
+
+int blink_sample(const float* logits, int rows, int vocab, const int32_t* top_k, const float* temperature,
+                 const uint64_t* ticket, const int32_t* gen_index, const uint64_t* seed, int32_t* out) {
+  return sample_impl(logits, rows, vocab, top_k, temperature, nullptr, ticket, gen_index, seed, out);
+}
+
+int blink_sample_top_p(const float* logits, int rows, int vocab, const int32_t* top_k, const float* temperature,
+                       const float* top_p, const uint64_t* ticket, const int32_t* gen_index, const uint64_t* seed,
+                       int32_t* out) {
+  if (!top_p) return BLINK_EINVAL;
+  return sample_impl(logits, rows, vocab, top_k, temperature, top_p, ticket, gen_index, seed, out);
 }
 
 // ---- sampler for callers that cannot allocate --------------------------------------------------
@@ -448,7 +467,7 @@ int blink_sample_noalloc(const float* logits, int rows, int vocab, const int32_t
     return BLINK_ECUDA;
   const int grid = rows < 1184 ? rows : 1184;
   blink_sample_kernel<<<grid, FWD_THREADS, SAMPLE_SMEM_FLOATS * sizeof(float), st>>>(logits, rows, vocab, d_topk, d_temp,
-                                                                                     d_ticket, d_gen, d_seed, d_out);
+                                                                                     d_ticket, d_gen, d_seed, d_out, nullptr);
   if (cudaGetLastError() != cudaSuccess) return BLINK_ECUDA;
   if (cudaMemcpyAsync(out, d_out, n * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) return BLINK_ECUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess) return BLINK_ECUDA;
@@ -510,7 +529,8 @@ int blink_create(const blink_model_cfg* model, const blink_sched_cfg* sched, con
     c.gemm_tc = tc_available() && tc_shape_ok(c);
   if (sched->gemm_impl == BLINK_GEMM_TC && !c.gemm_tc) { delete x; return BLINK_EINVAL; }
   // epilogue fusion needs whole 128-feature tiles that do not straddle q|k|v or gate|up
-  c.fused = c.gemm_tc && c.qkv_dim % 128 == 0 && c.q_dim % 128 == 0 && c.kv_dim % 128 == 0 && c.F % 128 == 0 &&
+  if (sched->epilogue_fusion < BLINK_FUSION_AUTO || sched->epilogue_fusion > BLINK_FUSION_ON) { delete x; return BLINK_EINVAL; }
+  c.fused = sched->epilogue_fusion == BLINK_FUSION_ON && c.gemm_tc && c.qkv_dim % 128 == 0 && c.q_dim % 128 == 0 && c.kv_dim % 128 == 0 && c.F % 128 == 0 &&
             c.d % 128 == 0 && 128 % c.hd == 0;
   c.fused_norm = c.fused && c.E == 0;
   c.w_streaming = model->weights_layout == BLINK_WEIGHTS_STREAMING;
@@ -550,7 +570,7 @@ int blink_create(const blink_model_cfg* model, const blink_sched_cfg* sched, con
   TRY(dev_alloc(x, &c.b_N, MB)); TRY(dev_alloc(x, &c.b_prefilled, MB)); TRY(dev_alloc(x, &c.b_generated, MB));
   TRY(dev_alloc(x, &c.b_phase, MB)); TRY(dev_alloc(x, &c.b_have, MB)); TRY(dev_alloc(x, &c.b_need, MB));
   TRY(dev_alloc(x, &c.b_last, MB)); TRY(dev_alloc(x, &c.b_eos, MB)); TRY(dev_alloc(x, &c.b_topk, MB));
-  TRY(dev_alloc(x, &c.b_flags, MB)); TRY(dev_alloc(x, &c.b_temp, MB)); TRY(dev_alloc(x, &c.b_seed, MB));
+  TRY(dev_alloc(x, &c.b_flags, MB)); TRY(dev_alloc(x, &c.b_temp, MB)); TRY(dev_alloc(x, &c.b_topp, MB)); TRY(dev_alloc(x, &c.b_seed, MB));
   TRY(dev_alloc(x, &c.it_bslot, MB)); TRY(dev_alloc(x, &c.it_start, MB)); TRY(dev_alloc(x, &c.it_ntok, MB));
   TRY(dev_alloc(x, &c.it_qstart, MB)); TRY(dev_alloc(x, &c.it_row, MB));
   TRY(dev_alloc(x, &c.tok_id, TM)); TRY(dev_alloc(x, &c.tok_pos, TM)); TRY(dev_alloc(x, &c.tok_item, TM));
@@ -688,7 +708,9 @@ int blink_submit(blink_ctx* x, const blink_request* r, uint64_t* ticket_out) {
   const DevCtx& c = x->dc;
   if (r->n_prompt < 1 || r->n_prompt > c.max_prompt || r->max_new_tokens < 1 || r->max_new_tokens > c.max_new)
     return BLINK_EINVAL;
-  if (r->top_k < 0 || r->top_k > MAX_TOPK || (r->top_k > 0 && !(r->temperature > 0.f))) return BLINK_EINVAL;
+  if (!(r->top_p >= 0.f)) return BLINK_EINVAL;
+  const bool nucleus = r->top_p > 0.f && r->top_p < 1.f;
+  if (r->top_k < 0 || r->top_k > MAX_TOPK || ((r->top_k > 0 || nucleus) && !(r->temperature > 0.f))) return BLINK_EINVAL;
   if (r->eos_id >= c.V) return BLINK_EINVAL;
   for (int i = 0; i < r->n_prompt; ++i)
     if (r->prompt[i] < 0 || r->prompt[i] >= c.V) return BLINK_EINVAL;
@@ -718,7 +740,7 @@ int blink_submit(blink_ctx* x, const blink_request* r, uint64_t* ticket_out) {
   SubEntry& e = x->sub_q[ticket % (uint64_t)c.n_slots];
   e.ticket = ticket; e.seed = r->seed; e.user_tag = r->user_tag; e.slot = (uint32_t)slot;
   e.n_prompt = (uint32_t)r->n_prompt; e.max_new = (uint32_t)r->max_new_tokens; e.top_k = (uint32_t)r->top_k;
-  e.temperature = r->temperature; e.eos_id = r->eos_id; e.flags = r->forced_tokens ? REQ_FLAG_FORCED : 0; e.pad = 0;
+  e.temperature = r->temperature; e.eos_id = r->eos_id; e.flags = r->forced_tokens ? REQ_FLAG_FORCED : 0; e.top_p = r->top_p;
   SlotInfo& si = x->slots[slot];
   si.busy = true; si.ticket = ticket; si.user_tag = r->user_tag; si.max_new = r->max_new_tokens; si.consumed = 0;
   si.t_submit_ns = now_ns();

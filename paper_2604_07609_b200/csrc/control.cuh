@@ -70,7 +70,8 @@ __device__ __forceinline__ bool grid_barrier(const DevCtx& c, unsigned long long
     int ok = 1;
     SchedState* ss = c.ss;
     target += gridDim.x;
-    __threadfence();
+    // release at gpu scope is cumulative: the stores of the CTA's other threads, ordered before this
+    // point by the barrier above, are covered without a separate fence
     asm volatile("red.release.gpu.global.add.u64 [%0], 1;" ::"l"(&ss->bar_ctr) : "memory");
     long long t0 = 0;
     unsigned int polls = 0;
@@ -267,6 +268,7 @@ static __device__ void ingress(const DevCtx& c, unsigned long long tail) {
       cold.seed = en->seed;
       cold.user_tag = en->user_tag;
       cold.flags = flags;
+      cold.top_p = en->top_p;
       SlotHot& hot = c.slot_hot[slot];
       hot.n_prompt = np;
       hot.generated = 0;
@@ -361,6 +363,7 @@ static __device__ int schedule_step(const DevCtx& c, unsigned long long visible)
       c.b_eos[b] = cold.eos_id;
       c.b_topk[b] = (int)cold.top_k;
       c.b_temp[b] = cold.temperature;
+      c.b_topp[b] = cold.top_p;
       c.b_seed[b] = cold.seed;
       c.b_flags[b] = (int)cold.flags;
       reserved += need;

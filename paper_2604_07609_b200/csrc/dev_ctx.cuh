@@ -34,7 +34,7 @@ struct SlotCold {
   uint64_t seed;
   uint64_t user_tag;
   uint32_t flags;  // bit0: forced tokens present
-  uint32_t pad;
+  float top_p;     // outside (0, 1): no nucleus cut
 };
 enum { REQ_FLAG_FORCED = 1 };
 
@@ -50,7 +50,7 @@ struct SubEntry {
   float temperature;
   int32_t eos_id;
   uint32_t flags;
-  uint32_t pad;
+  float top_p;
 };
 
 // Pinned control mailbox (host and device both read and write single words of it).
@@ -163,7 +163,7 @@ struct DevCtx {
   long long* b_ticket;
   int32_t *b_slot, *b_P, *b_N, *b_prefilled, *b_generated, *b_phase, *b_have, *b_need, *b_last, *b_eos,
       *b_topk, *b_flags;
-  float* b_temp;
+  float *b_temp, *b_topp;
   unsigned long long* b_seed;
   // current step
   int32_t *it_bslot, *it_start, *it_ntok, *it_qstart, *it_row;  // [MB] per item

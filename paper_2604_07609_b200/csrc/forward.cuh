@@ -9,6 +9,7 @@
 // context attention, fused MLP, sampling captured inside the step); Section 6.1
 // lists the engine features.  The math is the standard pre-norm decoder.
 #pragma once
+#include "control.cuh"
 #include "dev_ctx.cuh"
 
 namespace blink {
@@ -210,16 +211,33 @@ template <typename WT>
 __device__ __noinline__ void norm_apply_rows(const float* __restrict__ h, const float* __restrict__ rowss,
                                              const float* __restrict__ g, WT* __restrict__ out, const int32_t* rows, int R,
                                              int d, float eps) {
+  constexpr int U = 4;   // items whose loads are in flight before the first store (one CTA per SM: latency-bound otherwise)
   const int d4 = d >> 2;
   const int total = R * d4;   // < 2^31
   const float inv_d = 1.0f / (float)d;
-  for (int idx = blockIdx.x * FWD_THREADS + threadIdx.x; idx < total; idx += gridDim.x * FWD_THREADS) {
-    const int r = idx / d4, j = (idx - r * d4) * 4;
-    const int t = rows != nullptr ? rows[r] : r;
-    const float4 v = __ldcg(reinterpret_cast<const float4*>(h + (size_t)t * d + j));
-    const float inv = 1.0f / sqrtf(__ldcg(rowss + t) * inv_d + eps);
-    const float4 gg = *reinterpret_cast<const float4*>(g + j);
-    store4<WT>(out + (size_t)r * d + j, v.x * inv * gg.x, v.y * inv * gg.y, v.z * inv * gg.z, v.w * inv * gg.w);
+  const int stride = gridDim.x * FWD_THREADS;
+  for (int base = blockIdx.x * FWD_THREADS + threadIdx.x; base < total; base += U * stride) {
+    float4 v[U], gg[U];
+    float ss[U];
+    int r[U], j[U];
+#pragma unroll
+    for (int k = 0; k < U; ++k) {
+      const int idx = min(base + k * stride, total - 1);   // clamped: the tail loads a valid item twice
+      r[k] = idx / d4;
+      j[k] = (idx - r[k] * d4) * 4;
+      const int t = rows != nullptr ? rows[r[k]] : r[k];
+      v[k] = __ldcg(reinterpret_cast<const float4*>(h + (size_t)t * d + j[k]));
+      ss[k] = __ldcg(rowss + t);
+      gg[k] = *reinterpret_cast<const float4*>(g + j[k]);
+    }
+#pragma unroll
+    for (int k = 0; k < U; ++k) {
+      if (base + k * stride < total) {
+        const float inv = 1.0f / sqrtf(ss[k] * inv_d + eps);
+        store4<WT>(out + (size_t)r[k] * d + j[k], v[k].x * inv * gg[k].x, v[k].y * inv * gg[k].y, v[k].z * inv * gg[k].z,
+                   v[k].w * inv * gg[k].w);
+      }
+    }
   }
 }
 
@@ -397,6 +415,10 @@ static __device__ void phase_rope_kv(const DevCtx& c, int layer) {
       store4<WT>(dst + i, x1.x, x1.y, x1.z, x1.w);
       store4<WT>(dst + i + half, x2.x, x2.y, x2.z, x2.w);
     }
+    if (c.gemm_tc) {   // the split-K GEMM of the next layer adds partial sums into this buffer: leave it cleared
+      *reinterpret_cast<float4*>(row + i) = make_float4(0.f, 0.f, 0.f, 0.f);
+      *reinterpret_cast<float4*>(row + i + half) = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
   }
 }
 
@@ -408,6 +430,9 @@ static __device__ void phase_rope_kv(const DevCtx& c, int layer) {
 // QKV tile nt: RoPE on the q and k heads it covers (the rotation partner i + hd/2 of a feature lies in
 // the same tile, hd/8 lanes away), q into the 16-bit attention operand, k and v into the paged pool;
 // then the tile is cleared for the next GEMM that adds partial sums into this buffer.
+constexpr int FIX_U = 8;   // rows per warp whose loads are issued before the first dependent use
+constexpr int FIX_WARPS = FWD_THREADS / 32;
+
 template <typename WT>
 __device__ __noinline__ void fixup_rope_kv(const DevCtx& c, int layer, int nt, int t0, int t1) {
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
@@ -418,38 +443,49 @@ __device__ __noinline__ void fixup_rope_kv(const DevCtx& c, int layer, int nt, i
   const int i = low ? i0 : i0 - half;         // rotation pair index
   const int partner = half >> 2;              // lanes between the two halves of a pair
   if (f >= c.qkv_dim) return;                 // whole warp: tiles are not ragged on this path
-  for (int t = t0 + w; t < t1; t += FWD_THREADS / 32) {
-    float4* src = reinterpret_cast<float4*>(c.qkv + (size_t)t * c.qkv_dim + f);
-    const float4 x = __ldcg(src);
-    float4 o;
-    o.x = __shfl_xor_sync(0xffffffffu, x.x, partner);
-    o.y = __shfl_xor_sync(0xffffffffu, x.y, partner);
-    o.z = __shfl_xor_sync(0xffffffffu, x.z, partner);
-    o.w = __shfl_xor_sync(0xffffffffu, x.w, partner);
-    float4 y = x;
-    if (hh < c.Hq + c.Hkv) {
-      const int pos = c.tok_pos[t];
-      const float4 cs = *reinterpret_cast<const float4*>(c.rope_cos + (size_t)pos * half + i);
-      const float4 sn = *reinterpret_cast<const float4*>(c.rope_sin + (size_t)pos * half + i);
-      // the same explicit fused forms as the stand-alone RoPE phase: x1 = low half, x2 = high half
-      if (low) {
-        y = make_float4(fmaf(x.x, cs.x, -__fmul_rn(o.x, sn.x)), fmaf(x.y, cs.y, -__fmul_rn(o.y, sn.y)),
-                        fmaf(x.z, cs.z, -__fmul_rn(o.z, sn.z)), fmaf(x.w, cs.w, -__fmul_rn(o.w, sn.w)));
-      } else {
-        y = make_float4(fmaf(x.x, cs.x, __fmul_rn(o.x, sn.x)), fmaf(x.y, cs.y, __fmul_rn(o.y, sn.y)),
-                        fmaf(x.z, cs.z, __fmul_rn(o.z, sn.z)), fmaf(x.w, cs.w, __fmul_rn(o.w, sn.w)));
+  const bool rot = hh < c.Hq + c.Hkv;
+  const bool is_q = hh < c.Hq;
+  const int kv = hh < c.Hq + c.Hkv ? 0 : 1;
+  const int kvh = hh - c.Hq - kv * c.Hkv;
+  for (int tb = t0 + w; tb < t1; tb += FIX_WARPS * FIX_U) {
+    float4 x[FIX_U];
+    int pos[FIX_U], sm[FIX_U];
+#pragma unroll
+    for (int u = 0; u < FIX_U; ++u) {
+      const int t = min(tb + u * FIX_WARPS, t1 - 1);   // clamped: rows past the end repeat the last one (not stored)
+      x[u] = __ldcg(reinterpret_cast<const float4*>(c.qkv + (size_t)t * c.qkv_dim + f));
+      pos[u] = rot ? c.tok_pos[t] : 0;
+      sm[u] = is_q ? 0 : c.tok_slotmap[t];
+    }
+#pragma unroll
+    for (int u = 0; u < FIX_U; ++u) {
+      const int t = tb + u * FIX_WARPS;
+      float4 o;
+      o.x = __shfl_xor_sync(0xffffffffu, x[u].x, partner);
+      o.y = __shfl_xor_sync(0xffffffffu, x[u].y, partner);
+      o.z = __shfl_xor_sync(0xffffffffu, x[u].z, partner);
+      o.w = __shfl_xor_sync(0xffffffffu, x[u].w, partner);
+      if (t >= t1) continue;   // uniform over the warp
+      float4 y = x[u];
+      float4 cs[FIX_U], sn[FIX_U];
+      if (rot) {
+        cs[u] = *reinterpret_cast<const float4*>(c.rope_cos + (size_t)pos[u] * half + i);
+        sn[u] = *reinterpret_cast<const float4*>(c.rope_sin + (size_t)pos[u] * half + i);
+        // the same explicit fused forms as the stand-alone RoPE phase: x1 = low half, x2 = high half
+        if (low) {
+          y = make_float4(fmaf(x[u].x, cs[u].x, -__fmul_rn(o.x, sn[u].x)), fmaf(x[u].y, cs[u].y, -__fmul_rn(o.y, sn[u].y)),
+                          fmaf(x[u].z, cs[u].z, -__fmul_rn(o.z, sn[u].z)), fmaf(x[u].w, cs[u].w, -__fmul_rn(o.w, sn[u].w)));
+        } else {
+          y = make_float4(fmaf(x[u].x, cs[u].x, __fmul_rn(o.x, sn[u].x)), fmaf(x[u].y, cs[u].y, __fmul_rn(o.y, sn[u].y)),
+                          fmaf(x[u].z, cs[u].z, __fmul_rn(o.z, sn[u].z)), fmaf(x[u].w, cs[u].w, __fmul_rn(o.w, sn[u].w)));
+        }
       }
+      WT* dst;
+      if (is_q) dst = reinterpret_cast<WT*>(c.qb) + (size_t)t * c.q_dim + (size_t)hh * hd + i0;
+      else dst = kv_tile<WT>(c, layer, kv, sm[u] / c.bs, kvh) + (size_t)(sm[u] % c.bs) * hd + i0;
+      store4<WT>(dst, y.x, y.y, y.z, y.w);
+      __stcg(reinterpret_cast<float4*>(c.qkv + (size_t)t * c.qkv_dim + f), make_float4(0.f, 0.f, 0.f, 0.f));
     }
-    WT* dst;
-    if (hh < c.Hq) {
-      dst = reinterpret_cast<WT*>(c.qb) + (size_t)t * c.q_dim + (size_t)hh * hd + i0;
-    } else {
-      const int sm = c.tok_slotmap[t];
-      const int kv = hh < c.Hq + c.Hkv ? 0 : 1;
-      dst = kv_tile<WT>(c, layer, kv, sm / c.bs, hh - c.Hq - kv * c.Hkv) + (size_t)(sm % c.bs) * hd + i0;
-    }
-    store4<WT>(dst, y.x, y.y, y.z, y.w);
-    __stcg(src, make_float4(0.f, 0.f, 0.f, 0.f));
   }
 }
 
@@ -459,29 +495,45 @@ __device__ __noinline__ void fixup_silu(float* gu, WT* act, int F, int j, int t0
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   const int f = j * 128 + lane * 4;
   if (f >= F) return;
-  for (int t = t0 + w; t < t1; t += FWD_THREADS / 32) {
-    float4* gp = reinterpret_cast<float4*>(gu + (size_t)t * 2 * F + f);
-    float4* up = reinterpret_cast<float4*>(gu + (size_t)t * 2 * F + F + f);
-    const float4 g = __ldcg(gp), u = __ldcg(up);
-    store4<WT>(act + (size_t)t * F + f, g.x / (1.0f + __expf(-g.x)) * u.x, g.y / (1.0f + __expf(-g.y)) * u.y,
-               g.z / (1.0f + __expf(-g.z)) * u.z, g.w / (1.0f + __expf(-g.w)) * u.w);
-    __stcg(gp, make_float4(0.f, 0.f, 0.f, 0.f));
-    __stcg(up, make_float4(0.f, 0.f, 0.f, 0.f));
+  for (int tb = t0 + w; tb < t1; tb += FIX_WARPS * FIX_U) {
+    float4 g[FIX_U], u4[FIX_U];
+#pragma unroll
+    for (int u = 0; u < FIX_U; ++u) {
+      const int t = min(tb + u * FIX_WARPS, t1 - 1);
+      g[u] = __ldcg(reinterpret_cast<const float4*>(gu + (size_t)t * 2 * F + f));
+      u4[u] = __ldcg(reinterpret_cast<const float4*>(gu + (size_t)t * 2 * F + F + f));
+    }
+#pragma unroll
+    for (int u = 0; u < FIX_U; ++u) {
+      const int t = tb + u * FIX_WARPS;
+      if (t >= t1) continue;
+      store4<WT>(act + (size_t)t * F + f, g[u].x / (1.0f + __expf(-g[u].x)) * u4[u].x, g[u].y / (1.0f + __expf(-g[u].y)) * u4[u].y,
+                 g[u].z / (1.0f + __expf(-g[u].z)) * u4[u].z, g[u].w / (1.0f + __expf(-g[u].w)) * u4[u].w);
+      __stcg(reinterpret_cast<float4*>(gu + (size_t)t * 2 * F + f), make_float4(0.f, 0.f, 0.f, 0.f));
+      __stcg(reinterpret_cast<float4*>(gu + (size_t)t * 2 * F + F + f), make_float4(0.f, 0.f, 0.f, 0.f));
+    }
   }
 }
 
 // residual tile nt of rows [t0, t1): its share of sum(x^2) per row
 static __device__ __noinline__ void fixup_sumsq(const float* h, int ld, int N, float* rowss, int nt, int t0, int t1) {
+  constexpr int U = 8;
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   const int f = nt * 128 + lane * 4;
-  for (int t = t0 + w; t < t1; t += FWD_THREADS / 32) {
-    float s = 0.f;
-    if (f < N) {
-      const float4 x = __ldcg(reinterpret_cast<const float4*>(h + (size_t)t * ld + f));
-      s = fmaf(x.x, x.x, fmaf(x.y, x.y, fmaf(x.z, x.z, x.w * x.w)));
+  for (int tb = t0 + w; tb < t1; tb += FIX_WARPS * U) {
+    float4 x[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int t = min(tb + u * FIX_WARPS, t1 - 1);
+      x[u] = f < N ? __ldcg(reinterpret_cast<const float4*>(h + (size_t)t * ld + f)) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
-    s = warp_sum(s);
-    if (lane == 0) atomicAdd(rowss + t, s);
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int t = tb + u * FIX_WARPS;
+      float s = fmaf(x[u].x, x[u].x, fmaf(x[u].y, x[u].y, fmaf(x[u].z, x[u].z, x[u].w * x[u].w)));
+      s = warp_sum(s);
+      if (lane == 0 && t < t1) atomicAdd(rowss + t, s);
+    }
   }
 }
 
@@ -627,7 +679,7 @@ constexpr int ATTN_SMEM_FLOATS(int HD, int NREP) { return NREP * HD + 2 * 8 * NR
 // SILU_U items in flight before it stores.  A function of its own: inlined into the loop kernel
 // the buffers of loaded values end up in local memory.
 template <typename WT>
-__device__ __noinline__ void silu_mul_rows(const float* __restrict__ gu, WT* __restrict__ out, int T, int F) {
+__device__ __noinline__ void silu_mul_rows(float* __restrict__ gu, WT* __restrict__ out, int T, int F, bool clear) {
   constexpr int SILU_U = 4;
   const int F4 = F / 4;
   const int total = T * F4;   // < 2^31: at most a few thousand rows
@@ -649,6 +701,10 @@ __device__ __noinline__ void silu_mul_rows(const float* __restrict__ gu, WT* __r
         store4<WT>(out + (size_t)t * F + j, g[k].x / (1.0f + __expf(-g[k].x)) * u[k].x,
                    g[k].y / (1.0f + __expf(-g[k].y)) * u[k].y, g[k].z / (1.0f + __expf(-g[k].z)) * u[k].z,
                    g[k].w / (1.0f + __expf(-g[k].w)) * u[k].w);
+        if (clear) {   // consumed: the next split-K gate/up GEMM adds partial sums into a cleared buffer
+          __stcg(reinterpret_cast<float4*>(gu + (size_t)t * 2 * F + j), make_float4(0.f, 0.f, 0.f, 0.f));
+          __stcg(reinterpret_cast<float4*>(gu + (size_t)t * 2 * F + F + j), make_float4(0.f, 0.f, 0.f, 0.f));
+        }
       }
     }
   }
@@ -656,7 +712,7 @@ __device__ __noinline__ void silu_mul_rows(const float* __restrict__ gu, WT* __r
 template <typename WT>
 static __device__ void phase_silu_mul(const DevCtx& c) {
   const int T = c.E > 0 ? c.ss->cur_T * c.topE : c.ss->cur_T;   // rows of the gate/up buffer
-  if (T > 0) silu_mul_rows<WT>(c.gu, reinterpret_cast<WT*>(c.act), T, c.F);
+  if (T > 0) silu_mul_rows<WT>(c.gu, reinterpret_cast<WT*>(c.act), T, c.F, c.gemm_tc != 0);
 }
 
 // ---- routed experts: group the (token, expert) pairs by expert and gather their rows ---------
@@ -728,12 +784,254 @@ __device__ __forceinline__ uint32_t float_key(float f) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
+// ---- top-p (nucleus) arithmetic: Section 4.2 names "Top-P with temperature" as the in-step sampler ----
+// Weights are integers, q = floor(exp(z - z0) * 2^40) with z0 the largest z of the row, so that every
+// sum is exact and no result depends on the order in which a parallel machine adds: the nucleus is
+// the smallest prefix of the order (z desc, index asc) with cum * 2^24 >= P24 * Q (Q = total weight,
+// P24 = round(top_p * 2^24) in [1, 2^24]); the draw is renormalised to its weight M: with the 24-bit
+// uniform x24, the token is the first of the order with cum > (x24 * M) >> 24.
+__device__ __forceinline__ unsigned long long nucleus_weight(float z, float z0) {
+  return __double2ull_rd(exp((double)z - (double)z0) * 1099511627776.0);
+}
+__device__ __forceinline__ unsigned long long nucleus_p24(float top_p) {
+  long long p = (long long)rint((double)top_p * 16777216.0);
+  return (unsigned long long)(p < 1 ? 1 : (p > 16777216 ? 16777216 : p));
+}
+// ceil(p24 * Q / 2^24): the weight the nucleus has to reach (Q < 2^58, p24 <= 2^24)
+__device__ __forceinline__ unsigned long long nucleus_need(unsigned long long p24, unsigned long long Q) {
+  unsigned long long lo = p24 * Q, hi = __umul64hi(p24, Q);
+  const unsigned long long lo2 = lo + 16777215ull;
+  if (lo2 < lo) hi += 1;
+  return (hi << 40) | (lo2 >> 24);
+}
+// (x24 * M) >> 24
+__device__ __forceinline__ unsigned long long nucleus_target(unsigned long long x24, unsigned long long M) {
+  return (__umul64hi(x24, M) << 40) | ((x24 * M) >> 24);
+}
+
+// Shared state of the whole-row nucleus search (one CTA per row).
+constexpr int NUC_CAND = 1024;
+struct NucShared {
+  unsigned long long m0[256];   // level 0: weight per bucket of z (linear in z between the row's min and max)
+  unsigned int c0[256];         //          and number of entries
+  unsigned long long m[256];    // deeper levels: buckets linear in the float key inside [klo, khi]
+  unsigned int cn[256];
+  unsigned long long acc;       // weight of everything ahead of the current member set in the order
+  unsigned long long res_cum;   // result: cumulative weight up to and including the entry found
+  unsigned int klo, khi, cnt;
+  int b0, first, done, res_idx, n;
+  float zmin, scale;
+  unsigned int chunk_cnt[FWD_THREADS];
+};
+__device__ __forceinline__ int nuc_bucket0(float z, float zmin, float scale) {
+  const int b = (int)((z - zmin) * scale);
+  return b < 0 ? 0 : (b > 255 ? 255 : b);
+}
+
+// First entry of the order (z desc, index asc) whose cumulative weight exceeds t (t < total weight).
+// The member set starts as one level-0 bucket and is narrowed 256-fold per pass over the row (buckets
+// over the float-key interval of the set) until it fits the candidate buffer, which is then ranked
+// exactly.  A set that cannot be narrowed (more than NUC_CAND equal values) is resolved by index.
+static __device__ __noinline__ void nucleus_locate(NucShared& st, const float* lg, int V, float temp, float z0,
+                                                   unsigned long long t, float* s_cz, int* s_ci, float* s_sz, int* s_si) {
+  const int tid = threadIdx.x;
+  if (tid == 0) {
+    unsigned long long acc = 0;
+    int b = 255;
+    for (; b > 0; --b) {
+      if (acc + st.m0[b] > t) break;
+      acc += st.m0[b];
+    }
+    st.b0 = b; st.acc = acc; st.cnt = st.c0[b]; st.klo = 0u; st.khi = 0xffffffffu; st.first = 1; st.done = 0;
+  }
+  __syncthreads();
+  const float zmin = st.zmin, scale = st.scale;
+  for (int level = 0; level < 8; ++level) {   // a level divides the key interval by 256: four suffice
+    const int b0 = st.b0;
+    const unsigned int klo = st.klo, khi = st.khi;
+    if (st.cnt <= (unsigned)NUC_CAND) {
+      // ---- gather the members, rank them exactly, walk the cumulative weights ----
+      if (tid == 0) st.n = 0;
+      __syncthreads();
+      for (int i = tid; i < V; i += FWD_THREADS) {
+        const float z = __fdiv_rn(lg[i], temp);
+        const unsigned int key = float_key(z);
+        if (nuc_bucket0(z, zmin, scale) == b0 && key >= klo && key <= khi) {
+          const int p = atomicAdd(&st.n, 1);
+          if (p < NUC_CAND) { s_cz[p] = z; s_ci[p] = i; }
+        }
+      }
+      __syncthreads();
+      const int nc = min(st.n, NUC_CAND);
+      for (int a = tid; a < nc; a += FWD_THREADS) {
+        const float za = s_cz[a];
+        const int ia = s_ci[a];
+        int rank = 0;
+        for (int j = 0; j < nc; ++j) {
+          const float zj = s_cz[j];
+          rank += (zj > za) || (zj == za && s_ci[j] < ia);
+        }
+        s_sz[rank] = za; s_si[rank] = ia;
+      }
+      __syncthreads();
+      if (tid == 0) {
+        unsigned long long cum = st.acc;
+        int pick = nc > 0 ? s_si[nc - 1] : 0;
+        for (int j = 0; j < nc; ++j) {
+          cum += nucleus_weight(s_sz[j], z0);
+          if (cum > t) { pick = s_si[j]; break; }
+        }
+        st.res_idx = pick; st.res_cum = cum; st.done = 1;
+      }
+      __syncthreads();
+      return;
+    }
+    if (st.first) {   // key interval of the level-0 bucket's members
+      __syncthreads();
+      if (tid == 0) { st.klo = 0xffffffffu; st.khi = 0u; }
+      __syncthreads();
+      for (int i = tid; i < V; i += FWD_THREADS) {
+        const float z = __fdiv_rn(lg[i], temp);
+        if (nuc_bucket0(z, zmin, scale) == b0) {
+          const unsigned int key = float_key(z);
+          atomicMin(&st.klo, key);
+          atomicMax(&st.khi, key);
+        }
+      }
+      __syncthreads();
+      if (tid == 0) st.first = 0;
+      __syncthreads();
+      continue;   // same member set, now with its key interval
+    }
+    if (klo == khi) {
+      // ---- more than NUC_CAND entries with one and the same z: equal weights, ordered by index ----
+      const float z = __uint_as_float((klo & 0x80000000u) ? (klo & 0x7fffffffu) : ~klo);
+      const unsigned long long q0 = nucleus_weight(z, z0);            // > 0: the set's weight exceeds t - acc
+      const unsigned long long jl = q0 > 0 ? (t - st.acc) / q0 : 0;   // entries of the set ahead of the one sought
+      const int ch = (V + FWD_THREADS - 1) / FWD_THREADS;
+      const int i0 = tid * ch, i1 = min(V, i0 + ch);
+      unsigned int mine = 0;
+      for (int i = i0; i < i1; ++i) {
+        const float zi = __fdiv_rn(lg[i], temp);
+        mine += (nuc_bucket0(zi, zmin, scale) == b0 && float_key(zi) == klo) ? 1u : 0u;
+      }
+      st.chunk_cnt[tid] = mine;
+      __syncthreads();
+      unsigned long long before = 0;
+      for (int k = 0; k < tid; ++k) before += st.chunk_cnt[k];
+      if (jl >= before && jl < before + mine) {
+        unsigned long long seen = before;
+        for (int i = i0; i < i1; ++i) {
+          const float zi = __fdiv_rn(lg[i], temp);
+          if (nuc_bucket0(zi, zmin, scale) == b0 && float_key(zi) == klo) {
+            if (seen == jl) { st.res_idx = i; st.res_cum = st.acc + (jl + 1) * q0; st.done = 1; break; }
+            ++seen;
+          }
+        }
+      }
+      __syncthreads();
+      if (tid == 0 && !st.done) { st.res_idx = 0; st.res_cum = st.acc; st.done = 1; }   // cannot happen for t < total
+      __syncthreads();
+      return;
+    }
+    // ---- one more level: 256 buckets over the key interval [klo, khi] ----
+    st.m[tid] = 0ull;
+    st.cn[tid] = 0u;
+    __syncthreads();
+    const unsigned long long W = (unsigned long long)khi - klo + 1ull;
+    for (int i = tid; i < V; i += FWD_THREADS) {
+      const float z = __fdiv_rn(lg[i], temp);
+      const unsigned int key = float_key(z);
+      if (nuc_bucket0(z, zmin, scale) == b0 && key >= klo && key <= khi) {
+        const int b = (int)((((unsigned long long)(key - klo)) << 8) / W);
+        atomicAdd(&st.m[b], nucleus_weight(z, z0));
+        atomicAdd(&st.cn[b], 1u);
+      }
+    }
+    __syncthreads();
+    if (tid == 0) {
+      unsigned long long acc = st.acc;
+      int b = 255;
+      for (; b > 0; --b) {
+        if (acc + st.m[b] > t) break;
+        acc += st.m[b];
+      }
+      st.acc = acc;
+      st.cnt = st.cn[b];
+      // keys of bucket b: (key - klo) * 256 / W == b
+      st.klo = klo + (unsigned int)(((unsigned long long)b * W + 255ull) >> 8);
+      st.khi = klo + (unsigned int)((((unsigned long long)(b + 1) * W + 255ull) >> 8) - 1ull);
+    }
+    __syncthreads();
+  }
+  if (tid == 0 && !st.done) { st.res_idx = 0; st.res_cum = st.acc; st.done = 1; }
+  __syncthreads();
+}
+
+// Top-p over the whole row (no top-k cut): z = logit / T, weights and order as described above.
+// The result is returned by thread 0 (other threads return -1).
+static __device__ __noinline__ int sample_row_nucleus(const float* lg, int V, float temp, float top_p, unsigned long long ticket,
+                                                      int gen_index, unsigned long long seed, float* smem) {
+  __shared__ NucShared st;
+  __shared__ float s_mx[FWD_THREADS / 32], s_mn[FWD_THREADS / 32];
+  const int tid = threadIdx.x;
+  float* s_cz = smem + 256;
+  int* s_ci = reinterpret_cast<int*>(smem + 256 + NUC_CAND);
+  float* s_sz = smem + 256 + 2 * NUC_CAND;
+  int* s_si = reinterpret_cast<int*>(smem + 256 + 3 * NUC_CAND);
+  __syncthreads();
+  // range of the row (z is monotone in the logit, so min and max can be taken on logits)
+  float lmax = -INFINITY, lmin = INFINITY;
+  for (int i = tid; i < V; i += FWD_THREADS) {
+    const float v = lg[i];
+    lmax = fmaxf(lmax, v);
+    lmin = fminf(lmin, v);
+  }
+  lmax = warp_max(lmax);
+  lmin = -warp_max(-lmin);
+  if ((tid & 31) == 0) { s_mx[tid >> 5] = lmax; s_mn[tid >> 5] = lmin; }
+  st.m0[tid] = 0ull;
+  st.c0[tid] = 0u;
+  __syncthreads();
+#pragma unroll
+  for (int i = 0; i < FWD_THREADS / 32; ++i) { lmax = fmaxf(lmax, s_mx[i]); lmin = fminf(lmin, s_mn[i]); }
+  const float z0 = __fdiv_rn(lmax, temp), zmin = __fdiv_rn(lmin, temp);
+  const float scale = z0 > zmin ? 255.0f / (z0 - zmin) : 0.0f;
+  if (tid == 0) { st.zmin = zmin; st.scale = scale; }
+  // level 0: weights per bucket of z
+  for (int i = tid; i < V; i += FWD_THREADS) {
+    const float z = __fdiv_rn(lg[i], temp);
+    const int b = nuc_bucket0(z, zmin, scale);
+    atomicAdd(&st.m0[b], nucleus_weight(z, z0));
+    atomicAdd(&st.c0[b], 1u);
+  }
+  __syncthreads();
+  __shared__ unsigned long long s_t;
+  if (tid == 0) {
+    unsigned long long Q = 0;
+    for (int b = 0; b < 256; ++b) Q += st.m0[b];
+    s_t = nucleus_need(nucleus_p24(top_p), Q) - 1ull;   // first entry with cum >= need  <=>  cum > need - 1
+  }
+  __syncthreads();
+  nucleus_locate(st, lg, V, temp, z0, s_t, s_cz, s_ci, s_sz, s_si);   // end of the nucleus: its weight is res_cum
+  if (tid == 0) {
+    const uint32_t x = philox4x32_10_word0((uint32_t)ticket, (uint32_t)(ticket >> 32), (uint32_t)gen_index, 0u,
+                                           (uint32_t)seed, (uint32_t)(seed >> 32));
+    s_t = nucleus_target((unsigned long long)(x >> 8), st.res_cum);
+  }
+  __syncthreads();
+  nucleus_locate(st, lg, V, temp, z0, s_t, s_cz, s_ci, s_sz, s_si);
+  const int result = tid == 0 ? st.res_idx : -1;
+  __syncthreads();
+  return result;
+}
+
 // One CTA per sampled row.  Greedy: lowest index among the maxima.  Top-k: z = logit / T
 // (IEEE fp32 divide); the k largest by (z desc, index asc) are found with a radix select
 // on the float keys; weights exp(z - z0) and the inverse-CDF walk run in fp64.
 // The result is returned by thread 0 (other threads return -1).
-static __device__ int sample_row(const float* lg, int V, int top_k, float temp, unsigned long long ticket, int gen_index,
-                          unsigned long long seed, float* smem) {
+static __device__ int sample_row(const float* lg, int V, int top_k, float temp, float top_p, unsigned long long ticket,
+                                 int gen_index, unsigned long long seed, float* smem) {
   constexpr int CAND_MAX = 1024;
   const int tid = threadIdx.x;
   uint32_t* s_hist = reinterpret_cast<uint32_t*>(smem);             // [256]
@@ -746,6 +1044,8 @@ static __device__ int sample_row(const float* lg, int V, int top_k, float temp, 
   __shared__ float s_tz[MAX_TOPK];
   __shared__ int s_ti[MAX_TOPK];
   int result = -1;
+  const bool nucleus = top_p > 0.f && top_p < 1.f;   // outside (0, 1): no nucleus cut
+  if (top_k <= 0 && nucleus) return sample_row_nucleus(lg, V, temp, top_p, ticket, gen_index, seed, smem);
   __syncthreads();
   if (top_k <= 0) {
     float bv = -INFINITY;
@@ -897,18 +1197,39 @@ static __device__ int sample_row(const float* lg, int V, int top_k, float temp, 
   if (tid == 0) {
     const uint32_t x = philox4x32_10_word0((uint32_t)ticket, (uint32_t)(ticket >> 32), (uint32_t)gen_index, 0u,
                                            (uint32_t)seed, (uint32_t)(seed >> 32));
-    const double u = (double)(x >> 8) * (1.0 / 16777216.0);
     const int kk = min(k, nc);
-    double total = 0.0;
-    for (int j = 0; j < kk; ++j) total += exp((double)s_tz[j] - (double)s_tz[0]);
-    const double target = u * total;
-    double accum = 0.0;
-    int pick = s_ti[kk - 1];
-    for (int j = 0; j < kk; ++j) {
-      accum += exp((double)s_tz[j] - (double)s_tz[0]);
-      if (accum > target) { pick = s_ti[j]; break; }
+    if (nucleus) {
+      // nucleus inside the k candidates (already in the order), integer weights
+      unsigned long long Q = 0;
+      for (int j = 0; j < kk; ++j) Q += nucleus_weight(s_tz[j], s_tz[0]);
+      const unsigned long long need = nucleus_need(nucleus_p24(top_p), Q);
+      unsigned long long M = 0;
+      int m = 0;
+      for (; m < kk; ++m) {
+        M += nucleus_weight(s_tz[m], s_tz[0]);
+        if (M >= need) { ++m; break; }
+      }
+      const unsigned long long target = nucleus_target((unsigned long long)(x >> 8), M);
+      unsigned long long cum = 0;
+      int pick = s_ti[m - 1];
+      for (int j = 0; j < m; ++j) {
+        cum += nucleus_weight(s_tz[j], s_tz[0]);
+        if (cum > target) { pick = s_ti[j]; break; }
+      }
+      result = pick;
+    } else {
+      const double u = (double)(x >> 8) * (1.0 / 16777216.0);
+      double total = 0.0;
+      for (int j = 0; j < kk; ++j) total += exp((double)s_tz[j] - (double)s_tz[0]);
+      const double target = u * total;
+      double accum = 0.0;
+      int pick = s_ti[kk - 1];
+      for (int j = 0; j < kk; ++j) {
+        accum += exp((double)s_tz[j] - (double)s_tz[0]);
+        if (accum > target) { pick = s_ti[j]; break; }
+      }
+      result = pick;
     }
-    result = pick;
   }
   __syncthreads();
   return result;
@@ -927,11 +1248,11 @@ static __device__ void phase_sample(const DevCtx& c, float* smem) {
       float* dst = c.logits_capture + (size_t)(rows_before + r) * V;
       for (int i = tid; i < V; i += FWD_THREADS) dst[i] = lg[i];
     }
-    const int tok = sample_row(lg, V, min(c.b_topk[b], MAX_TOPK), c.b_temp[b], (unsigned long long)c.b_ticket[b],
+    const int tok = sample_row(lg, V, min(c.b_topk[b], MAX_TOPK), c.b_temp[b], c.b_topp[b], (unsigned long long)c.b_ticket[b],
                                c.b_generated[b], c.b_seed[b], smem);
     if (tid == 0) c.row_sampled[r] = tok;
   }
 }
-constexpr int SAMPLE_SMEM_FLOATS = 256 + 2 * 1024;
+constexpr int SAMPLE_SMEM_FLOATS = 256 + 4 * 1024;
 
 }  // namespace blink

@@ -215,3 +215,60 @@ def test_decode_attention_many_rows_whole_and_split_units():
     err, _, trace, toks, ora = _compare(model, sched, reqs, w, O2.round_bf16, TOL_BF16)
     print(f"64 rows, long contexts: max-abs logit error {err:.3e}; rows/step up to "
           f"{max(sum(s[4] for s in r['scheduled']) for r in trace)}")
+
+
+# ---- top-p (nucleus) sampling ------------------------------------------------------------------------
+def test_top_p_sampler_alone_bit_exact_on_oracle_logits():
+    """The nucleus sampler on given logits must pick the oracle's token, row for row: whole-vocabulary
+    nuclei of very different sizes (from one token to most of a 128256-entry row), nuclei cut from the
+    top-k candidates, rows made of one repeated value or a few values (thousands of exact ties, resolved
+    by index), and many draws on one row."""
+    rng = np.random.default_rng(9)
+    V, rows = 128256, 40
+    logits = (rng.normal(size=(rows, V)) * 1.3).astype(np.float32)
+    logits[0, :] = 0.25                                  # one value: the order is the index order
+    logits[1] = np.round(logits[1])                      # about ten distinct values, tens of thousands of ties each
+    logits[2, 777] = 40.0                                # one dominant token: the nucleus is that token
+    logits[3] = np.round(logits[3] * 4) / 4
+    top_k = np.array([0, 0, 0, 0] + [(0, 50, 0, 64, 7)[i % 5] for i in range(rows - 4)], dtype=np.int32)
+    top_p = np.array([0.9, 0.5, 0.9, 0.7] + [(0.9, 0.8, 0.3, 0.95, 0.5, 0.999, 0.05)[i % 7] for i in range(rows - 4)], dtype=np.float32)
+    temp = np.where(np.arange(rows) % 2 == 0, 0.8, 1.3).astype(np.float32)
+    ticket = np.arange(rows, dtype=np.uint64) * 613 + (1 << 34)
+    gen = (np.arange(rows) * 7 % 89).astype(np.int32)
+    seed = (np.arange(rows, dtype=np.uint64) * np.uint64(0x9E3779B97F4A7C15)) ^ np.uint64(0xB11C0009)
+    dev = torch.from_numpy(logits).cuda()
+    got = B.blink_sample_top_p(dev, top_k, temp, top_p, ticket, gen, seed)
+    for r in range(rows):
+        want = S.sample(logits[r], int(top_k[r]), float(temp[r]), int(ticket[r]), int(gen[r]), int(seed[r]), float(top_p[r]))
+        assert int(got[r]) == want, (r, int(got[r]), want, int(top_k[r]), float(top_p[r]))
+    # top_p outside (0, 1) switches the cut off: same tokens as the plain entry point
+    off = np.where(np.arange(rows) % 2 == 0, 0.0, 1.0).astype(np.float32)
+    assert np.array_equal(B.blink_sample_top_p(dev, top_k, temp, off, ticket, gen, seed),
+                          B.blink_sample(dev, top_k, temp, ticket, gen, seed))
+    # many draws on two rows (a continuous one and the all-equal one)
+    n = 120
+    for r, p in ((5, 0.9), (0, 0.6), (1, 0.8)):
+        rowdev = dev[r:r + 1].repeat(n, 1).contiguous()
+        g2 = B.blink_sample_top_p(rowdev, np.zeros(n, np.int32), np.full(n, 0.8, np.float32), np.full(n, p, np.float32),
+                                  np.full(n, 11, np.uint64), np.arange(n, dtype=np.int32), np.full(n, 4242, np.uint64))
+        idx, q = S.nucleus(logits[r], 0, 0.8, p)
+        qs, M = np.cumsum(np.array(q, dtype=object)), sum(q)
+        for i in range(n):
+            x24 = S.philox_word(11, i, 4242) >> 8
+            target = (x24 * M) >> 24
+            j = int(np.argmax(qs > target))
+            assert int(g2[i]) == int(idx[j]), (r, p, i)
+
+
+def test_top_p_sampling_end_to_end_fp32():
+    model, sched = model_cfg(1, dtype="fp32"), sched_cfg(1)
+    reqs = make_requests(1, n_requests=6)
+    for i, r in enumerate(reqs):
+        r.temperature, r.top_p = 0.8, (0.9, 0.6)[i % 2]
+        r.top_k = 0 if i < 4 else 20
+    w = make_weights(model, 6, "cpu")
+    err, n_margin, trace, toks, ora = _compare(model, sched, reqs, w, None, TOL_FP32)
+    agree = sum(toks[t][i] == ora["sampled"][t][i] for t in toks for i in range(len(toks[t])))
+    total = sum(len(v) for v in toks.values())
+    print(f"top-p end to end: {agree}/{total} tokens identical, {n_margin} decisions inside the margin")
+    assert total - agree <= n_margin
