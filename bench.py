@@ -34,6 +34,9 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
 
+POLICY = 0   # BLINK_POLICY_* used by every engine this run creates (--policy)
+
+
 def log(*a):
     print(*a, file=sys.stderr, flush=True)
 
@@ -258,7 +261,7 @@ def decode_point(B, m, sched, wbuf, kv, wl, gemm_impl, n, in_len, out_len, steps
     reqs = closed_batch(n, in_len, out_len, m.vocab, seed=7, top_k=50 if cfg_i >= 3 else 0, temperature=0.8)
     ramp = (n * in_len + sched.prefill_chunk_tokens - 1) // sched.prefill_chunk_tokens + 2
     eng = B.Blink(m, sched, wbuf, kv, exec_mode=B.EXEC_MANUAL, gemm_impl=gemm_impl, stats_iters=ramp + steps + 16,
-                  idle_exit_us=200_000, weights_layout=wl)
+                  idle_exit_us=200_000, weights_layout=wl, policy=POLICY)
     try:
         for r in reqs:
             eng.submit_request(r)
@@ -303,7 +306,7 @@ def realtime_run(B, m, sched, wbuf, kv, reqs, time_limit_s, use_arrivals=True, w
     """Persistent loop, requests submitted at their arrival times from host buffers, tokens
     read back with blink_poll.  Returns throughput and latency figures."""
     eng = B.Blink(m, sched, wbuf, kv, exec_mode=B.EXEC_PERSISTENT, stats_iters=1 << 17, idle_exit_us=2_000_000,
-                  weights_layout=weights_layout)
+                  weights_layout=weights_layout, policy=POLICY)
     try:
         off = eng.blink_get_stats().device_clock_offset_ns
         n_expected = 0
@@ -389,6 +392,8 @@ def main():
                     "rate; reports the highest rate whose goodput reaches 0.95 x offered")
     ap.add_argument("--rate-seconds", type=float, default=30.0, help="measurement window per rate of the sweep")
     ap.add_argument("--skip-parity", action="store_true")
+    ap.add_argument("--policy", default="chunked", choices=["chunked", "pause-resume"],
+                    help="chunked prefill (default), or the paper's whole-prompt prefill steps that pause decoding")
     ap.add_argument("--skip-cpu", action="store_true")
     ap.add_argument("--skip-e2e", action="store_true")
     ap.add_argument("--skip-latency", action="store_true")
@@ -414,6 +419,10 @@ def main():
     if args.layers > 0:
         m = m.with_(n_layers=args.layers)
     sched = sched_cfg(cfg_i)
+    if args.policy == "pause-resume":
+        global POLICY
+        POLICY = 1
+        sched = sched.with_(prefill_chunk_tokens=max(sched.prefill_chunk_tokens, sched.max_prompt))
     workload = f"C{cfg_i} {('8B' if cfg_i in (3, 4) else '')} stream".replace("  ", " ")
     if args.layers > 0:
         workload += f" ({args.layers} layers only)"
@@ -510,7 +519,7 @@ def main():
         # profiling aid: the same device code, one host launch per phase, so that a profiler sees
         # the phases as separate kernels (1 control launch + 9 per layer + 3 per iteration)
         eng = B.Blink(m, sched, wbuf, kv, exec_mode=B.EXEC_STEPPED, gemm_impl=gemm_impl, stats_iters=ramp + W + K + 64,
-                      weights_layout=wl)
+                      weights_layout=wl, policy=POLICY)
         try:
             for r in reqs:
                 eng.submit_request(r)
@@ -531,7 +540,7 @@ def main():
 
     # ---- closed-loop saturation run: ramp, W warm-up steps, then exactly K timed steps --------
     eng = B.Blink(m, sched, wbuf, kv, exec_mode=B.EXEC_MANUAL, gemm_impl=gemm_impl, stats_iters=ramp + W + K + 64,
-                  idle_exit_us=200_000, weights_layout=wl)
+                  idle_exit_us=200_000, weights_layout=wl, policy=POLICY)
     try:
         for r in reqs:
             eng.submit_request(r)
@@ -598,7 +607,7 @@ def main():
                             l2="per-step inputs (weights + KV) exceed L2 many times over; no flush needed",
                             rows_per_step=float(its["n_tokens"].mean()),
                             decode_rows_per_step=float(its["n_decode"].mean()),
-                            parallelism="replicas" if world > 1 else "1 GPU", gemm=args.gemm,
+                            parallelism="replicas" if world > 1 else "1 GPU", gemm=args.gemm, policy=args.policy,
                             weights_layout="streaming" if wl else "row-major"),
                 gpu_launches=1, clocks=clk, roofline=roof,
                 step_ms_device=dict(p50=float(np.median(step_dev_ms)), max=float(step_dev_ms.max())),

@@ -87,6 +87,17 @@ enum {
   BLINK_FUSION_ON = 2    /* in the GEMM epilogues: the CTA that completes an output tile consumes it      */
 };
 
+/* how prompts enter a running batch */
+enum {
+  BLINK_POLICY_CHUNKED = 0,      /* chunked prefill: every step carries all decode rows plus up to
+                                    prefill_chunk_tokens prompt tokens, in ticket order              */
+  BLINK_POLICY_PAUSE_RESUME = 1  /* the paper's inline prefill (Section 4.2 "Continuous batching with inline
+                                    prefill"): a step is either a decode step or a prefill step that runs the
+                                    whole prompts of the newly admitted requests (in ticket order, as many as
+                                    fit into prefill_chunk_tokens, which must be >= max_prompt) while the
+                                    decode requests are paused (slot state DECODE_PAUSED) for that one step */
+};
+
 /* why the device loop is not running (blink_stats.loop_state) */
 enum {
   BLINK_LOOP_NOT_STARTED = 0,
@@ -138,7 +149,7 @@ typedef struct blink_sched_cfg {
                                    receives the logits of the r-th sampled row since create      */
   int64_t logits_capture_rows;
   int32_t epilogue_fusion;      /* BLINK_FUSION_*                                               */
-  int32_t reserved0;
+  int32_t policy;               /* BLINK_POLICY_*                                               */
 } blink_sched_cfg;
 
 /* Caller-owned DEVICE memory for the paged KV cache.  The library derives

@@ -28,6 +28,19 @@ One iteration, given the watermark W (highest ticket visible to it):
                release the reservation and the batch slot.  Freed resources are
                usable from the next iteration.
 Iterations that schedule nothing are not counted.
+
+Second policy, "pause_resume": the paper's own inline prefill (Section 4.2, "Continuous
+batching with inline prefill").  A step is either a decode step (every DECODE request feeds one
+token) or a prefill step: the scheduler pauses the in-flight decode requests after the current
+step (their slots are DECODE_PAUSED meanwhile), runs the whole prompts of the newly admitted
+requests, merges them into the decode batch and resumes.  The paper's three conditions for
+pausing are (i) pending prefills, (ii) free batch-slot capacity, (iii) launch-window headroom
+for the prefill graph plus the resumed decode.  Here (i) and (ii) are the admission rule above;
+(iii) belongs to the device-side graph-launch window, which the fused loop does not have, and is
+always true.  Readings where the paper is silent: admitted prompts are taken whole, in ticket
+order, while their total stays within the step's token capacity (never smaller than the longest
+prompt, so the first always fits; nobody overtakes); a prefill step is followed by a decode step
+whenever a DECODE request exists, so generation is paused for one step at a time.
 """
 from __future__ import annotations
 
@@ -47,6 +60,9 @@ LEGAL_TRANSITIONS = {
     (DECODE_COMPLETED, EMPTY),
     # a request whose only new token is produced by its last prefill chunk
     (PREFILL_PROCESSING, DECODE_COMPLETED),
+    # pause-and-resume prefill: decode requests wait while new prompts are prefetched
+    (DECODE_PROCESSING, DECODE_PAUSED),
+    (DECODE_PAUSED, DECODE_PROCESSING),
 }
 
 
@@ -107,7 +123,10 @@ class Scheduler:
     (trace_record, items) or None when nothing could be scheduled."""
 
     def __init__(self, requests: Sequence[SimRequest], max_batch: int, chunk: int,
-                 n_blocks: int, block: int = 16):
+                 n_blocks: int, block: int = 16, policy: str = "chunked"):
+        assert policy in ("chunked", "pause_resume")
+        self.policy = policy
+        self.last_was_prefill = False
         self.req = {r.ticket: r for r in requests}
         self.MB, self.chunk, self.n_blocks, self.block = max_batch, chunk, n_blocks, block
         self.batch: list[Optional[_Entry]] = [None] * max_batch
@@ -140,18 +159,40 @@ class Scheduler:
         assert self._pending is None
         admitted = self._admit(W)
         take = {}
-        for b, e in enumerate(self.batch):
-            if e is not None and e.phase == DECODE:
+        decoding = [b for b, e in enumerate(self.batch) if e is not None and e.phase == DECODE]
+        prefilling = sorted((b for b, e in enumerate(self.batch) if e is not None and e.phase == PREFILL),
+                            key=lambda b: self.batch[b].ticket)
+        if self.policy == "chunked":
+            for b in decoding:
                 take[b] = 1
-        budget = self.chunk
-        for b in sorted((b for b, e in enumerate(self.batch) if e is not None and e.phase == PREFILL),
-                        key=lambda b: self.batch[b].ticket):
-            if budget == 0:
-                break
-            e = self.batch[b]
-            n = min(e.P - e.prefilled, budget)
-            take[b] = n
-            budget -= n
+            budget = self.chunk
+            for b in prefilling:
+                if budget == 0:
+                    break
+                e = self.batch[b]
+                n = min(e.P - e.prefilled, budget)
+                take[b] = n
+                budget -= n
+        else:
+            prefill_turn = bool(prefilling) and (not self.last_was_prefill or not decoding)
+            if prefill_turn:
+                room = self.chunk             # token capacity of a prefill step
+                for b in prefilling:
+                    e = self.batch[b]
+                    if e.P > room:
+                        break                 # whole prompts only, nobody overtakes
+                    take[b] = e.P
+                    room -= e.P
+                for b in decoding:
+                    if self.slot_state[self.batch[b].ticket] == DECODE_PROCESSING:
+                        self._move(self.batch[b].ticket, DECODE_PAUSED)
+            else:
+                for b in decoding:
+                    take[b] = 1
+                    if self.slot_state[self.batch[b].ticket] == DECODE_PAUSED:
+                        self._move(self.batch[b].ticket, DECODE_PROCESSING)
+            if take:
+                self.last_was_prefill = prefill_turn
         if not take:
             assert not admitted
             return None
@@ -229,12 +270,12 @@ class Scheduler:
 def simulate(requests: Sequence[SimRequest], max_batch: int, chunk: int, n_blocks: int,
              block: int = 16, watermarks: Optional[Sequence[int]] = None,
              sample_fn: Optional[Callable] = None, vocab: int = 1 << 30,
-             max_iters: int = 10_000_000, check: Optional[Callable] = None):
+             max_iters: int = 10_000_000, check: Optional[Callable] = None, policy: str = "chunked"):
     """Run to drain.  `watermarks[i]` is W of traced iteration i (default: all
     requests visible from the start).  `sample_fn(items) -> tokens for the sample
     rows in order` (default: the control-only fake sampler).
     Returns (trace, tokens_by_ticket)."""
-    sch = Scheduler(requests, max_batch, chunk, n_blocks, block)
+    sch = Scheduler(requests, max_batch, chunk, n_blocks, block, policy)
     last = max((r.ticket for r in requests), default=-1)
     trace, out = [], {r.ticket: [] for r in requests}
     while len(trace) < max_iters:

@@ -15,7 +15,7 @@ from . import transformer as O2
 
 
 def run(model_cfg, sched, weights: O2.Weights, requests, watermarks=None, act_round=None,
-        keep_logits=True, max_iters=10_000_000, forced=None):
+        keep_logits=True, max_iters=10_000_000, forced=None, policy="chunked"):
     """requests: objects with ticket, prompt, max_new, top_k, temperature, seed, eos_id (and top_p, optional).
     forced: optional {ticket: [tokens]}: teacher forcing, the given tokens are fed back instead of
     the sampled ones (the sampled ones are still what `sampled` reports).
@@ -47,5 +47,5 @@ def run(model_cfg, sched, weights: O2.Weights, requests, watermarks=None, act_ro
 
     trace, tokens, sch = O1.simulate(sim, sched.max_batch, sched.prefill_chunk_tokens,
                                      sched.n_blocks, sched.block_size, watermarks, sample_fn,
-                                     max_iters=max_iters)
+                                     max_iters=max_iters, policy=policy)
     return dict(trace=trace, tokens=tokens, sampled=sampled, logits=logs, scheduler=sch)

@@ -23,6 +23,7 @@ EXEC_PERSISTENT, EXEC_STEPPED, EXEC_MANUAL = 0, 1, 2
 GEMM_AUTO, GEMM_SIMT, GEMM_TC = 0, 1, 2
 WEIGHTS_ROW_MAJOR, WEIGHTS_STREAMING = 0, 1
 FUSION_AUTO, FUSION_OFF, FUSION_ON = 0, 1, 2
+POLICY_CHUNKED, POLICY_PAUSE_RESUME = 0, 1
 LOOP_NOT_STARTED, LOOP_RUNNING, LOOP_EXIT_STOP, LOOP_EXIT_BUDGET, LOOP_EXIT_IDLE, LOOP_EXIT_ERROR = range(6)
 TRACE_MAGIC = 0x424C4B31
 TRACE_HDR_WORDS = 12
@@ -43,7 +44,7 @@ class blink_sched_cfg(C.Structure):
                 ("wait_limit_ms", C.c_int32), ("iteration_budget", C.c_int64), ("idle_exit_us", C.c_int64),
                 ("trace_capacity_words", C.c_int64), ("stats_capacity_iters", C.c_int64),
                 ("logits_capture", C.c_void_p), ("logits_capture_rows", C.c_int64), ("epilogue_fusion", C.c_int32),
-                ("reserved0", C.c_int32)]
+                ("policy", C.c_int32)]
 
 
 class blink_kv_pool(C.Structure):
@@ -296,7 +297,7 @@ class Blink:
     def __init__(self, model, sched, weights=None, kv_pool=None, *, exec_mode=EXEC_PERSISTENT, gemm_impl=GEMM_AUTO,
                  control_only=False, start_paused=False, iteration_budget=0, idle_exit_us=0, trace_words=0,
                  stats_iters=0, logits_capture=None, kv_bytes=None, weights_layout=WEIGHTS_ROW_MAJOR, wait_limit_ms=0,
-                 epilogue_fusion=FUSION_AUTO):
+                 epilogue_fusion=FUSION_AUTO, policy=POLICY_CHUNKED):
         L = lib()
         self.model, self.sched = model, sched
         self._keep = (weights, kv_pool, logits_capture)
@@ -308,7 +309,7 @@ class Blink:
         sc = blink_sched_cfg(C.sizeof(blink_sched_cfg), sched.max_batch, sched.prefill_chunk_tokens, sched.n_slots,
                              sched.max_prompt, sched.max_new, exec_mode, gemm_impl, int(control_only),
                              int(start_paused), wait_limit_ms, iteration_budget, idle_exit_us, trace_words, stats_iters,
-                             cap_ptr, cap_rows, epilogue_fusion, 0)
+                             cap_ptr, cap_rows, epilogue_fusion, policy)
         if kv_pool is not None:
             kv = blink_kv_pool(C.sizeof(blink_kv_pool), sched.block_size, kv_pool.data_ptr(),
                                kv_pool.numel() * kv_pool.element_size())

@@ -529,6 +529,9 @@ int blink_create(const blink_model_cfg* model, const blink_sched_cfg* sched, con
     c.gemm_tc = tc_available() && tc_shape_ok(c);
   if (sched->gemm_impl == BLINK_GEMM_TC && !c.gemm_tc) { delete x; return BLINK_EINVAL; }
   // epilogue fusion needs whole 128-feature tiles that do not straddle q|k|v or gate|up
+  if (sched->policy != BLINK_POLICY_CHUNKED && sched->policy != BLINK_POLICY_PAUSE_RESUME) { delete x; return BLINK_EINVAL; }
+  if (sched->policy == BLINK_POLICY_PAUSE_RESUME && sched->prefill_chunk_tokens < sched->max_prompt) { delete x; return BLINK_EINVAL; }
+  c.policy = sched->policy;
   if (sched->epilogue_fusion < BLINK_FUSION_AUTO || sched->epilogue_fusion > BLINK_FUSION_ON) { delete x; return BLINK_EINVAL; }
   c.fused = sched->epilogue_fusion == BLINK_FUSION_ON && c.gemm_tc && c.qkv_dim % 128 == 0 && c.q_dim % 128 == 0 && c.kv_dim % 128 == 0 && c.F % 128 == 0 &&
             c.d % 128 == 0 && 128 % c.hd == 0;

@@ -8,6 +8,7 @@
 // "Continuous batching with inline prefill" (FCFS), "Ring buffer" (state machine,
 // fences order the externally visible updates).
 #pragma once
+#include "../../include/blink.h"
 #include "dev_ctx.cuh"
 
 namespace blink {
@@ -400,14 +401,30 @@ static __device__ int schedule_step(const DevCtx& c, unsigned long long visible)
   s_rem[tid] = (phase == PHASE_PREFILL) ? (P - prefilled) : 0;
   __syncthreads();
   int take = 0, start = 0;
-  if (phase == PHASE_DECODE) {
+  // prompt tokens already promised to earlier tickets in this iteration
+  long long before = 0;
+  if (phase == PHASE_PREFILL)
+    for (int j = 0; j < MB; ++j)
+      if (s_rem[j] > 0 && s_ticket[j] < ticket) before += s_rem[j];
+  bool prefill_turn = false;
+  if (c.policy == BLINK_POLICY_PAUSE_RESUME) {
+    // Section 4.2 "Continuous batching with inline prefill": a step is a decode step, or a prefill step
+    // for the whole prompts of the newly admitted requests while decoding is paused for this one step
+    const int has_pf = __syncthreads_or(phase == PHASE_PREFILL);
+    const int has_dec = __syncthreads_or(phase == PHASE_DECODE);
+    prefill_turn = has_pf && (!ss->last_was_prefill || !has_dec);
+    if (prefill_turn) {
+      if (phase == PHASE_PREFILL && before + P <= (long long)c.chunk) take = P;   // whole prompts, nobody overtakes
+      if (phase == PHASE_DECODE) c.slot_hot[slot].state = SLOT_DECODE_PAUSED;
+    } else if (phase == PHASE_DECODE) {
+      take = 1;
+      start = P + gen - 1;
+      c.slot_hot[slot].state = SLOT_DECODE_PROCESSING;
+    }
+  } else if (phase == PHASE_DECODE) {
     take = 1;
     start = P + gen - 1;
   } else if (phase == PHASE_PREFILL) {
-    // prompt tokens already promised to earlier tickets in this iteration
-    long long before = 0;
-    for (int j = 0; j < MB; ++j)
-      if (s_rem[j] > 0 && s_ticket[j] < ticket) before += s_rem[j];
     const long long left = (long long)c.chunk - before;
     take = (int)max(0ll, min((long long)(P - prefilled), left));
     start = prefilled;
@@ -543,6 +560,7 @@ static __device__ int schedule_step(const DevCtx& c, unsigned long long visible)
     ss->cur_kv = (long long)s_kv;
     ss->cur_t_begin = t_begin;
     ss->pending_post = 1;
+    ss->last_was_prefill = prefill_turn ? 1 : 0;
     if (c.dec_row != nullptr) {
       const long long TT = (long long)tot_kb * c.Hkv;
       // Sub-ranges: k per warp of the grid.  Every cut of a unit costs a partial record and a merge,

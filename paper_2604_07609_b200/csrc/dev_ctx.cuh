@@ -106,7 +106,7 @@ struct SchedState {
   unsigned long long bar_ctr;       // grid barrier: arrivals since the launch (the host zeroes it before a launch)
   unsigned long long cur_t_begin, cur_t_forward;
   int exit_reason;
-  int pad;
+  int last_was_prefill;             // pause-and-resume policy: the step before was a prefill step
   unsigned long long cur_phase_ns[N_PHASE_TIMERS];  // device time per phase kind of the open iteration
 };
 
@@ -136,6 +136,7 @@ struct DevCtx {
   // scheduler shape
   int MB, chunk, n_slots, max_prompt, max_new, Tmax, bs, n_blocks, max_blocks_seq, max_pos;
   int control_only, start_paused, stepped, gemm_tc;
+  int policy;        // BLINK_POLICY_*: chunked prefill, or whole-prompt prefill steps that pause decoding
   int n_warps_grid;  // warps of the whole grid (attention work split)
   int w_streaming;   // GEMM matrices are stored as contiguous pre-swizzled 128 x 64 tiles
   long long iteration_budget;

@@ -17,16 +17,20 @@ def sim_requests(reqs):
 
 
 def run_control_only(model, sched, reqs, *, exec_mode=B.EXEC_PERSISTENT, iteration_budget=0, trace_words=1 << 22,
-                     submit_all_first=True, step_iters=8):
+                     submit_all_first=True, step_iters=8, policy=B.POLICY_CHUNKED, trickle=0):
     """Control-only run (no model math).  Returns (parsed trace, tokens by ticket, stats)."""
     stepped = exec_mode == B.EXEC_STEPPED
     eng = B.Blink(model, sched, control_only=True, start_paused=True, exec_mode=exec_mode,
                   iteration_budget=iteration_budget, trace_words=trace_words, stats_iters=1 << 16,
-                  idle_exit_us=300_000)
+                  idle_exit_us=300_000, policy=policy)
     try:
-        for r in reqs:
+        import time
+        for r in reqs[:len(reqs) - trickle]:
             eng.submit_request(r)
         eng.blink_start()
+        for r in reqs[len(reqs) - trickle:]:      # the rest arrive while the loop runs (watermarks are logged)
+            time.sleep(0.0005)
+            eng.submit_request(r)
         total = sum(r.max_new for r in reqs)
         ev = eng.drain(total, timeout_s=120, step_iters=step_iters if stepped else 0)
         if stepped:
@@ -39,10 +43,10 @@ def run_control_only(model, sched, reqs, *, exec_mode=B.EXEC_PERSISTENT, iterati
         assert eng.blink_destroy() == B.BLINK_OK
 
 
-def oracle_control_trace(sched, reqs, trace_gpu, vocab):
+def oracle_control_trace(sched, reqs, trace_gpu, vocab, policy="chunked"):
     W = [r["W"] for r in trace_gpu]
     tr, toks, _ = O1.simulate(sim_requests(reqs), sched.max_batch, sched.prefill_chunk_tokens, sched.n_blocks,
-                              sched.block_size, watermarks=W, vocab=vocab)
+                              sched.block_size, watermarks=W, vocab=vocab, policy=policy)
     return tr, toks
 
 
@@ -62,7 +66,8 @@ def oracle_run(model, sched, reqs, weights_cpu, act_round, dtype=np.float64):
 
 
 def gpu_run_forced(model, sched, reqs, weights_cpu, forced, *, exec_mode=B.EXEC_PERSISTENT, gemm_impl=B.GEMM_AUTO,
-                   capture_rows=None, step_iters=4, iteration_budget=0, weights_layout=B.WEIGHTS_ROW_MAJOR):
+                   capture_rows=None, step_iters=4, iteration_budget=0, weights_layout=B.WEIGHTS_ROW_MAJOR,
+                   epilogue_fusion=B.FUSION_AUTO, policy=B.POLICY_CHUNKED):
     """Teacher-forced run: request t is fed forced[t] but reports its own samples.
     Returns (trace, sampled tokens by ticket, captured logits [rows, V] as numpy)."""
     dev = torch.device("cuda:0")
@@ -75,7 +80,8 @@ def gpu_run_forced(model, sched, reqs, weights_cpu, forced, *, exec_mode=B.EXEC_
     stepped = exec_mode == B.EXEC_STEPPED
     eng = B.Blink(model, sched, wd, kv, start_paused=True, exec_mode=exec_mode, gemm_impl=gemm_impl,
                   trace_words=1 << 22, stats_iters=1 << 14, logits_capture=cap, idle_exit_us=300_000,
-                  iteration_budget=iteration_budget, weights_layout=weights_layout)
+                  iteration_budget=iteration_budget, weights_layout=weights_layout, epilogue_fusion=epilogue_fusion,
+                  policy=policy)
     try:
         for r in reqs:
             eng.submit_request(r, forced_tokens=None if forced is None else forced[r.ticket])
@@ -184,7 +190,8 @@ def compare_with_oracle(model, sched, reqs, weights_cpu, tol, *, oracle_dtype=np
     the logit tolerance."""
     matched_round = O2.round_bf16 if model.dtype == "bf16" else None
     W = O2.Weights(model, weights_as_numpy(model, weights_cpu), dtype=oracle_dtype)
-    ora = OS.run(model, sched, W, reqs, act_round=matched_round)
+    opol = "pause_resume" if kw.get("policy", B.POLICY_CHUNKED) == B.POLICY_PAUSE_RESUME else "chunked"
+    ora = OS.run(model, sched, W, reqs, act_round=matched_round, policy=opol)
     trace, toks, logits, its = gpu_run_forced(model, sched, reqs, weights_cpu, ora["tokens"], **kw)
     assert_traces_equal([{**r, "sampled": []} for r in trace], [{**r, "sampled": []} for r in ora["trace"]])
     lo = np.stack([np.asarray(row, dtype=np.float32) for (_, _, _, _, row) in ora["logits"]])
@@ -204,7 +211,7 @@ def compare_with_oracle(model, sched, reqs, weights_cpu, tol, *, oracle_dtype=np
                logit_std=float(lo[: min(64, lo.shape[0])].std()), trace=trace, toks=toks, ora=ora, its=its, logits=logits)
     tol_eff = tol
     if matched_round is not None and (plain_too or noise_relative):
-        plain = OS.run(model, sched, W, reqs, act_round=None, forced=ora["tokens"])
+        plain = OS.run(model, sched, W, reqs, act_round=None, forced=ora["tokens"], policy=opol)
         lp = np.stack([np.asarray(row, dtype=np.float32) for (_, _, _, _, row) in plain["logits"]])
         (ep, ep_rms), (nm, n_rms) = dist(lg, lp), dist(lo, lp)
         out.update(err_plain=ep, err_plain_rms=ep_rms, noise_max=nm, noise_rms=n_rms)

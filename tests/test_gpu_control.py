@@ -201,3 +201,26 @@ def test_a_wait_that_runs_out_unwinds_the_loop_with_a_status():
     # the CUDA context is intact: a fresh loop on the same device works
     trace, toks, st2, _ = run_control_only(model_cfg(1), sched_cfg(1), make_requests(1))
     assert st2.device_status == 0 and len(toks) == 8
+
+
+def test_pause_resume_policy_trace_bit_exact():
+    """The paper's own inline prefill (whole prompts in prefill-only steps while decoding is paused for one
+    step): device trace equal to the oracle's under the same policy, with requests that arrive while the
+    loop is running (the logged watermarks are replayed)."""
+    model = model_cfg(1)
+    sched = sched_cfg(1, max_batch=6, prefill_chunk_tokens=160, n_blocks=128, max_prompt=64, max_new=32)
+    rng = np.random.default_rng(17)
+    reqs = [Request(t, 0.0, rng.integers(0, 4096, size=int(p)).astype(np.int32), int(n))
+            for t, (p, n) in enumerate(zip(rng.integers(5, 65, size=40), rng.integers(1, 33, size=40)))]
+    trace, toks, st, _ = run_control_only(model, sched, reqs, policy=B.POLICY_PAUSE_RESUME, trickle=30)
+    assert st.device_status == 0
+    tr_o, toks_o = oracle_control_trace(sched, reqs, trace, model.vocab, policy="pause_resume")
+    assert_traces_equal(trace, tr_o)
+    assert toks == toks_o
+    kinds = [{s[2] for s in r["scheduled"]} for r in trace]
+    assert all(len(k) == 1 for k in kinds) and {1} in kinds and {2} in kinds      # never a mixed step
+    assert all(s[3] == 0 and s[4] == reqs[s[1]].n_prompt for r in trace for s in r["scheduled"] if s[2] == 1)
+    assert st.free_blocks == sched.n_blocks and st.reserved_blocks == 0 and st.batch_live == 0
+    # a prefill budget below the longest accepted prompt cannot run whole prompts: refused at create
+    with pytest.raises(B.BlinkError):
+        B.Blink(model, sched_cfg(1, prefill_chunk_tokens=32, max_prompt=64), control_only=True, policy=B.POLICY_PAUSE_RESUME)

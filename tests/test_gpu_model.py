@@ -116,11 +116,13 @@ def test_sampler_alone_bit_exact_on_oracle_logits():
 
 
 # ---- tensor-core (tcgen05 / TMEM / TMA) path of the dense contractions ---------------------------
-def test_config1_bf16_tensor_core_path_matches_oracle():
+@pytest.mark.parametrize("fusion", [B.FUSION_OFF, B.FUSION_ON], ids=["separate-phases", "fused-epilogues"])
+def test_config1_bf16_tensor_core_path_matches_oracle(fusion):
     model, sched = model_cfg(1, dtype="bf16"), sched_cfg(1)
     reqs = make_requests(1)
     w = make_weights(model, 1234, "cpu")
-    err, n_margin, trace, toks, ora = _compare(model, sched, reqs, w, O2.round_bf16, TOL_BF16, gemm_impl=B.GEMM_TC)
+    err, n_margin, trace, toks, ora = _compare(model, sched, reqs, w, O2.round_bf16, TOL_BF16, gemm_impl=B.GEMM_TC,
+                                               epilogue_fusion=fusion)
     print(f"C1 bf16 tensor cores: max-abs logit error {err:.3e}, {n_margin} in-margin decisions")
     assert err <= TOL_BF16
 
@@ -135,7 +137,8 @@ def test_tensor_core_path_multi_pass_ragged_shapes():
     reqs = [Request(t, 0.0, rng.integers(0, model.vocab, size=int(p)).astype(np.int32), 6)
             for t, p in enumerate([310, 17, 301, 64, 129, 256, 5, 300, 33])]
     w = make_weights(model, 77, "cpu", random_gains=True)
-    err, n_margin, trace, toks, ora = _compare(model, sched, reqs, w, O2.round_bf16, TOL_BF16, gemm_impl=B.GEMM_TC)
+    err, n_margin, trace, toks, ora = _compare(model, sched, reqs, w, O2.round_bf16, TOL_BF16, gemm_impl=B.GEMM_TC,
+                                               epilogue_fusion=B.FUSION_ON)
     print(f"multi-pass tensor cores: max-abs logit error {err:.3e}; max rows/step "
           f"{max(sum(s[4] for s in r['scheduled']) for r in trace)}")
     assert err <= TOL_BF16
@@ -272,3 +275,17 @@ def test_top_p_sampling_end_to_end_fp32():
     total = sum(len(v) for v in toks.values())
     print(f"top-p end to end: {agree}/{total} tokens identical, {n_margin} decisions inside the margin")
     assert total - agree <= n_margin
+
+
+def test_pause_resume_policy_logits_and_tokens_fp32():
+    """Whole-prompt prefill steps of several requests at once, decode paused meanwhile: same model math."""
+    model = model_cfg(1, dtype="fp32")
+    sched = sched_cfg(1, max_batch=4, prefill_chunk_tokens=128, n_blocks=64)
+    reqs = make_requests(1, n_requests=7)
+    for r in reqs:
+        r.max_new = 9
+    w = make_weights(model, 8, "cpu", random_gains=True)
+    err, n_margin, trace, toks, ora = _compare(model, sched, reqs, w, None, TOL_FP32, policy=B.POLICY_PAUSE_RESUME)
+    print(f"pause-and-resume fp32: max-abs logit error {err:.3e}")
+    assert all(len({s[2] for s in r["scheduled"]}) == 1 for r in trace)
+    assert any(len(r["scheduled"]) > 1 and r["scheduled"][0][2] == 1 for r in trace)     # several prompts in one step

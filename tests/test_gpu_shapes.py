@@ -36,7 +36,8 @@ def _report(name, r):
     return rows, dec
 
 
-def test_8b_layer_shape_small_sample_topk():
+@pytest.mark.parametrize("fusion", [B.FUSION_OFF, B.FUSION_ON], ids=["separate-phases", "fused-epilogues"])
+def test_8b_layer_shape_small_sample_topk(fusion):
     """Four requests, prompts of at most 64 tokens, 16 new tokens each, top-k 50 at T 0.8: the sample
     the benchmark's CPU leg times, on four layers of the 8B shape (d 4096, 32/8 heads of 128, FFN
     14336, vocabulary 128256), streaming weight layout, tensor-core GEMMs."""
@@ -48,7 +49,7 @@ def test_8b_layer_shape_small_sample_topk():
         r.max_new = 16
     w = make_weights(model, 20260407, "cpu")
     r = compare_with_oracle(model, sched, reqs, w, TOL_BF16, oracle_dtype=np.float32, noise_relative=True, gemm_impl=B.GEMM_TC,
-                            weights_layout=B.WEIGHTS_STREAMING)
+                            weights_layout=B.WEIGHTS_STREAMING, epilogue_fusion=fusion)
     _report("8B layer shape, 4 requests", r)
 
 

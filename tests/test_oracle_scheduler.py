@@ -142,3 +142,104 @@ def test_config3_stream_trace_runs_at_full_scale():
     tr, toks, sch = O1.simulate(sim, 256, 512, 60000, 16, vocab=128256)
     assert sum(len(v) for v in toks.values()) == sum(r.max_new for r in reqs)
     assert sch.reserved == 0 and len(sch.stack) == 60000
+
+
+# ---- second policy: whole-prompt prefill with pause-and-resume (Section 4.2, "Continuous batching with
+# inline prefill") -------------------------------------------------------------------------------------
+def _pr(reqs, MB, cap, n_blocks, W=None, **kw):
+    return O1.simulate(reqs, MB, cap, n_blocks, 16, watermarks=W, vocab=4096, policy="pause_resume",
+                       check=O1.check_invariants, **kw)
+
+
+def test_pause_resume_single_request_closed_form():
+    for P, N in ((1, 1), (17, 5), (64, 32), (300, 2)):
+        tr, toks, sch = _pr([O1.SimRequest(0, P, N)], 4, 512, 64)
+        assert len(tr) == 1 + (N - 1)                                   # one whole-prompt step, then N - 1 decode steps
+        assert tr[0]["scheduled"] == [(0, 0, O1.PREFILL, 0, P)]
+        assert all(r["scheduled"] == [(0, 0, O1.DECODE, P + i, 1)] for i, r in enumerate(tr[1:]))
+        assert len(toks[0]) == N and sch.idle and sch.reserved == 0
+
+
+def test_pause_resume_steps_never_mix_phases_and_alternate():
+    rng = np.random.default_rng(4)
+    reqs = [O1.SimRequest(t, int(rng.integers(5, 120)), int(rng.integers(2, 30))) for t in range(24)]
+    # arrivals trickle in: request t becomes visible at iteration 2 t
+    W = [min(23, i // 2) for i in range(4000)]
+    tr, toks, sch = _pr(reqs, 6, 160, 200, W=W)
+    assert sch.idle and all(len(toks[r.ticket]) == r.N for r in reqs)
+    kinds = []
+    for rec in tr:
+        ph = {s[2] for s in rec["scheduled"]}
+        assert len(ph) == 1                                             # a step is a prefill step or a decode step
+        kinds.append(ph.pop())
+        if kinds[-1] == O1.PREFILL:
+            assert all(s[3] == 0 and s[4] == reqs[s[1]].P for s in rec["scheduled"])   # whole prompts
+            assert sum(s[4] for s in rec["scheduled"]) <= 160                          # within the step's capacity
+            tk = [s[1] for s in sorted(rec["scheduled"], key=lambda s: s[1])]
+            assert tk == list(range(tk[0], tk[0] + len(tk)))                           # consecutive tickets: nobody overtakes
+    assert sum(s[4] for rec in tr for s in rec["scheduled"] if s[2] == O1.PREFILL) == sum(r.P for r in reqs)
+    # generation is paused for one step at a time: two prefill steps in a row only while nothing decodes
+    live_decode = set()
+    for i, rec in enumerate(tr):
+        if i > 0 and kinds[i] == O1.PREFILL and kinds[i - 1] == O1.PREFILL:
+            assert not live_decode
+        for s in rec["scheduled"]:
+            if s[2] == O1.PREFILL and reqs[s[1]].N > 1:
+                live_decode.add(s[1])
+        for t in rec["finished"]:
+            live_decode.discard(t)
+    assert O1.PREFILL in kinds and O1.DECODE in kinds
+
+
+def test_pause_resume_matches_a_restatement_from_history():
+    """Every step is recomputed from the trace so far alone (no incremental state): which requests are
+    admitted, prefetched, decoding or finished, whether the step before was a prefill step, and hence
+    what this step must schedule."""
+    rng = np.random.default_rng(12)
+    for seed in range(4):
+        n = 14
+        reqs = [O1.SimRequest(t, int(rng.integers(3, 90)), int(rng.integers(1, 12))) for t in range(n)]
+        W = sorted(int(x) for x in rng.integers(0, n, size=3000))
+        MB, cap, nb = 4, 128, 40
+        tr, toks, _ = _pr(reqs, MB, cap, nb, W=W)
+        need = lambda r: O1.blocks_needed(r.P, r.N, 16)
+        for i, rec in enumerate(tr):
+            hist = tr[:i]
+            admitted = {t: b for h in hist for (t, b) in h["admitted"]}
+            finished = {t for h in hist for t in h["finished"]}
+            prefilled = {s[1] for h in hist for s in h["scheduled"] if s[2] == O1.PREFILL}
+            ngen = {t: sum(1 for h in hist for s in h["scheduled"] if s[1] == t) for t in admitted}
+            live = {t: b for t, b in admitted.items() if t not in finished}
+            reserved = sum(need(reqs[t]) for t in live)
+            occupied = set(live.values())
+            # admission
+            exp_adm, nxt = [], len(admitted)
+            while nxt < n and nxt <= W[i]:
+                free = [b for b in range(MB) if b not in occupied]
+                if not free or reserved + need(reqs[nxt]) > nb:
+                    break
+                exp_adm.append((nxt, free[0])); occupied.add(free[0]); live[nxt] = free[0]; reserved += need(reqs[nxt]); nxt += 1
+            assert rec["admitted"] == exp_adm
+            decoding = [t for t in live if t in prefilled]
+            waiting = sorted(t for t in live if t not in prefilled)
+            last_prefill = bool(hist) and hist[-1]["scheduled"][0][2] == O1.PREFILL
+            if waiting and (not last_prefill or not decoding):
+                exp, room = [], cap
+                for t in waiting:
+                    if reqs[t].P > room:
+                        break
+                    exp.append((live[t], t, O1.PREFILL, 0, reqs[t].P)); room -= reqs[t].P
+            else:
+                exp = [(live[t], t, O1.DECODE, reqs[t].P + ngen[t] - 1, 1) for t in decoding]
+            assert sorted(rec["scheduled"]) == sorted(exp), (seed, i)
+
+
+def test_pause_resume_slot_states_follow_the_paper_state_machine():
+    reqs = [O1.SimRequest(t, 20 + t, 6) for t in range(6)]
+    W = [0, 0, 0, 1, 1, 2, 2, 3, 4, 5] + [5] * 200
+    tr, toks, sch = _pr(reqs, 3, 64, 64, W=W)
+    assert all((a, b) in O1.LEGAL_TRANSITIONS for (_, a, b) in sch.transitions)
+    paused = [(t, a, b) for (t, a, b) in sch.transitions if b == O1.DECODE_PAUSED]
+    resumed = [(t, a, b) for (t, a, b) in sch.transitions if a == O1.DECODE_PAUSED]
+    assert paused and len(paused) == len(resumed)                       # every pause is followed by a resume
+    assert all(b == O1.DECODE_PROCESSING for (_, _, b) in resumed)
