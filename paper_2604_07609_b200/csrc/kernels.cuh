@@ -127,8 +127,13 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) blink_loop_kernel(const __grid
       const bool timed = c.stats_cap > 0 && blockIdx.x == 0 && threadIdx.x == 0;
       uint64_t t_prev = timed ? global_timer_ns() : 0;
       const int T = __ldcg(&c.ss->cur_T);   // fixed for the whole step: one L2 read instead of one per phase
-      auto step_phase = [&](int ph, int layer, int sub, bool barrier = true) {
+      auto step_phase = [&](int ph, int layer, int sub) {
         if (c.fused && (ph == PH_ROPE || ph == PH_SILU)) return;   // done by the epilogues of the QKV and gate/up GEMMs
+        // The experts' GEMMs are independent of one another (own weights, own gathered rows; the down
+        // projections add into the residual rows with reductions): one grid barrier after the last
+        // expert, none in between, so every CTA streams its share of all experts back to back.  (With
+        // fused epilogues the barriers stay: their tile counters are per GEMM.)
+        const bool barrier = !(c.E > 0 && !c.fused && (ph == PH_GU || ph == PH_DOWN) && sub + 1 < c.E);
         run_phase<WT, HD, NREP>(c, ph, layer, sub, smem, tc, as, T);
         if (!barrier) return;
         ok = grid_barrier(c, gen);
@@ -138,10 +143,7 @@ __global__ void __launch_bounds__(FWD_THREADS, 1) blink_loop_kernel(const __grid
         for (int ph = PH_NORM1; ph <= PH_DOWN && ok; ++ph) {
           if (c.E > 0 && (ph == PH_GU || ph == PH_DOWN)) {
             if (ph == PH_GU) step_phase(PH_MOE_GROUP, layer, 0);   // routing lists and gathered rows first
-            // The experts' GEMMs are independent of one another (own weights, own gathered rows; the
-            // down projections add into the residual rows with reductions): one grid barrier after the
-            // last expert, none in between, so every CTA streams its share of all experts back to back.
-            for (int e = 0; e < c.E && ok; ++e) step_phase(ph, layer, e, e + 1 == c.E || c.fused);   // (the tile counters of the fused epilogues are per GEMM)
+            for (int e = 0; e < c.E && ok; ++e) step_phase(ph, layer, e);
           } else {
             step_phase(ph, layer, 0);
           }
