@@ -207,8 +207,8 @@ typedef struct blink_stats {
   int32_t free_blocks, reserved_blocks, batch_live, reserved1;
   int64_t bytes_to_device;   /* bytes blink_submit wrote into the mapped submit areas (entries, prompts,
                                 forced tokens) since create                                          */
-  int64_t bytes_from_device; /* bytes blink_poll read from the device-written mirrors (count words it
-                                looked at, tokens and timestamps it handed out) since create         */
+  int64_t bytes_from_device; /* bytes the device wrote into the mapped host mirrors for the tokens blink_poll
+                                has handed out since create (token, timestamp and count word: 16 each) */
 } blink_stats;
 
 /* One record per traced iteration, for throughput / roofline arithmetic. */

@@ -772,7 +772,6 @@ int blink_poll(blink_ctx* x, blink_token_event* out, int max_events, int timeout
         const int slot = *it;
         SlotInfo& si = x->slots[slot];
         const uint32_t cnt = __atomic_load_n(&x->out_count[slot], __ATOMIC_ACQUIRE);
-        x->bytes_from_device += 4;
         const int have = (int)(cnt & 0x7fffffffu);
         const bool fin = (cnt >> 31) != 0;
         while (si.consumed < have && n < max_events) {
@@ -786,7 +785,7 @@ int blink_poll(blink_ctx* x, blink_token_event* out, int max_events, int timeout
           ev.t_host_ns = t_now;
           ev.t_submit_ns = si.t_submit_ns;
           si.consumed += 1;
-          x->bytes_from_device += 12;   // token + timestamp
+          x->bytes_from_device += 16;   // what the device wrote into the host mirrors for it: token, timestamp, count word
         }
         if (fin && si.consumed == have) {
           si.busy = false;  // DECODE_COMPLETED -> EMPTY: the frontend owns this transition
