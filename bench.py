@@ -36,6 +36,26 @@ sys.path.insert(0, ROOT)
 
 POLICY = 0   # BLINK_POLICY_* used by every engine this run creates (--policy)
 
+# DRAM traffic of one step (dram__bytes_read.sum + dram__bytes_write.sum over all phases), from the ncu
+# capture summarised in the named file under profiles/: the same device code launched phase by phase on a
+# 4-layer model of the same layer shape, per-layer phases averaged and scaled to the full layer count.
+# `algorithmic_gb` is the algorithmic figure (step_bytes_flops) of the captured step at the full layer
+# count; the bench scales the traffic to its own steps by the ratio of algorithmic bytes.  `digest` is
+# kernel_digest() at capture time: once the kernels change the figure is stale and is reported as null.
+TRAFFIC = {
+    "C3 8B stream": dict(traffic_gb=0.0, algorithmic_gb=0.0, digest="", source="profiles/dram_traffic_8B_stepped.md"),
+}
+
+
+def kernel_digest():
+    import hashlib
+    h = hashlib.sha256()
+    d = os.path.join(ROOT, "paper_2604_07609_b200", "csrc")
+    for f in sorted(os.listdir(d)):
+        if f.endswith((".cu", ".cuh", ".h")):
+            h.update(open(os.path.join(d, f), "rb").read())
+    return h.hexdigest()[:16]
+
 
 def log(*a):
     print(*a, file=sys.stderr, flush=True)
@@ -392,6 +412,7 @@ def main():
                     "rate; reports the highest rate whose goodput reaches 0.95 x offered")
     ap.add_argument("--rate-seconds", type=float, default=30.0, help="measurement window per rate of the sweep")
     ap.add_argument("--skip-parity", action="store_true")
+    ap.add_argument("--print-digest", action="store_true", help="print kernel_digest() and exit")
     ap.add_argument("--policy", default="chunked", choices=["chunked", "pause-resume"],
                     help="chunked prefill (default), or the paper's whole-prompt prefill steps that pause decoding")
     ap.add_argument("--skip-cpu", action="store_true")
@@ -408,6 +429,9 @@ def main():
                     help="stepped = one host launch per phase (profiling aid for ncu; prints no bench value)")
     args = ap.parse_args()
 
+    if args.print_digest:
+        print(kernel_digest())
+        return
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -543,7 +567,12 @@ def main():
             eng.blink_step(K)
             dt = time.perf_counter() - t0
             its = eng.blink_get_iter_stats()[-K:]
+            by_s, _ = step_bytes_flops(m, its)
+            by_full, _ = step_bytes_flops(model_cfg(cfg_i), its)
             print(json.dumps(dict(mode="stepped (profiling aid, not a bench value)", workload=workload, steps=K,
+                                  algorithmic_gb_per_step=float(by_s.mean() / 1e9),
+                                  algorithmic_gb_per_step_full_layer_count=float(by_full.mean() / 1e9),
+                                  kv_tokens_per_step=float(its["kv_tokens"].mean()), kernel_digest=kernel_digest(),
                                   wall_ms_per_step=dt * 1e3 / K, rows_per_step=float(its["n_tokens"].mean()),
                                   decode_rows_per_step=float(its["n_decode"].mean()),
                                   launches_per_step=1 + 9 * m.n_layers + 3)), flush=True)
@@ -601,7 +630,14 @@ def main():
         roof = dict(bound="tensor", achieved=float(fl.sum() / (ms / 1e3) / 1e12), peak=pk["tf_sustained"],
                     unit="TFLOP/s")
     roof["frac"] = roof["achieved"] / roof["peak"]
-    roof["traffic"] = None
+    tr = TRAFFIC.get(workload)
+    if tr and tr["digest"] == kernel_digest() and tr["algorithmic_gb"] > 0:
+        # bytes per launch (one launch = the K timed steps), like `achieved`
+        roof["traffic"] = float(tr["traffic_gb"] * 1e9 * (by.sum() / 1e9) / tr["algorithmic_gb"])
+        roof["traffic_over_algorithmic"] = tr["traffic_gb"] / tr["algorithmic_gb"]
+        roof["traffic_source"] = tr["source"]
+    else:
+        roof["traffic"] = None   # no capture for this workload, or the kernels changed since it was taken
     roof["peak_source"] = pk["source"]
     roof["kernel"] = "blink_loop_kernel (one launch = the K timed steps)"
     roof["algorithmic_gb_per_step"] = float(by.mean() / 1e9)
