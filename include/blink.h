@@ -77,7 +77,10 @@ enum {
 enum {
   BLINK_GEMM_AUTO = 0, /* tensor cores for bf16, CUDA cores for fp32 */
   BLINK_GEMM_SIMT = 1, /* CUDA-core reference kernels                */
-  BLINK_GEMM_TC = 2    /* tcgen05 / TMEM / TMA kernels (bf16 only)   */
+  BLINK_GEMM_TC = 2,   /* tcgen05 / TMEM / TMA kernels (bf16 only)   */
+  BLINK_GEMM_TC_PAIR = 3 /* the same on CTA pairs (tcgen05 cta_group::2, kernels launched with clusters of two): each
+                          CTA stages its own weight tile and half of the token tile.  bf16, four query heads per
+                          kv head, separate element-wise phases; BLINK_EINVAL otherwise */
 };
 
 /* where RoPE + KV write, SwiGLU and the norms' sums of squares run (tensor-core path only) */

@@ -169,6 +169,7 @@ struct blink_ctx {
   TcHost tc_host;
   KernelSet ks{nullptr, nullptr};
   bool manual = false;
+  bool pair = false;   // GEMMs on CTA pairs: kernels launched with clusters of two
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
 };
 
@@ -234,7 +235,18 @@ int launch_loop(blink_ctx* x) {
   const void* fn = x->ks.loop;
   // the grid barrier counts arrivals from zero in every launch
   if (cudaMemsetAsync(&x->dc.ss->bar_ctr, 0, sizeof(unsigned long long), x->stream) != cudaSuccess) return BLINK_ECUDA;
-  cudaError_t e = cudaLaunchCooperativeKernel(fn, dim3(x->grid), dim3(FWD_THREADS), args, x->smem_bytes, x->stream);
+  cudaError_t e;
+  if (x->pair) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(x->grid); cfg.blockDim = dim3(FWD_THREADS); cfg.dynamicSmemBytes = x->smem_bytes; cfg.stream = x->stream;
+    cudaLaunchAttribute at[2];
+    at[0].id = cudaLaunchAttributeClusterDimension; at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    at[1].id = cudaLaunchAttributeCooperative; at[1].val.cooperative = 1;
+    cfg.attrs = at; cfg.numAttrs = 2;
+    e = cudaLaunchKernelExC(&cfg, fn, args);
+  } else {
+    e = cudaLaunchCooperativeKernel(fn, dim3(x->grid), dim3(FWD_THREADS), args, x->smem_bytes, x->stream);
+  }
   if (e != cudaSuccess) {
     x->mbox->loop_state = BLINK_LOOP_EXIT_ERROR;
     fprintf(stderr, "blink: persistent launch failed: %s\n", cudaGetErrorString(e));
@@ -259,7 +271,16 @@ int pump(blink_ctx* x) {
 
 void launch_phase(blink_ctx* x, int phase, int layer, int sub = 0) {
   void* args[] = {(void*)&x->dc, (void*)&phase, (void*)&layer, (void*)&sub};
-  cudaLaunchKernel(x->ks.phase, dim3(x->grid), dim3(FWD_THREADS), args, x->smem_bytes, x->stream);
+  if (x->pair) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(x->grid); cfg.blockDim = dim3(FWD_THREADS); cfg.dynamicSmemBytes = x->smem_bytes; cfg.stream = x->stream;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension; at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    cudaLaunchKernelExC(&cfg, x->ks.phase, args);
+  } else {
+    cudaLaunchKernel(x->ks.phase, dim3(x->grid), dim3(FWD_THREADS), args, x->smem_bytes, x->stream);
+  }
   x->launches += 1;
 }
 
@@ -527,7 +548,11 @@ int blink_create(const blink_model_cfg* model, const blink_sched_cfg* sched, con
   c.gemm_tc = 0;
   if (!c.control_only && model->dtype == BLINK_DTYPE_BF16 && sched->gemm_impl != BLINK_GEMM_SIMT)
     c.gemm_tc = tc_available() && tc_shape_ok(c);
-  if (sched->gemm_impl == BLINK_GEMM_TC && !c.gemm_tc) { delete x; return BLINK_EINVAL; }
+  if ((sched->gemm_impl == BLINK_GEMM_TC || sched->gemm_impl == BLINK_GEMM_TC_PAIR) && !c.gemm_tc) { delete x; return BLINK_EINVAL; }
+  if (sched->gemm_impl < BLINK_GEMM_AUTO || sched->gemm_impl > BLINK_GEMM_TC_PAIR) { delete x; return BLINK_EINVAL; }
+  // CTA pairs: built for four query heads per kv head, need an even grid and separate element-wise phases
+  x->pair = sched->gemm_impl == BLINK_GEMM_TC_PAIR;
+  if (x->pair && (c.n_rep != 4 || (x->n_sms & 1) || sched->epilogue_fusion == BLINK_FUSION_ON)) { delete x; return BLINK_EINVAL; }
   // epilogue fusion needs whole 128-feature tiles that do not straddle q|k|v or gate|up
   if (sched->policy != BLINK_POLICY_CHUNKED && sched->policy != BLINK_POLICY_PAUSE_RESUME) { delete x; return BLINK_EINVAL; }
   if (sched->policy == BLINK_POLICY_PAUSE_RESUME && sched->prefill_chunk_tokens < sched->max_prompt) { delete x; return BLINK_EINVAL; }
@@ -676,8 +701,8 @@ int blink_create(const blink_model_cfg* model, const blink_sched_cfg* sched, con
 
   x->smem_bytes = phase_smem_bytes(x);
   x->grid = c.control_only ? 1 : x->n_sms;
-  x->ks = c.dtype == BLINK_DTYPE_BF16 ? (c.hd == 64 ? kernels_bf16_hd64(c.n_rep) : kernels_bf16_hd128(c.n_rep))
-                                      : (c.hd == 64 ? kernels_fp32_hd64(c.n_rep) : kernels_fp32_hd128(c.n_rep));
+  x->ks = c.dtype == BLINK_DTYPE_BF16 ? (c.hd == 64 ? kernels_bf16_hd64(c.n_rep, x->pair) : kernels_bf16_hd128(c.n_rep, x->pair))
+                                      : (c.hd == 64 ? kernels_fp32_hd64(c.n_rep, false) : kernels_fp32_hd128(c.n_rep, false));
   const void* loop_fn = x->ks.loop;
   const void* ph_fn = x->ks.phase;
   if (!loop_fn || !ph_fn) return fail(BLINK_EINVAL);
@@ -687,6 +712,15 @@ int blink_create(const blink_model_cfg* model, const blink_sched_cfg* sched, con
   int occ = 0;
   if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, loop_fn, FWD_THREADS, x->smem_bytes) != cudaSuccess || occ < 1)
     return fail(BLINK_ECUDA);
+  if (x->pair) {   // every cluster of two must be resident at once (the loop's grid barrier needs the whole grid)
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(x->grid); cfg.blockDim = dim3(FWD_THREADS); cfg.dynamicSmemBytes = x->smem_bytes;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension; at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    int ncl = 0;
+    if (cudaOccupancyMaxActiveClusters(&ncl, loop_fn, &cfg) != cudaSuccess || 2 * ncl < x->grid) return fail(BLINK_EINVAL);
+  }
   if (cudaDeviceSynchronize() != cudaSuccess) return fail(BLINK_ECUDA);
   if (!c.stepped && !x->manual) {
     rc = launch_loop(x);

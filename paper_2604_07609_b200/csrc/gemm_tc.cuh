@@ -198,6 +198,81 @@ __device__ __forceinline__ uint32_t idesc_bf16(int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 }
 
+// ---- CTA pairs (tcgen05 cta_group::2) ------------------------------------------------------------------
+// Two CTAs of a cluster work on one MMA of 256 weight rows: each stages its own 128-row weight tile and
+// half of the token tile (N / 2 rows), CTA 0 issues the MMAs, each CTA receives its 128 rows of the
+// result in its own TMEM.  Per k-block a CTA fills 16 KiB of weights + half a token tile instead of a
+// whole one.  No multicast loads: every CTA fetches its operands itself.
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// arrive (optionally announcing `bytes` of copies) on the barrier at the same shared-memory offset in CTA 0 of the pair
+__device__ __forceinline__ void mbar_expect_tx_cta0(uint64_t* bar, uint32_t bytes) {
+  asm volatile(
+      "{\n\t.reg .b32 ra;\n\t"
+      "mapa.shared::cluster.u32 ra, %0, 0;\n\t"
+      "mbarrier.arrive.expect_tx.shared::cluster.b64 _, [ra], %1;\n\t}" ::"r"(smem_u32(bar)),
+      "r"(bytes)
+      : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cta0(uint64_t* bar) {
+  asm volatile(
+      "{\n\t.reg .b32 ra;\n\t"
+      "mapa.shared::cluster.u32 ra, %0, 0;\n\t"
+      "mbarrier.arrive.shared::cluster.b64 _, [ra];\n\t}" ::"r"(smem_u32(bar))
+      : "memory");
+}
+// Tile copies of a pair: the bytes are counted on CTA 0's barrier (the CTA bit of the barrier's address is
+// cleared), whichever CTA of the pair issues the copy and receives the data.
+constexpr uint32_t PAIR_CTA0_MASK = 0xFEFFFFFFu;
+__device__ __forceinline__ void tma_pair_load_2d(void* smem_dst, const CUtensorMap* map, int x, int y, uint64_t* bar,
+                                                 uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+      "[%0], [%1, {%2, %3}], [%4], %5;" ::"r"(smem_u32(smem_dst)),
+      "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar) & PAIR_CTA0_MASK), "l"(policy)
+      : "memory");
+}
+__device__ __forceinline__ void tma_pair_load_3d(void* smem_dst, const CUtensorMap* map, int x, int y, int z, uint64_t* bar,
+                                                 uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+      "[%0], [%1, {%2, %3, %4}], [%5], %6;" ::"r"(smem_u32(smem_dst)),
+      "l"(map), "r"(x), "r"(y), "r"(z), "r"(smem_u32(bar) & PAIR_CTA0_MASK), "l"(policy)
+      : "memory");
+}
+__device__ __forceinline__ uint64_t l2_evict_normal() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+// D[tmem of both CTAs] (+)= A[smem of both CTAs] * B[smem of both CTAs]^T, M = 256 (128 per CTA), K = 16
+__device__ __forceinline__ void umma_bf16_pair(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
+                                               uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
+      "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// arrive on `bar` in both CTAs of the pair once all MMAs issued so far have completed
+__device__ __forceinline__ void umma_commit_pair(uint64_t* bar) {
+  asm volatile(
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(
+          smem_u32(bar)),
+      "h"((uint16_t)3)
+      : "memory");
+}
+__device__ __forceinline__ uint32_t idesc_bf16_pair(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+}
+
 // The same wait for warps that have nothing else to do for most of a phase: sleep between polls.
 __device__ __forceinline__ bool mbar_wait_idle(const DevCtx& c, uint64_t* bar, uint32_t parity, volatile int* dead) {
   if (*dead) return false;
@@ -215,40 +290,52 @@ __device__ __forceinline__ bool mbar_wait_idle(const DevCtx& c, uint64_t* bar, u
 }
 
 // ---- TMEM allocation for the life of the kernel ---------------------------------------------
+template <bool PAIR>
 __device__ __forceinline__ void tc_init(const DevCtx& c, float*, TcState& s) {
   s.tmem_base = 0;
   s.fill_bits = s.use_bits = s.acc_mma = s.acc_epi = s.last_bit = 0;
   if (!c.gemm_tc) return;
   if (threadIdx.x == 32) {
-    for (int i = 0; i < TC_MAX_STAGES; ++i) { mbar_init(&g_tc.full[i], 2); mbar_init(&g_tc.empty[i], 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(&g_tc.acc_full[b], 1); mbar_init(&g_tc.acc_empty[b], 4); }
+    // pairs: the operands of a stage come from four producers (two per CTA), counted on CTA 0's barrier;
+    // an accumulator is free again when the epilogue warps of both CTAs have drained it
+    for (int i = 0; i < TC_MAX_STAGES; ++i) { mbar_init(&g_tc.full[i], PAIR ? 4 : 2); mbar_init(&g_tc.empty[i], 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&g_tc.acc_full[b], 1); mbar_init(&g_tc.acc_empty[b], PAIR ? 8 : 4); }
     mbar_init(&g_tc.acc_last, 1);
     g_tc.dead = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (threadIdx.x < 32) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&g_tc.tmem))
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if constexpr (PAIR) {
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&g_tc.tmem)) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&g_tc.tmem)) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
   }
   tc_fence_before();
   __syncthreads();
+  if constexpr (PAIR) cluster_sync_all();   // both CTAs' barriers exist before either touches the other's
   tc_fence_after();
   s.tmem_base = *(volatile uint32_t*)&g_tc.tmem;
 }
+template <bool PAIR>
 __device__ __forceinline__ void tc_fini(const DevCtx& c, TcState& s) {
   if (!c.gemm_tc) return;
   tc_fence_before();
   __syncthreads();
+  if constexpr (PAIR) cluster_sync_all();   // the other CTA no longer signals into this one's shared memory
   if (threadIdx.x < 32) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(s.tmem_base) : "memory");
+    if constexpr (PAIR) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, 512;" ::"r"(s.tmem_base) : "memory");
+    else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(s.tmem_base) : "memory");
   }
 }
 
 struct TcMaps {
   CUtensorMap w[GEMM_KINDS];
   CUtensorMap act[ACT_BUFS][TC_BOXES];
+  CUtensorMap ws[GEMM_KINDS][2];   // streaming layout seen as [tiles][128][64]: box of one tile, of two consecutive tiles
 };
 
 // Where the epilogue's results go; held in registers by the warps that store (the arguments live
@@ -295,15 +382,15 @@ __device__ __forceinline__ int tc_epi_half(int n_mma) { return n_mma >= 128 ? ((
 // ---- the GEMM phase -----------------------------------------------------------------------------
 // Shape of one GEMM's pipeline for the current step; every role derives the same numbers.
 struct TcGeom {
-  int kblocks, ntiles, passes, box_id, box_rows, KPS, S;
+  int kblocks, ntiles, passes, box_id, box_rows, load_box, KPS, S;
   int pass_fixed, pdiv;   // one token pass per CTA (or -1), and the passes interleaved in its unit order
   uint32_t b_bytes, stage_bytes;
   long long u0, u1;
 };
-__device__ __forceinline__ TcGeom tc_geom(const DevCtx& c, int T, int N, int K, bool whole_tiles) {
+__device__ __forceinline__ TcGeom tc_geom(const DevCtx& c, int T, int N, int K, bool whole_tiles, int nb, int b, int ntiles, bool half_tokens) {
   TcGeom g;
   g.kblocks = K / 64;
-  g.ntiles = (N + 127) / 128;
+  g.ntiles = ntiles;   // weight tiles of 128 rows, or pairs of them
   g.passes = (T + 255) / 256;
   g.box_id = TC_BOXES - 1;
   if (g.passes == 1) {
@@ -314,28 +401,29 @@ __device__ __forceinline__ TcGeom tc_geom(const DevCtx& c, int T, int N, int K, 
   // A stage holds one k-block, or two when the token tile is small and the weights are stored as
   // contiguous tiles (then one bulk copy brings 32 KiB): fewer, larger copies per producer step.
   g.KPS = (c.w_streaming && g.box_rows <= 128) ? 2 : 1;
-  g.b_bytes = (uint32_t)g.box_rows * 128u;
+  // pairs: each CTA stages half of the token rows of a pass (the box that covers n_mma / 2 rows)
+  g.load_box = half_tokens ? (g.box_id > 0 ? g.box_id - 1 : 0) : g.box_id;
+  g.b_bytes = (uint32_t)(16 << g.load_box) * 128u;
   g.stage_bytes = (uint32_t)g.KPS * (TC_A_BYTES + g.b_bytes);
   g.S = TC_TILE_BUDGET / (int)g.stage_bytes;
   if (g.S > TC_MAX_STAGES) g.S = TC_MAX_STAGES;
   const long long total = (long long)g.passes * g.ntiles * g.kblocks;
-  g.u0 = total * blockIdx.x / gridDim.x;
-  g.u1 = total * (blockIdx.x + 1) / gridDim.x;
+  g.u0 = total * b / nb;
+  g.u1 = total * (b + 1) / nb;
   g.pass_fixed = -1;
   g.pdiv = g.passes;
   if (whole_tiles && g.passes == 1) {
-    // every CTA gets whole weight tiles (at most one more than its neighbours): no partial sums at all
-    g.u0 = (long long)g.kblocks * ((long long)g.ntiles * blockIdx.x / gridDim.x);
-    g.u1 = (long long)g.kblocks * ((long long)g.ntiles * (blockIdx.x + 1) / gridDim.x);
+    // every worker gets whole weight tiles (at most one more than its neighbours): no partial sums at all
+    g.u0 = (long long)g.kblocks * ((long long)g.ntiles * b / nb);
+    g.u1 = (long long)g.kblocks * ((long long)g.ntiles * (b + 1) / nb);
     return g;
   }
-  // More than 256 token rows: the passes of a weight tile go to neighbouring CTAs, which walk the
+  // More than 256 token rows: the passes of a weight tile go to neighbouring workers, which walk the
   // same (weight tile, k-block) range at the same time, so the tile comes from HBM once and from
-  // L2 for the others.  One CTA doing the passes in turn re-reads it after the whole grid has
+  // L2 for the others.  One worker doing the passes in turn re-reads it after the whole grid has
   // streamed more than L2 holds in between.
-  if (g.passes > 1 && (int)gridDim.x >= g.passes) {
-    const int groups = (int)gridDim.x / g.passes;
-    const int b = (int)blockIdx.x;
+  if (g.passes > 1 && nb >= g.passes) {
+    const int groups = nb / g.passes;
     const long long units = (long long)g.ntiles * g.kblocks;
     g.pdiv = 1;
     if (b < groups * g.passes) {
@@ -349,14 +437,13 @@ __device__ __forceinline__ TcGeom tc_geom(const DevCtx& c, int T, int N, int K, 
     }
   }
   // Few weight tiles (QKV, O, down at decode sizes): give every tile the same whole number of
-  // CTAs, so that no CTA's range crosses a tile and each has one partial tile to reduce at the
-  // end instead of two.  The longest range grows by (per * grid - total) / grid k-blocks of about
+  // workers, so that no range crosses a tile and each has one partial tile to reduce at the
+  // end instead of two.  The longest range grows by (per * nb - total) / nb k-blocks of about
   // 0.4 us each; the saved reduction takes about 0.018 us per token row.
-  const int split = (int)gridDim.x / g.ntiles;
+  const int split = nb / g.ntiles;
   if (g.passes == 1 && split >= 2) {
     const int per = (g.kblocks + split - 1) / split;
-    if (((long long)per * gridDim.x - total) * 23 < (long long)T * gridDim.x) {
-      const int b = (int)blockIdx.x;
+    if (((long long)per * nb - total) * 23 < (long long)T * nb) {
       if (b < g.ntiles * split) {
         const int nt = b / split, part = b % split;
         g.u0 = (long long)nt * g.kblocks + (long long)g.kblocks * part / split;
@@ -379,9 +466,14 @@ __device__ __forceinline__ char* tc_tiles(float* smem_f) {
   return reinterpret_cast<char*>(smem_f) + (((raw + 1023u) & ~1023u) - raw);
 }
 
+// In pair mode a unit names a PAIR of weight tiles (2 nt, 2 nt + 1): CTA r of the pair owns tile 2 nt + r.
+template <bool PAIR>
+__device__ __forceinline__ int tc_my_tile(int nt_unit, uint32_t rank) { return PAIR ? 2 * nt_unit + (int)rank : nt_unit; }
+
 // Weight producer (one thread): stream the weight tiles of this CTA's range through the ring.
+template <bool PAIR>
 __device__ __forceinline__ void tc_produce_weights(const DevCtx& c, const void* w, long long w_row0, int which,
-                                                   const TcGeom& g, char* tiles, TcState& tc) {
+                                                   const TcGeom& g, char* tiles, TcState& tc, uint32_t rank) {
   const TcMaps* maps = reinterpret_cast<const TcMaps*>(c.tc_maps);
   const CUtensorMap* map_a = &maps->w[which];
   const int row_a0 = (int)w_row0;
@@ -393,17 +485,27 @@ __device__ __forceinline__ void tc_produce_weights(const DevCtx& c, const void* 
     const long long seg_end = min(g.u1, (u / g.kblocks + 1) * (long long)g.kblocks);
     const int nk = (int)min((long long)g.KPS, seg_end - u);
     const int kb = (int)(u % g.kblocks);
-    const int nt = tc_unit_nt(g, u);
+    const int nt = tc_my_tile<PAIR>(tc_unit_nt(g, u), rank);
     // the n-th fill of a stage waits for its (n-1)-th release
     if (!mbar_wait(c, &g_tc.empty[stage], ((tc.fill_bits >> stage) & 1u) ^ 1u, dead)) break;
     tc.fill_bits ^= 1u << stage;
     char* sa = tiles + (size_t)stage * g.stage_bytes;
-    mbar_expect_tx(&g_tc.full[stage], (uint32_t)nk * TC_A_BYTES);
-    if (c.w_streaming) {  // contiguous tiles, already in the shared-memory operand image
-      tma_bulk_load_hint(sa, reinterpret_cast<const char*>(w) + ((size_t)nt * g.kblocks + kb) * TC_A_BYTES,
-                         (uint32_t)nk * TC_A_BYTES, &g_tc.full[stage], stream_policy);
+    if constexpr (PAIR) {
+      mbar_expect_tx_cta0(&g_tc.full[stage], (uint32_t)nk * TC_A_BYTES);
+      if (c.w_streaming) {   // tile index inside the whole tensor; one or two consecutive tiles per copy
+        const int tile = (int)(((w_row0 >> 7) + nt) * g.kblocks + kb);
+        tma_pair_load_3d(sa, &maps->ws[which][nk - 1], 0, 0, tile, &g_tc.full[stage], stream_policy);
+      } else {
+        tma_pair_load_2d(sa, map_a, kb * 64, row_a0 + nt * 128, &g_tc.full[stage], stream_policy);
+      }
     } else {
-      tma_load_2d_hint(sa, map_a, kb * 64, row_a0 + nt * 128, &g_tc.full[stage], stream_policy);
+      mbar_expect_tx(&g_tc.full[stage], (uint32_t)nk * TC_A_BYTES);
+      if (c.w_streaming) {  // contiguous tiles, already in the shared-memory operand image
+        tma_bulk_load_hint(sa, reinterpret_cast<const char*>(w) + ((size_t)nt * g.kblocks + kb) * TC_A_BYTES,
+                           (uint32_t)nk * TC_A_BYTES, &g_tc.full[stage], stream_policy);
+      } else {
+        tma_load_2d_hint(sa, map_a, kb * 64, row_a0 + nt * 128, &g_tc.full[stage], stream_policy);
+      }
     }
     u += nk;
     if (++stage == g.S) stage = 0;
@@ -458,16 +560,23 @@ static __device__ __noinline__ void tc_finish_tiles(const DevCtx& c, const GemmA
   }
 }
 
+template <bool PAIR>
 static __device__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int which, int layer, float* smem_f, TcState& tc) {
   const int T = a.M, N = a.N, K = a.K;
   if (T <= 0) return;  // uniform over the grid
   const TcMaps* maps = reinterpret_cast<const TcMaps*>(c.tc_maps);
-  const TcGeom g = tc_geom(c, T, N, K, which == GEMM_LMHEAD && lm_head_whole_tiles(c));
-  const int kblocks = g.kblocks, ntiles = g.ntiles, KPS = g.KPS, S = g.S;
+  const uint32_t rank = PAIR ? cluster_ctarank() : 0u;
+  const int n_tiles128 = (N + 127) / 128;
+  // workers are CTAs, or CTA pairs that take two weight tiles at a time
+  const TcGeom g = PAIR ? tc_geom(c, T, N, K, which == GEMM_LMHEAD && lm_head_whole_tiles(c), (int)gridDim.x / 2,
+                                  (int)blockIdx.x / 2, (n_tiles128 + 1) / 2, true)
+                        : tc_geom(c, T, N, K, which == GEMM_LMHEAD && lm_head_whole_tiles(c), (int)gridDim.x, (int)blockIdx.x,
+                                  n_tiles128, false);
+  const int kblocks = g.kblocks, KPS = g.KPS, S = g.S;
   const uint32_t b_bytes = g.b_bytes, stage_bytes = g.stage_bytes;
   const int act_id = which == GEMM_O ? ACT_ATTN : which == GEMM_DOWN ? ACT_ACT : which == GEMM_LMHEAD ? ACT_XS
                      : (which == GEMM_GU && c.E > 0) ? ACT_XG : ACT_XN;
-  const CUtensorMap* map_b = &maps->act[act_id][g.box_id];
+  const CUtensorMap* map_b = &maps->act[act_id][g.load_box];
   char* tiles = tc_tiles(smem_f);
   const long long u0 = g.u0, u1 = g.u1;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -475,12 +584,13 @@ static __device__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int whi
 
   if (warp == 0) {
     if (lane == 0) {
-      tc_produce_weights(c, a.w, a.w_row0, which, g, tiles, tc);
+      tc_produce_weights<PAIR>(c, a.w, a.w_row0, which, g, tiles, tc, rank);
     }
   } else if (warp == 2) {
     // token-tile producer: walks the same sequence of stages (nk k-blocks of one segment each)
     if (lane == 0) {
       const int x_row0 = a.x_row0;
+      const uint64_t keep_policy = l2_evict_normal();
       int stage = 0;
       long long u = u0;
       while (u < u1) {
@@ -491,15 +601,24 @@ static __device__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int whi
         if (!mbar_wait(c, &g_tc.empty[stage], ((tc.fill_bits >> stage) & 1u) ^ 1u, dead)) break;
         tc.fill_bits ^= 1u << stage;
         char* sa = tiles + (size_t)stage * stage_bytes;
-        mbar_expect_tx(&g_tc.full[stage], (uint32_t)nk * b_bytes);
-        for (int j = 0; j < nk; ++j)
-          tma_load_2d(sa + KPS * TC_A_BYTES + j * b_bytes, map_b, (kb + j) * 64, x_row0 + pass * 256, &g_tc.full[stage]);
+        if constexpr (PAIR) {
+          // this CTA's half of the pass: rows [rank * n_mma / 2, + n_mma / 2) (the box may reach further)
+          const int n_mma = (min(256, T - pass * 256) + 15) & ~15;
+          const int row0 = x_row0 + pass * 256 + (int)rank * (n_mma / 2);
+          mbar_expect_tx_cta0(&g_tc.full[stage], (uint32_t)nk * b_bytes);
+          for (int j = 0; j < nk; ++j)
+            tma_pair_load_2d(sa + KPS * TC_A_BYTES + j * b_bytes, map_b, (kb + j) * 64, row0, &g_tc.full[stage], keep_policy);
+        } else {
+          mbar_expect_tx(&g_tc.full[stage], (uint32_t)nk * b_bytes);
+          for (int j = 0; j < nk; ++j)
+            tma_load_2d(sa + KPS * TC_A_BYTES + j * b_bytes, map_b, (kb + j) * 64, x_row0 + pass * 256, &g_tc.full[stage]);
+        }
         u += nk;
         if (++stage == S) stage = 0;
       }
     }
   } else if (warp == 1) {
-    if (lane == 0) {
+    if (lane == 0 && rank == 0) {   // pairs: CTA 0 issues the MMAs for both
       int stage = 0;
       int abuf = 0;
       long long u = u0;
@@ -508,7 +627,7 @@ static __device__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int whi
         const int pass = tc_unit_pass(g, u);
         const int rows = min(256, T - pass * 256);
         const int n_mma = (rows + 15) & ~15;
-        const uint32_t idesc = idesc_bf16(n_mma);
+        const uint32_t idesc = PAIR ? idesc_bf16_pair(n_mma) : idesc_bf16(n_mma);
         const uint32_t d_tmem = tc.tmem_base + (uint32_t)abuf * 256u;
         if (!mbar_wait(c, &g_tc.acc_empty[abuf], ((tc.acc_mma >> abuf) & 1u) ^ 1u, dead)) break;
         tc.acc_mma ^= 1u << abuf;
@@ -527,21 +646,28 @@ static __device__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int whi
 #pragma unroll
             for (int k16 = 0; k16 < 4; ++k16) {
               // 16 bf16 = 32 bytes further along K inside the swizzle atom: +2 in 16-byte units
-              umma_bf16(d_tmem, da + (uint64_t)(2 * k16), db + (uint64_t)(2 * k16), idesc, (first && k16 == 0) ? 0u : 1u);
+              if constexpr (PAIR) umma_bf16_pair(d_tmem, da + (uint64_t)(2 * k16), db + (uint64_t)(2 * k16), idesc, (first && k16 == 0) ? 0u : 1u);
+              else umma_bf16(d_tmem, da + (uint64_t)(2 * k16), db + (uint64_t)(2 * k16), idesc, (first && k16 == 0) ? 0u : 1u);
             }
             first = false;
           }
-          umma_commit(&g_tc.empty[stage]);
+          if constexpr (PAIR) umma_commit_pair(&g_tc.empty[stage]);
+          else umma_commit(&g_tc.empty[stage]);
           u += nk;
           if (++stage == S) stage = 0;
         }
         if (!ok) break;
-        umma_commit(&g_tc.acc_full[abuf]);
         // Warps 0-3 take part of the CTA's last accumulator.  They cannot wait on acc_full: a parity
         // wait tells two consecutive completions apart, not the first use of a buffer in this phase
         // from its third, and they arrive here long before the epilogue warps.  A barrier of their own
         // that completes exactly once per phase has no such ambiguity.
-        if (u == u1) umma_commit(&g_tc.acc_last);
+        if constexpr (PAIR) {
+          umma_commit_pair(&g_tc.acc_full[abuf]);
+          if (u == u1) umma_commit_pair(&g_tc.acc_last);
+        } else {
+          umma_commit(&g_tc.acc_full[abuf]);
+          if (u == u1) umma_commit(&g_tc.acc_last);
+        }
         abuf ^= 1;
       }
     }
@@ -555,7 +681,7 @@ static __device__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int whi
       const long long seg_end = min(u1, (u / kblocks + 1) * (long long)kblocks);
       const int kb0 = (int)(u % kblocks);
       const int kb1 = kb0 + (int)(seg_end - u);
-      const int nt = tc_unit_nt(g, u);
+      const int nt = tc_my_tile<PAIR>(tc_unit_nt(g, u), rank);
       const int pass = tc_unit_pass(g, u);
       const int rows = min(256, T - pass * 256);
       const int n_mma = (rows + 15) & ~15;
@@ -569,7 +695,10 @@ static __device__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int whi
       tc_epi_columns(eo, taddr, nt * 128 + q * 32 + lane, pass * 256, 0, c_end, plain);
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&g_tc.acc_empty[abuf]);
+      if (lane == 0) {
+        if constexpr (PAIR) mbar_arrive_cta0(&g_tc.acc_empty[abuf]);   // the MMA issuer sits in CTA 0
+        else mbar_arrive(&g_tc.acc_empty[abuf]);
+      }
       abuf ^= 1;
       u = seg_end;
     }
@@ -589,7 +718,7 @@ static __device__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int whi
         if (u < u1) last_abuf ^= 1;
       }
       const int kb0 = (int)(last_u % kblocks);
-      const int nt = tc_unit_nt(g, last_u);
+      const int nt = tc_my_tile<PAIR>(tc_unit_nt(g, last_u), rank);
       const int pass = tc_unit_pass(g, last_u);
       const int n_mma = (min(256, T - pass * 256) + 15) & ~15;
       const int c_begin = tc_epi_half(n_mma);
@@ -605,7 +734,9 @@ static __device__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int whi
     }
   }
   __syncthreads();
-  if (a.fix != FIX_NONE) tc_finish_tiles(c, a, g, layer);
+  if constexpr (!PAIR) {
+    if (a.fix != FIX_NONE) tc_finish_tiles(c, a, g, layer);
+  }
 }
 
 // ---- host side: tensor maps ----------------------------------------------------------------
@@ -661,6 +792,23 @@ inline int tc_host_setup(TcHost& h, DevCtx& c) {
   ok &= tc_make_map(enc, &hm->w[GEMM_GU], w + c.w_off[3], L * E1 * 2 * c.F, c.d, 128, true);
   ok &= tc_make_map(enc, &hm->w[GEMM_DOWN], w + c.w_off[4], L * E1 * c.d, c.F, 128, true);
   ok &= tc_make_map(enc, &hm->w[GEMM_LMHEAD], w + c.w_off[9], c.V, c.d, 128, true);
+  if (c.w_streaming) {
+    // the streaming layout as a rank-3 tensor [tiles][128 rows][64 columns] of verbatim 16 KiB tile images
+    // (no swizzle: the image is already the operand image), boxes of one and of two consecutive tiles
+    const uint64_t rows_tot[GEMM_KINDS] = {L * c.qkv_dim, L * c.d, L * E1 * 2 * c.F, L * E1 * c.d, (uint64_t)c.V};
+    const uint64_t cols_k[GEMM_KINDS] = {(uint64_t)c.d, (uint64_t)c.q_dim, (uint64_t)c.d, (uint64_t)c.F, (uint64_t)c.d};
+    const int ids[GEMM_KINDS] = {1, 2, 3, 4, 9};
+    for (int k = 0; k < GEMM_KINDS; ++k)
+      for (int two = 0; two < 2; ++two) {
+        cuuint64_t dims[3] = {64, 128, rows_tot[k] / 128 * (cols_k[k] / 64)};
+        cuuint64_t strides[2] = {128, 16384};
+        cuuint32_t box[3] = {64, 128, (cuuint32_t)(two + 1)};
+        cuuint32_t estr[3] = {1, 1, 1};
+        ok &= enc(&hm->ws[k][two], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<char*>(w + c.w_off[ids[k]]), dims, strides, box,
+                  estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+      }
+  }
   const void* bufs[ACT_BUFS] = {c.xn, c.attn, c.act, c.xs, c.xg ? c.xg : c.xn};
   const uint64_t RA = (uint64_t)c.Tmax * (c.E > 0 ? c.topE : 1);   // routed experts: one row per (token, expert)
   const uint64_t rows[ACT_BUFS] = {(uint64_t)c.Tmax, (uint64_t)c.Tmax, RA, (uint64_t)c.MB, c.xg ? RA : (uint64_t)c.Tmax};

@@ -13,8 +13,8 @@ struct KernelSet {
   const void* loop;   // persistent cooperative loop: (DevCtx)
   const void* phase;  // one phase of one layer: (DevCtx, int phase, int layer, int expert)
 };
-KernelSet kernels_bf16_hd64(int n_rep);
-KernelSet kernels_bf16_hd128(int n_rep);
-KernelSet kernels_fp32_hd64(int n_rep);
-KernelSet kernels_fp32_hd128(int n_rep);
+KernelSet kernels_bf16_hd64(int n_rep, bool pair);
+KernelSet kernels_bf16_hd128(int n_rep, bool pair);
+KernelSet kernels_fp32_hd64(int n_rep, bool pair);
+KernelSet kernels_fp32_hd128(int n_rep, bool pair);
 }  // namespace blink
