@@ -551,8 +551,9 @@ int blink_create(const blink_model_cfg* model, const blink_sched_cfg* sched, con
   if ((sched->gemm_impl == BLINK_GEMM_TC || sched->gemm_impl == BLINK_GEMM_TC_PAIR) && !c.gemm_tc) { delete x; return BLINK_EINVAL; }
   if (sched->gemm_impl < BLINK_GEMM_AUTO || sched->gemm_impl > BLINK_GEMM_TC_PAIR) { delete x; return BLINK_EINVAL; }
   // CTA pairs: built for four query heads per kv head, need an even grid and separate element-wise phases
-  x->pair = sched->gemm_impl == BLINK_GEMM_TC_PAIR;
-  if (x->pair && (c.n_rep != 4 || (x->n_sms & 1) || sched->epilogue_fusion == BLINK_FUSION_ON)) { delete x; return BLINK_EINVAL; }
+  const bool pair_ok = c.gemm_tc && c.n_rep == 4 && !(x->n_sms & 1) && sched->epilogue_fusion != BLINK_FUSION_ON;
+  if (sched->gemm_impl == BLINK_GEMM_TC_PAIR && !pair_ok) { delete x; return BLINK_EINVAL; }
+  x->pair = pair_ok && (sched->gemm_impl == BLINK_GEMM_TC_PAIR || sched->gemm_impl == BLINK_GEMM_AUTO);   // measured faster
   // epilogue fusion needs whole 128-feature tiles that do not straddle q|k|v or gate|up
   if (sched->policy != BLINK_POLICY_CHUNKED && sched->policy != BLINK_POLICY_PAUSE_RESUME) { delete x; return BLINK_EINVAL; }
   if (sched->policy == BLINK_POLICY_PAUSE_RESUME && sched->prefill_chunk_tokens < sched->max_prompt) { delete x; return BLINK_EINVAL; }
@@ -701,8 +702,29 @@ int blink_create(const blink_model_cfg* model, const blink_sched_cfg* sched, con
 
   x->smem_bytes = phase_smem_bytes(x);
   x->grid = c.control_only ? 1 : x->n_sms;
-  x->ks = c.dtype == BLINK_DTYPE_BF16 ? (c.hd == 64 ? kernels_bf16_hd64(c.n_rep, x->pair) : kernels_bf16_hd128(c.n_rep, x->pair))
-                                      : (c.hd == 64 ? kernels_fp32_hd64(c.n_rep, false) : kernels_fp32_hd128(c.n_rep, false));
+  auto pick_kernels = [&]() {
+    x->ks = c.dtype == BLINK_DTYPE_BF16 ? (c.hd == 64 ? kernels_bf16_hd64(c.n_rep, x->pair) : kernels_bf16_hd128(c.n_rep, x->pair))
+                                        : (c.hd == 64 ? kernels_fp32_hd64(c.n_rep, false) : kernels_fp32_hd128(c.n_rep, false));
+  };
+  pick_kernels();
+  if (x->pair) {   // every cluster of two must be resident at once (the loop's grid barrier needs the whole grid)
+    bool fits = x->ks.loop != nullptr;
+    if (fits) {
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3(x->grid); cfg.blockDim = dim3(FWD_THREADS); cfg.dynamicSmemBytes = x->smem_bytes;
+      cudaLaunchAttribute at[1];
+      at[0].id = cudaLaunchAttributeClusterDimension; at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+      cfg.attrs = at; cfg.numAttrs = 1;
+      int ncl = 0;
+      fits = cudaFuncSetAttribute(x->ks.loop, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)x->smem_bytes) == cudaSuccess &&
+             cudaOccupancyMaxActiveClusters(&ncl, x->ks.loop, &cfg) == cudaSuccess && 2 * ncl >= x->grid;
+    }
+    if (!fits) {
+      if (sched->gemm_impl == BLINK_GEMM_TC_PAIR) return fail(BLINK_EINVAL);
+      x->pair = false;   // chosen automatically: fall back to single CTAs
+      pick_kernels();
+    }
+  }
   const void* loop_fn = x->ks.loop;
   const void* ph_fn = x->ks.phase;
   if (!loop_fn || !ph_fn) return fail(BLINK_EINVAL);
@@ -712,15 +734,6 @@ int blink_create(const blink_model_cfg* model, const blink_sched_cfg* sched, con
   int occ = 0;
   if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, loop_fn, FWD_THREADS, x->smem_bytes) != cudaSuccess || occ < 1)
     return fail(BLINK_ECUDA);
-  if (x->pair) {   // every cluster of two must be resident at once (the loop's grid barrier needs the whole grid)
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(x->grid); cfg.blockDim = dim3(FWD_THREADS); cfg.dynamicSmemBytes = x->smem_bytes;
-    cudaLaunchAttribute at[1];
-    at[0].id = cudaLaunchAttributeClusterDimension; at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
-    cfg.attrs = at; cfg.numAttrs = 1;
-    int ncl = 0;
-    if (cudaOccupancyMaxActiveClusters(&ncl, loop_fn, &cfg) != cudaSuccess || 2 * ncl < x->grid) return fail(BLINK_EINVAL);
-  }
   if (cudaDeviceSynchronize() != cudaSuccess) return fail(BLINK_ECUDA);
   if (!c.stepped && !x->manual) {
     rc = launch_loop(x);

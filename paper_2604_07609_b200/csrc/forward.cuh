@@ -182,7 +182,7 @@ __device__ __forceinline__ void norm_row_cta(const DevCtx& c, float* hrow, const
 // ---- RMSNorm of the residual rows into the operand buffer; layer 0 gathers the
 // embedding first.
 template <typename WT>
-static __device__ void phase_norm(const DevCtx& c, int layer, int which /*0: norm1, 1: norm2*/) {
+static __device__ __noinline__ void phase_norm(const DevCtx& c, int layer, int which /*0: norm1, 1: norm2*/) {
   __shared__ float s_red[FWD_THREADS / 32];
   const int T = c.ss->cur_T;
   const float* g = wptr_f(c, which == 0 ? 6 : 7) + (size_t)layer * c.d;
@@ -245,7 +245,7 @@ __device__ __noinline__ void norm_apply_rows(const float* __restrict__ h, const 
 // which 0 = first norm of layer > 0 (reads rowss_b, clears rowss_a), 1 = second norm (reads rowss_a,
 // clears rowss_b).  The cleared buffer is the one the next GEMM epilogue adds into.
 template <typename WT>
-static __device__ void phase_norm_apply(const DevCtx& c, int layer, int which, int T) {
+static __device__ __noinline__ void phase_norm_apply(const DevCtx& c, int layer, int which, int T) {
   const float* g = wptr_f(c, which == 0 ? 6 : 7) + (size_t)layer * c.d;
   float* clear = which == 0 ? c.rowss_a : c.rowss_b;
   for (int i = blockIdx.x * FWD_THREADS + threadIdx.x; i < T; i += gridDim.x * FWD_THREADS) clear[i] = 0.f;
@@ -254,7 +254,7 @@ static __device__ void phase_norm_apply(const DevCtx& c, int layer, int which, i
 
 // Final norm of the sampled rows only (the LM head runs on those rows).
 template <typename WT>
-static __device__ void phase_final_norm(const DevCtx& c) {
+static __device__ __noinline__ void phase_final_norm(const DevCtx& c) {
   __shared__ float s_red[FWD_THREADS / 32];
   const int R = c.ss->cur_rows;
   const float* g = wptr_f(c, 8);
@@ -297,7 +297,7 @@ struct GemmArgs {
 };
 
 template <typename WT>
-static __device__ void phase_gemm_simt(const GemmArgs& a) {
+static __device__ __noinline__ void phase_gemm_simt(const GemmArgs& a) {
   constexpr int BM = 64, BN = 64, BK = 16;
   __shared__ float xs[BK][BM + 4];
   __shared__ float ws[BK][BN + 4];
@@ -368,7 +368,7 @@ __device__ __forceinline__ WT* kv_tile(const DevCtx& c, int layer, int kv, int b
 }
 
 template <typename WT>
-static __device__ void phase_rope_kv(const DevCtx& c, int layer) {
+static __device__ __noinline__ void phase_rope_kv(const DevCtx& c, int layer) {
   // one thread: four consecutive rotation pairs (i .. i+3, i+half .. i+half+3) of one head of one row
   const int T = c.ss->cur_T;
   const int half = c.hd / 2, quads = half / 4;
@@ -543,7 +543,7 @@ static __device__ __noinline__ void fixup_sumsq(const float* h, int ld, int N, f
 // vector load per lane covers whole (block, head) tiles with coalesced 512-byte rows.
 // Online softmax per warp, merged across warps in shared memory at the end.
 template <typename WT, int HD, int NREP>
-static __device__ void phase_attention(const DevCtx& c, int layer, float* smem) {
+static __device__ __noinline__ void phase_attention(const DevCtx& c, int layer, float* smem) {
   constexpr int CE = 16 / (int)sizeof(WT);  // elements per 16-byte chunk
   constexpr int LPK = HD / CE;              // lanes per key
   constexpr int KPP = 32 / LPK;             // keys per pass
@@ -710,7 +710,7 @@ __device__ __noinline__ void silu_mul_rows(float* __restrict__ gu, WT* __restric
   }
 }
 template <typename WT>
-static __device__ void phase_silu_mul(const DevCtx& c) {
+static __device__ __noinline__ void phase_silu_mul(const DevCtx& c) {
   const int T = c.E > 0 ? c.ss->cur_T * c.topE : c.ss->cur_T;   // rows of the gate/up buffer
   if (T > 0) silu_mul_rows<WT>(c.gu, reinterpret_cast<WT*>(c.act), T, c.F, c.gemm_tc != 0);
 }
@@ -720,7 +720,7 @@ static __device__ void phase_silu_mul(const DevCtx& c) {
 // the order does not depend on timing), CTA 0 publishes them, and all CTAs copy the normed rows
 // of the tokens into expert-contiguous order for the per-expert GEMMs.
 template <typename WT>
-static __device__ void phase_moe_group(const DevCtx& c, float* smem) {
+static __device__ __noinline__ void phase_moe_group(const DevCtx& c, float* smem) {
   const int T = c.ss->cur_T, K = c.topE, E = c.E;
   const int A = T * K;   // assignments
   __shared__ int s_off[MAX_EXPERTS + 1];
@@ -1235,7 +1235,7 @@ static __device__ int sample_row(const float* lg, int V, int top_k, float temp, 
   return result;
 }
 
-static __device__ void phase_sample(const DevCtx& c, float* smem) {
+static __device__ __noinline__ void phase_sample(const DevCtx& c, float* smem) {
   const int R = c.ss->cur_rows;
   const int V = c.V;
   const int tid = threadIdx.x;

@@ -561,7 +561,7 @@ static __device__ __noinline__ void tc_finish_tiles(const DevCtx& c, const GemmA
 }
 
 template <bool PAIR>
-static __device__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int which, int layer, float* smem_f, TcState& tc) {
+static __device__ __noinline__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int which, int layer, float* smem_f, TcState& tc) {
   const int T = a.M, N = a.N, K = a.K;
   if (T <= 0) return;  // uniform over the grid
   const TcMaps* maps = reinterpret_cast<const TcMaps*>(c.tc_maps);

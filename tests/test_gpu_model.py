@@ -127,9 +127,12 @@ def test_config1_bf16_tensor_core_path_matches_oracle(fusion):
     assert err <= TOL_BF16
 
 
-def test_tensor_core_path_multi_pass_ragged_shapes():
-    """More than 256 rows in a step (two token passes), 24 k-blocks, 35 n-tiles, GQA 4:1 with
-    head_dim 128, non-unit gains: every stream-K segment kind (whole tile, head, tail) occurs."""
+@pytest.mark.parametrize("gemm,fusion", [(B.GEMM_TC, B.FUSION_ON), (B.GEMM_TC, B.FUSION_OFF), (B.GEMM_TC_PAIR, B.FUSION_OFF)],
+                         ids=["single-cta-fused", "single-cta", "cta-pairs"])
+def test_tensor_core_path_multi_pass_ragged_shapes(gemm, fusion):
+    """More than 256 rows in a step (two token passes), 24 k-blocks, 35 n-tiles (an odd number: the
+    last CTA pair has one real weight tile), GQA 4:1 with head_dim 128, non-unit gains: every stream-K
+    segment kind (whole tile, head, tail) occurs."""
     model = model_cfg(1, d_model=512, n_q_heads=4, n_kv_heads=1, head_dim=128, d_ff=1536, vocab=4480, dtype="bf16")
     sched = sched_cfg(1, prefill_chunk_tokens=300, max_batch=8, n_blocks=256, max_prompt=320, max_new=8)
     rng = np.random.default_rng(21)
@@ -137,8 +140,8 @@ def test_tensor_core_path_multi_pass_ragged_shapes():
     reqs = [Request(t, 0.0, rng.integers(0, model.vocab, size=int(p)).astype(np.int32), 6)
             for t, p in enumerate([310, 17, 301, 64, 129, 256, 5, 300, 33])]
     w = make_weights(model, 77, "cpu", random_gains=True)
-    err, n_margin, trace, toks, ora = _compare(model, sched, reqs, w, O2.round_bf16, TOL_BF16, gemm_impl=B.GEMM_TC,
-                                               epilogue_fusion=B.FUSION_ON)
+    err, n_margin, trace, toks, ora = _compare(model, sched, reqs, w, O2.round_bf16, TOL_BF16, gemm_impl=gemm,
+                                               epilogue_fusion=fusion)
     print(f"multi-pass tensor cores: max-abs logit error {err:.3e}; max rows/step "
           f"{max(sum(s[4] for s in r['scheduled']) for r in trace)}")
     assert err <= TOL_BF16
@@ -156,7 +159,8 @@ def test_tensor_core_and_cuda_core_paths_agree():
     assert_traces_equal([{**r, "sampled": []} for r in a[0]], [{**r, "sampled": []} for r in b[0]])
 
 
-def test_streaming_weight_layout_round_trip_and_parity():
+@pytest.mark.parametrize("gemm", [B.GEMM_TC, B.GEMM_TC_PAIR], ids=["single-cta", "cta-pairs"])
+def test_streaming_weight_layout_round_trip_and_parity(gemm):
     """The GEMM matrices converted in place to the tile-contiguous streaming layout: converting back
     restores every byte, and the loop reading the streaming layout meets the same tolerance."""
     model = model_cfg(1, d_model=512, n_q_heads=4, n_kv_heads=1, head_dim=128, d_ff=1536, vocab=4480, dtype="bf16")
@@ -180,7 +184,7 @@ def test_streaming_weight_layout_round_trip_and_parity():
     for r in (0, 1, 7, 8, 77, 127):
         for c8 in range(8):
             assert torch.equal(tile[r, c8 ^ (r & 7)], rm[r, c8])
-    err, _, trace, toks, ora = _compare(model, sched, reqs, w, O2.round_bf16, TOL_BF16, gemm_impl=B.GEMM_TC,
+    err, _, trace, toks, ora = _compare(model, sched, reqs, w, O2.round_bf16, TOL_BF16, gemm_impl=gemm,
                                         weights_layout=B.WEIGHTS_STREAMING)
     print(f"streaming layout: max-abs logit error {err:.3e}")
     # the SIMT path cannot read the streaming layout: refused, not misread

@@ -36,8 +36,9 @@ def _report(name, r):
     return rows, dec
 
 
-@pytest.mark.parametrize("fusion", [B.FUSION_OFF, B.FUSION_ON], ids=["separate-phases", "fused-epilogues"])
-def test_8b_layer_shape_small_sample_topk(fusion):
+@pytest.mark.parametrize("gemm,fusion", [(B.GEMM_TC_PAIR, B.FUSION_OFF), (B.GEMM_TC, B.FUSION_OFF), (B.GEMM_TC, B.FUSION_ON)],
+                         ids=["cta-pairs", "single-cta", "single-cta-fused-epilogues"])
+def test_8b_layer_shape_small_sample_topk(gemm, fusion):
     """Four requests, prompts of at most 64 tokens, 16 new tokens each, top-k 50 at T 0.8: the sample
     the benchmark's CPU leg times, on four layers of the 8B shape (d 4096, 32/8 heads of 128, FFN
     14336, vocabulary 128256), streaming weight layout, tensor-core GEMMs."""
@@ -48,7 +49,7 @@ def test_8b_layer_shape_small_sample_topk(fusion):
         r.prompt = r.prompt[:64]
         r.max_new = 16
     w = make_weights(model, 20260407, "cpu")
-    r = compare_with_oracle(model, sched, reqs, w, TOL_BF16, oracle_dtype=np.float32, noise_relative=True, gemm_impl=B.GEMM_TC,
+    r = compare_with_oracle(model, sched, reqs, w, TOL_BF16, oracle_dtype=np.float32, noise_relative=True, gemm_impl=gemm,
                             weights_layout=B.WEIGHTS_STREAMING, epilogue_fusion=fusion)
     _report("8B layer shape, 4 requests", r)
 
@@ -66,7 +67,7 @@ def test_8b_layer_shape_128_row_decode_batch_and_multi_pass_prefill():
     reqs = [Request(t, 0.0, rng.integers(0, model.vocab, size=int(p)).astype(np.int32), 7)
             for t, p in enumerate(rng.integers(100, 201, size=128))]
     w = make_weights(model, 20260408, "cpu")
-    r = compare_with_oracle(model, sched, reqs, w, TOL_BF16, oracle_dtype=np.float32, noise_relative=True, gemm_impl=B.GEMM_TC,
+    r = compare_with_oracle(model, sched, reqs, w, TOL_BF16, oracle_dtype=np.float32, noise_relative=True, gemm_impl=B.GEMM_AUTO,
                             weights_layout=B.WEIGHTS_STREAMING)
     rows, dec = _report("8B layer shape, 128-row batch", r)
     assert rows > 4096 and dec == 128
@@ -81,7 +82,7 @@ def test_1b_layer_shape_head_dim_64_four_heads_per_group():
     reqs = [Request(t, 0.0, rng.integers(0, model.vocab, size=int(p)).astype(np.int32), 8)
             for t, p in enumerate(rng.integers(40, 321, size=48))]
     w = make_weights(model, 20260409, "cpu")
-    r = compare_with_oracle(model, sched, reqs, w, TOL_BF16, oracle_dtype=np.float32, noise_relative=True, gemm_impl=B.GEMM_TC,
+    r = compare_with_oracle(model, sched, reqs, w, TOL_BF16, oracle_dtype=np.float32, noise_relative=True, gemm_impl=B.GEMM_AUTO,
                             weights_layout=B.WEIGHTS_STREAMING)
     rows, dec = _report("1B layer shape", r)
     assert dec == 48
@@ -96,6 +97,6 @@ def test_moe_layer_shape_two_layers():
     reqs = [Request(t, 0.0, rng.integers(0, model.vocab, size=int(p)).astype(np.int32), 3)
             for t, p in enumerate(rng.integers(8, 33, size=8))]
     w = make_weights(model, 20260410, "cpu")
-    r = compare_with_oracle(model, sched, reqs, w, TOL_BF16, oracle_dtype=np.float32, noise_relative=True, gemm_impl=B.GEMM_TC,
+    r = compare_with_oracle(model, sched, reqs, w, TOL_BF16, oracle_dtype=np.float32, noise_relative=True, gemm_impl=B.GEMM_AUTO,
                             weights_layout=B.WEIGHTS_STREAMING)
     _report("routed-expert layer shape", r)
