@@ -276,6 +276,16 @@ int blink_submit(blink_ctx* ctx, const blink_request* req, uint64_t* ticket_out)
  * that left the GPU (budget, idle) while work is outstanding. */
 int blink_poll(blink_ctx* ctx, blink_token_event* out, int max_events, int timeout_us);
 
+/* Ask the loop to drop a request (the paper lists early exits among what the serving path has to handle,
+ * Section 1; it gives no mechanism).  The device retires it at the end of the step in which it sees the mark:
+ * its KV blocks return to the free list, its reservation and batch slot are released, no further token is
+ * produced.  Tokens published before that are still delivered; then blink_poll hands out one closing event
+ * for the request with token = -1, index = number of tokens it produced, and is_last set (no other event of
+ * a cancelled request carries is_last).  A request that was still waiting for admission is admitted first and
+ * retired at the end of its first step.  BLINK_EINVAL when the ticket is unknown or the request has already
+ * delivered its last token.  Thread-safe, non-blocking. */
+int blink_cancel(blink_ctx* ctx, uint64_t ticket);
+
 /* Stepped mode only: run `n_iterations` iterations, one host launch per phase,
  * and wait for them. */
 int blink_step(blink_ctx* ctx, int n_iterations);

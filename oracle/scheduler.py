@@ -63,6 +63,8 @@ LEGAL_TRANSITIONS = {
     # pause-and-resume prefill: decode requests wait while new prompts are prefetched
     (DECODE_PROCESSING, DECODE_PAUSED),
     (DECODE_PAUSED, DECODE_PROCESSING),
+    # a cancelled request is retired from wherever it stands (PREFILL_PROCESSING -> DECODE_COMPLETED is above)
+    (DECODE_PAUSED, DECODE_COMPLETED),
 }
 
 
@@ -225,7 +227,11 @@ class Scheduler:
         return items
 
     # -- step 5
-    def finish(self, items, sampled_tokens: Sequence[int]):
+    def finish(self, items, sampled_tokens: Sequence[int], cancelled: Sequence[int] = ()):
+        """`cancelled`: tickets whose cancellation the loop saw at the end of this iteration (the paper lists
+        early exits among what the serving path must handle, Section 1; no mechanism is given): after the
+        iteration's own completions, every live request among them is retired in ascending batch slot, its
+        blocks pushed back in logical order and its reservation released, exactly as at a normal end."""
         rec = self._pending
         self._pending = None
         sampled, finished, freed = [], [], []
@@ -252,6 +258,15 @@ class Scheduler:
                     freed.append(blk)
                 self.reserved -= e.need
                 self.batch[item.bslot] = None
+        for b, e in enumerate(self.batch):
+            if e is not None and e.ticket in cancelled:
+                self._move(e.ticket, DECODE_COMPLETED)
+                finished.append(e.ticket)
+                for blk in e.blocks:
+                    self.stack.append(blk)
+                    freed.append(blk)
+                self.reserved -= e.need
+                self.batch[b] = None
         rec.update(sampled=sampled, finished=finished, freed=freed,
                    free_count=len(self.stack), reserved=self.reserved)
         self.iter += 1
@@ -270,7 +285,8 @@ class Scheduler:
 def simulate(requests: Sequence[SimRequest], max_batch: int, chunk: int, n_blocks: int,
              block: int = 16, watermarks: Optional[Sequence[int]] = None,
              sample_fn: Optional[Callable] = None, vocab: int = 1 << 30,
-             max_iters: int = 10_000_000, check: Optional[Callable] = None, policy: str = "chunked"):
+             max_iters: int = 10_000_000, check: Optional[Callable] = None, policy: str = "chunked",
+             cancels: Optional[dict] = None):
     """Run to drain.  `watermarks[i]` is W of traced iteration i (default: all
     requests visible from the start).  `sample_fn(items) -> tokens for the sample
     rows in order` (default: the control-only fake sampler).
@@ -289,7 +305,7 @@ def simulate(requests: Sequence[SimRequest], max_batch: int, chunk: int, n_block
             toks = [fake_token(i.ticket, i.gen_index, vocab) for i in items if i.sample]
         else:
             toks = sample_fn(items)
-        rec = sch.finish(items, toks)
+        rec = sch.finish(items, toks, (cancels or {}).get(len(trace), ()))
         for (b, tok), item in zip(rec["sampled"], [i for i in items if i.sample]):
             out[item.ticket].append(tok)
         trace.append(rec)

@@ -91,7 +91,7 @@ EVENT_DTYPE = np.dtype([("ticket", "<u8"), ("user_tag", "<u8"), ("index", "<i4")
                         ("t_submit_ns", "<u8")])
 
 EXPORTS = ["blink_weights_bytes", "blink_weight_offset", "blink_convert_weights", "blink_kv_blocks_for_bytes", "blink_create",
-           "blink_start", "blink_submit", "blink_poll", "blink_step", "blink_run", "blink_stop", "blink_destroy",
+           "blink_start", "blink_submit", "blink_cancel", "blink_poll", "blink_step", "blink_run", "blink_stop", "blink_destroy",
            "blink_get_stats", "blink_get_trace", "blink_get_iter_stats", "blink_sample", "blink_sample_top_p",
            "blink_sample_noalloc",
            "blink_strerror"]
@@ -123,6 +123,8 @@ def lib():
     L.blink_start.argtypes = [C.c_void_p]
     L.blink_submit.restype = C.c_int
     L.blink_submit.argtypes = [C.c_void_p, P(blink_request), P(C.c_uint64)]
+    L.blink_cancel.restype = C.c_int
+    L.blink_cancel.argtypes = [C.c_void_p, C.c_uint64]
     L.blink_poll.restype = C.c_int
     L.blink_poll.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int]
     L.blink_step.restype = C.c_int
@@ -343,6 +345,9 @@ class Blink:
                 raise BlinkError(rc, "blink_submit")
             return rc
         return int(t.value)
+
+    def blink_cancel(self, ticket: int) -> int:
+        return int(lib().blink_cancel(self._h, ticket))
 
     def blink_poll(self, max_events=4096, timeout_us=0) -> np.ndarray:
         max_events = min(max_events, self._ev.shape[0])

@@ -154,6 +154,7 @@ struct blink_ctx {
   int32_t *sub_tokens = nullptr, *sub_forced = nullptr, *out_tokens = nullptr;
   uint64_t* out_time = nullptr;
   uint32_t* out_count = nullptr;
+  uint32_t* cancel = nullptr;    // host view of the cancel marks
   std::mutex mu;
   std::vector<SlotInfo> slots;
   std::deque<int> active;
@@ -686,6 +687,7 @@ int blink_create(const blink_model_cfg* model, const blink_sched_cfg* sched, con
     TRY(pinned_alloc(x, &x->out_tokens, &od, S * c.max_new)); c.out_tokens = od;
     TRY(pinned_alloc(x, &x->out_time, &tmd, S * c.max_new)); c.out_time = tmd;
     TRY(pinned_alloc(x, &x->out_count, &cd, S)); c.out_count = cd;
+    { uint32_t* cn; TRY(pinned_alloc(x, &x->cancel, &cn, S)); c.cancel = cn; }
   }
   if (c.gemm_tc) TRY(tc_host_setup(x->tc_host, c));
 #undef TRY
@@ -787,6 +789,7 @@ int blink_submit(blink_ctx* x, const blink_request* r, uint64_t* ticket_out) {
   memcpy(x->sub_tokens + (size_t)slot * c.max_prompt, r->prompt, (size_t)r->n_prompt * 4);
   if (r->forced_tokens) memcpy(x->sub_forced + (size_t)slot * c.max_new, r->forced_tokens, (size_t)r->max_new_tokens * 4);
   x->out_count[slot] = 0;
+  x->cancel[slot] = 0;
   SubEntry& e = x->sub_q[ticket % (uint64_t)c.n_slots];
   e.ticket = ticket; e.seed = r->seed; e.user_tag = r->user_tag; e.slot = (uint32_t)slot;
   e.n_prompt = (uint32_t)r->n_prompt; e.max_new = (uint32_t)r->max_new_tokens; e.top_k = (uint32_t)r->top_k;
@@ -819,20 +822,27 @@ int blink_poll(blink_ctx* x, blink_token_event* out, int max_events, int timeout
         const int slot = *it;
         SlotInfo& si = x->slots[slot];
         const uint32_t cnt = __atomic_load_n(&x->out_count[slot], __ATOMIC_ACQUIRE);
-        const int have = (int)(cnt & 0x7fffffffu);
+        const int have = (int)(cnt & 0x3fffffffu);
         const bool fin = (cnt >> 31) != 0;
+        const bool cancelled = (cnt & 0x40000000u) != 0;
         while (si.consumed < have && n < max_events) {
           blink_token_event& ev = out[n++];
           const size_t idx = (size_t)slot * c.max_new + si.consumed;
           ev.ticket = si.ticket; ev.user_tag = si.user_tag; ev.index = si.consumed;
           ev.token = x->out_tokens[idx];
           ev.is_first = si.consumed == 0;
-          ev.is_last = fin && si.consumed + 1 == have;
+          ev.is_last = fin && !cancelled && si.consumed + 1 == have;
           ev.t_device_ns = x->out_time[idx];
           ev.t_host_ns = t_now;
           ev.t_submit_ns = si.t_submit_ns;
           si.consumed += 1;
           x->bytes_from_device += 16;   // what the device wrote into the host mirrors for it: token, timestamp, count word
+        }
+        if (fin && cancelled && si.consumed == have) {
+          if (n >= max_events) { ++it; continue; }   // no room for the closing event in this call
+          blink_token_event& ev = out[n++];           // a cancelled request ends with an event of its own
+          ev.ticket = si.ticket; ev.user_tag = si.user_tag; ev.index = have; ev.token = -1;
+          ev.is_first = 0; ev.is_last = 1; ev.t_device_ns = 0; ev.t_host_ns = t_now; ev.t_submit_ns = si.t_submit_ns;
         }
         if (fin && si.consumed == have) {
           si.busy = false;  // DECODE_COMPLETED -> EMPTY: the frontend owns this transition
@@ -845,6 +855,19 @@ int blink_poll(blink_ctx* x, blink_token_event* out, int max_events, int timeout
     if (n > 0 || now_ns() >= deadline) return n;
     std::this_thread::sleep_for(std::chrono::microseconds(20));
   }
+}
+
+int blink_cancel(blink_ctx* x, uint64_t ticket) {
+  if (!x) return BLINK_EINVAL;
+  std::lock_guard<std::mutex> g(x->mu);
+  for (int slot : x->active) {
+    SlotInfo& si = x->slots[slot];
+    if (si.busy && si.ticket == ticket) {
+      __atomic_store_n(&x->cancel[slot], 1u, __ATOMIC_RELEASE);
+      return BLINK_OK;
+    }
+  }
+  return BLINK_EINVAL;   // unknown, or all of its tokens have been handed out already
 }
 
 int blink_step(blink_ctx* x, int n_iterations) {

@@ -198,21 +198,64 @@ static __device__ void post_step(const DevCtx& c) {
     c.b_phase[b] = PHASE_FREE;
   }
   __syncthreads();
+  // Cancellation (an early exit the host asks for): every request that is still live after the step's
+  // own completions and whose slot carries the host's cancel mark is retired here, in ascending batch
+  // slot, exactly as at a normal end: blocks pushed back in logical order, reservation released.
+  int cfin = 0, cfree = 0, cslot = 0;
+  long long cticket = 0;
+  if (c.cancel != nullptr && tid < c.MB && c.b_phase[tid] != PHASE_FREE) {
+    cslot = c.b_slot[tid];
+    if (ld_relaxed_sys_u32(&c.cancel[cslot]) != 0u) {
+      cfin = 1;
+      cfree = c.b_have[tid];
+      cticket = c.b_ticket[tid];
+      atomicAdd(&s_need_sum, c.b_need[tid]);
+    }
+  }
+  int tot_cfin, tot_cfree;
+  const int cfin_idx = block_exscan(cfin, &tot_cfin);
+  const int cfree_off = block_exscan(cfree, &tot_cfree);
+  if (cfin) {
+    if (tr) rec_post[2 * n_rows + tot_fin + tot_free + cfin_idx] = (int32_t)cticket;
+    for (int j = 0; j < cfree; ++j) {
+      const int blk = c.block_table[(size_t)tid * c.max_blocks_seq + j];
+      c.free_stack[top + tot_free + cfree_off + j] = blk;
+      if (tr) rec_post[2 * n_rows + tot_fin + tot_free + tot_cfin + cfree_off + j] = blk;
+    }
+    c.b_have[tid] = 0;
+    c.b_phase[tid] = PHASE_FREE;
+    c.slot_hot[cslot].state = SLOT_DECODE_COMPLETED;
+    __threadfence_system();
+    c.out_count[cslot] = (uint32_t)c.b_generated[tid] | 0xC0000000u;   // finished + cancelled
+  }
+  __syncthreads();
   if (tid == 0) {
-    ss->free_top = top + tot_free;
+    ss->free_top = top + tot_free + tot_cfree;
     ss->reserved -= s_need_sum;
     ss->tokens_out += (unsigned long long)n_rows;
     ss->prompt_tokens += s_ptok;
     ss->sample_rows_total += (unsigned long long)n_rows;
     const uint64_t t_end = global_timer_ns();
     if (tr) {
+      // The record lists finished tickets then freed blocks; with cancellations the order is: tickets
+      // that ended by themselves, their blocks, cancelled tickets, their blocks -- rewritten below into
+      // the record's two lists (tickets first, then blocks) when both kinds occur.
       int32_t* hdr = c.trace + ss->cur_hdr;
+      if (tot_cfin > 0 && tot_free > 0) {
+        // move the cancelled tickets in front of the first group's blocks (few words, one thread)
+        int32_t* base = rec_post + 2 * n_rows + tot_fin;
+        for (int k = 0; k < tot_cfin; ++k) {
+          const int32_t tk = base[tot_free + k];
+          for (int j = tot_free + k; j > k; --j) base[j] = base[j - 1];
+          base[k] = tk;
+        }
+      }
       hdr[6] = n_rows;
-      hdr[7] = tot_fin;
-      hdr[8] = tot_free;
+      hdr[7] = tot_fin + tot_cfin;
+      hdr[8] = tot_free + tot_cfree;
       hdr[9] = ss->free_top;
       hdr[10] = ss->reserved;
-      const long long end = ss->cur_post + 2 * n_rows + tot_fin + tot_free;
+      const long long end = ss->cur_post + 2 * n_rows + tot_fin + tot_cfin + tot_free + tot_cfree;
       hdr[11] = (int32_t)(end - ss->cur_hdr);
       ss->trace_pos = end;
     }
@@ -438,9 +481,11 @@ static __device__ int schedule_step(const DevCtx& c, unsigned long long visible)
   const int qstart = block_exscan(take, &T);
   const int aoff = block_exscan(want, &n_alloc);
   const int row = block_exscan(sample, &n_rows);
-  // blocks that post_step may free at most (for the trace space check)
-  int tot_may_free;
-  block_exscan(sample ? have + want : 0, &tot_may_free);
+  // blocks that post_step may free at most, and tickets that may end (completions and cancellations),
+  // for the trace space check
+  int tot_may_free, n_live;
+  block_exscan(phase != PHASE_FREE ? have + want : 0, &tot_may_free);
+  block_exscan(phase != PHASE_FREE ? 1 : 0, &n_live);
   // attention work lists: single-row requests stream their KV blocks, multi-row requests are
   // cut into blocks of 128 / n_rep query rows
   const int q_rows = 128 / c.n_rep;
@@ -457,8 +502,8 @@ static __device__ int schedule_step(const DevCtx& c, unsigned long long visible)
   if (tid == 0) {
     int ok = 1;
     if (hdr >= 0) {
-      const long long worst = hdr + TRACE_HDR_WORDS + 2ll * n_admit + 5ll * n_items + 3ll * n_alloc + 3ll * n_rows +
-                              tot_may_free;
+      const long long worst = hdr + TRACE_HDR_WORDS + 2ll * n_admit + 5ll * n_items + 3ll * n_alloc + 2ll * n_rows +
+                              n_live + tot_may_free;
       if (worst > c.trace_cap) {
         ok = 0;
         ss->trace_off = 1;

@@ -154,7 +154,8 @@ struct DevCtx {
   const int32_t* sub_forced;  // [n_slots][max_new]
   int32_t* out_tokens;        // [n_slots][max_new]
   uint64_t* out_time;         // [n_slots][max_new]
-  uint32_t* out_count;        // [n_slots] generated | 0x80000000 when finished
+  uint32_t* out_count;        // [n_slots] generated | 0x80000000 when finished | 0x40000000 when cancelled
+  const uint32_t* cancel;     // [n_slots] host: non-zero = retire the request in this slot at the next step boundary
   // scheduler state in HBM
   SchedState* ss;
   uint32_t* ticket_to_slot;   // [n_slots]

@@ -224,3 +224,63 @@ def test_pause_resume_policy_trace_bit_exact():
     # a prefill budget below the longest accepted prompt cannot run whole prompts: refused at create
     with pytest.raises(B.BlinkError):
         B.Blink(model, sched_cfg(1, prefill_chunk_tokens=32, max_prompt=64), control_only=True, policy=B.POLICY_PAUSE_RESUME)
+
+
+def test_cancel_retires_a_running_request_and_the_trace_equals_the_oracles():
+    """blink_cancel on a request that is generating: the device retires it at a step boundary (blocks and
+    reservation returned, batch slot released), its tokens so far are delivered, one closing event follows,
+    and the trace equals the oracle's when the oracle is told in which iteration the mark was seen."""
+    import time
+    model = model_cfg(1)
+    sched = sched_cfg(1, max_batch=3, n_blocks=2048, max_prompt=64, max_new=30000, n_slots=16)
+    rng = np.random.default_rng(23)
+    mk = lambda n: rng.integers(0, 4096, size=n).astype(np.int32)
+    reqs = [Request(0, 0.0, mk(40), 12), Request(1, 0.0, mk(25), 30000), Request(2, 0.0, mk(33), 20),
+            Request(3, 0.0, mk(10), 15), Request(4, 0.0, mk(50), 9)]
+    eng = B.Blink(model, sched, control_only=True, start_paused=True, trace_words=1 << 24, idle_exit_us=300_000)
+    try:
+        for r in reqs:
+            eng.submit_request(r)
+        eng.blink_start()
+        evs, closing = [], None
+        t0 = time.monotonic()
+        asked = False
+        while closing is None and time.monotonic() - t0 < 30:
+            e = eng.blink_poll(4096, 1000)
+            if len(e):
+                evs.append(e)
+                if not asked and (e["ticket"] == 1).sum() > 0:
+                    assert eng.blink_cancel(1) == B.BLINK_OK       # ticket 1 is generating: stop it
+                    asked = True
+                c = e[(e["ticket"] == 1) & (e["is_last"] == 1)]
+                if len(c):
+                    closing = c[0]
+        assert closing is not None and int(closing["token"]) == -1
+        # everything else runs to its end
+        rest = sum(r.max_new for r in reqs if r.ticket != 1)
+        got = sum(int((e["ticket"] != 1).sum()) for e in evs)
+        while got < rest and time.monotonic() - t0 < 60:
+            e = eng.blink_poll(4096, 1000)
+            evs.append(e)
+            got += int((e["ticket"] != 1).sum())
+        assert got == rest
+        assert eng.blink_cancel(1) == B.BLINK_EINVAL              # gone
+        assert eng.blink_cancel(99) == B.BLINK_EINVAL             # never existed
+        eng.blink_stop(final=False)
+        st = eng.blink_get_stats()
+        trace = B.parse_trace(eng.blink_get_trace())
+    finally:
+        assert eng.blink_destroy() == B.BLINK_OK
+    assert st.device_status == 0
+    ev = np.concatenate(evs)
+    mine = np.sort(ev[(ev["ticket"] == 1) & (ev["token"] >= 0)], order="index")
+    n1 = len(mine)
+    assert 0 < n1 < 30000 and list(mine["index"]) == list(range(n1)) and mine["is_last"].sum() == 0
+    assert int(closing["index"]) == n1
+    it_c = next(i for i, r in enumerate(trace) if 1 in r["finished"])
+    tr_o, toks_o, _ = O1.simulate([O1.SimRequest(r.ticket, r.n_prompt, r.max_new, r.eos_id, r.prompt) for r in reqs],
+                                  sched.max_batch, sched.prefill_chunk_tokens, sched.n_blocks, sched.block_size,
+                                  watermarks=[r["W"] for r in trace], vocab=model.vocab, cancels={it_c: [1]})
+    assert_traces_equal(trace, tr_o)
+    assert len(toks_o[1]) == n1 and [int(t) for t in mine["token"]] == toks_o[1]
+    assert st.free_blocks == sched.n_blocks and st.reserved_blocks == 0 and st.batch_live == 0

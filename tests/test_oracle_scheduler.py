@@ -243,3 +243,27 @@ def test_pause_resume_slot_states_follow_the_paper_state_machine():
     resumed = [(t, a, b) for (t, a, b) in sch.transitions if a == O1.DECODE_PAUSED]
     assert paused and len(paused) == len(resumed)                       # every pause is followed by a resume
     assert all(b == O1.DECODE_PROCESSING for (_, _, b) in resumed)
+
+
+# ---- cancellation (an early exit the host asks for) ----------------------------------------------------
+def test_cancel_retires_a_request_and_returns_everything_it_held():
+    # alone: cancelled at the end of iteration 3 -> four iterations, all blocks back, nothing reserved
+    tr, toks, sch = O1.simulate([O1.SimRequest(0, 40, 100)], 2, 64, 32, 16, vocab=4096, cancels={3: [0]},
+                                check=O1.check_invariants)
+    assert len(tr) == 4 and tr[3]["finished"] == [0] and len(toks[0]) == 4
+    assert tr[3]["freed"] == [0, 1, 2] and tr[3]["free_count"] == 32 and tr[3]["reserved"] == 0 and sch.idle
+    assert all((a, b) in O1.LEGAL_TRANSITIONS for (_, a, b) in sch.transitions)
+    # in a full batch: the freed batch slot and blocks let the waiting request in one iteration later
+    reqs = [O1.SimRequest(0, 30, 50), O1.SimRequest(1, 30, 50), O1.SimRequest(2, 20, 5)]
+    base, _, _ = O1.simulate(reqs, 2, 64, 64, 16, vocab=4096, check=O1.check_invariants)
+    cut, toks, _ = O1.simulate(reqs, 2, 64, 64, 16, vocab=4096, cancels={5: [1]}, check=O1.check_invariants)
+    first_in = lambda tr: next(i for i, r in enumerate(tr) if any(t == 2 for t, _ in r["admitted"]))
+    assert first_in(cut) == 6 and first_in(base) > 40
+    assert cut[5]["finished"] == [1] and len(toks[1]) == 6 and len(toks[0]) == 50 and len(toks[2]) == 5
+    assert cut[-1]["free_count"] == 64 and cut[-1]["reserved"] == 0
+    # a ticket that is not live at that iteration (finished already, or not admitted yet) changes nothing
+    same, _, _ = O1.simulate(reqs, 2, 64, 64, 16, vocab=4096, cancels={5: [2], 200: [0]})
+    assert same == base
+    # a request in the middle of a chunked prompt (no token yet) goes from PREFILL_PROCESSING to DECODE_COMPLETED
+    tr, toks, sch = O1.simulate([O1.SimRequest(0, 200, 9)], 2, 64, 32, 16, vocab=4096, cancels={1: [0]})
+    assert len(tr) == 2 and toks[0] == [] and (0, O1.PREFILL_PROCESSING, O1.DECODE_COMPLETED) in sch.transitions
