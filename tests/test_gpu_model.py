@@ -293,3 +293,28 @@ def test_pause_resume_policy_logits_and_tokens_fp32():
     print(f"pause-and-resume fp32: max-abs logit error {err:.3e}")
     assert all(len({s[2] for s in r["scheduled"]}) == 1 for r in trace)
     assert any(len(r["scheduled"]) > 1 and r["scheduled"][0][2] == 1 for r in trace)     # several prompts in one step
+
+
+def test_bf16_stepped_and_persistent_modes_agree_on_the_tensor_core_path():
+    """The persistent loop reads, through TMA, buffers that earlier phases of the same kernel wrote with
+    ordinary stores (normed rows, K/V rows, attention output, SwiGLU output); the stepped mode has a kernel
+    boundary between any two phases.  Both must give the same trace, logits within the bf16 tolerance of
+    each other and of the oracle, and tokens by the margin rule (split-K sums land in arrival order, so
+    the two are not bit-identical)."""
+    model = model_cfg(1, d_model=512, n_q_heads=4, n_kv_heads=1, head_dim=128, d_ff=1536, vocab=4480, dtype="bf16")
+    sched = sched_cfg(1, prefill_chunk_tokens=300, max_batch=8, n_blocks=256, max_prompt=320, max_new=8)
+    rng = np.random.default_rng(24)
+    from synth.workload import Request
+    reqs = [Request(t, 0.0, rng.integers(0, model.vocab, size=int(p)).astype(np.int32), 8)
+            for t, p in enumerate([300, 40, 129, 257, 16, 310])]
+    w = make_weights(model, 79, "cpu", random_gains=True)
+    runs = {}
+    for name, mode in (("persistent", B.EXEC_PERSISTENT), ("stepped", B.EXEC_STEPPED)):
+        runs[name] = compare_with_oracle(model, sched, reqs, w, TOL_BF16, gemm_impl=B.GEMM_AUTO,
+                                         weights_layout=B.WEIGHTS_STREAMING, exec_mode=mode)
+        assert runs[name]["err_plain"] <= TOL_BF16
+    a, b = runs["persistent"], runs["stepped"]
+    assert_traces_equal([{**r, "sampled": []} for r in a["trace"]], [{**r, "sampled": []} for r in b["trace"]])
+    d = float(np.abs(a["logits"] - b["logits"]).max())
+    print(f"bf16 persistent vs stepped: max-abs logit difference {d:.3e} (vs oracle {a['err']:.3e} / {b['err']:.3e})")
+    assert d <= TOL_BF16
