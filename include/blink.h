@@ -62,7 +62,10 @@ enum { BLINK_DTYPE_BF16 = 0, BLINK_DTYPE_FP32 = 1 };
  *     16-byte chunk c (columns 8 c .. 8 c + 7) sits at chunk position c ^ (r % 8): the operand
  *     image the tensor cores read from shared memory, so a weight tile reaches the SM as one
  *     contiguous 16 KiB copy and every SM streams long sequential runs of HBM.  Requires every
- *     matrix to have a multiple of 128 rows per layer and a multiple of 64 columns.
+ *     matrix to have a multiple of 128 rows per layer and a multiple of 64 columns.  The rows of
+ *     each gate/up matrix (tensor 3) are first interleaved: stored row 2 f is gate row f and
+ *     stored row 2 f + 1 is up row f, so one tile holds both halves of 64 features and the GEMM
+ *     that owns all of a tile's K writes silu(gate) * up itself.
  * blink_convert_weights switches a buffer between the two, in place. */
 enum { BLINK_WEIGHTS_ROW_MAJOR = 0, BLINK_WEIGHTS_STREAMING = 1 };
 
@@ -247,7 +250,7 @@ uint64_t blink_weight_offset(const blink_model_cfg* cfg, int tensor_id);
 /* Convert the GEMM matrices of `weights` (DEVICE, caller-owned, blink_weights_bytes(cfg) bytes)
  * in place from cfg->weights_layout to `to_layout`.  Part of set-up (the provisioning plane of
  * Section 4.1: the host prepares the engine once, then leaves the inference path).  Synchronous;
- * uses a temporary device scratch of one 128-row panel per SM.  BLINK_EINVAL when the shape does
+ * uses temporary device scratch of one 128-row panel per SM and of one gate/up matrix.  BLINK_EINVAL when the shape does
  * not admit the streaming layout or the dtype is not bf16; a no-op when the layouts are equal.
  * No context may be using the buffer meanwhile. */
 int blink_convert_weights(const blink_model_cfg* cfg, void* weights, int to_layout);

@@ -76,6 +76,20 @@ __global__ void __launch_bounds__(256) blink_retile_kernel(char* base, long long
   }
 }
 
+// Row permutation of one gate/up matrix ([2F][K], gate rows first): the streaming layout stores it with
+// gate row f and up row f adjacent (rows 2f and 2f + 1), so that one 128-row weight tile holds both
+// halves of 64 features and the GEMM epilogue can form silu(gate) * up from one accumulator.
+__global__ void __launch_bounds__(256) blink_interleave_rows_kernel(uint4* __restrict__ dst, const uint4* __restrict__ src,
+                                                                    long long F, int cpr, int interleave) {
+  const long long total = 2 * F * cpr;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+    const long long r = i / cpr;
+    const int cc = (int)(i - r * cpr);
+    const long long sr = interleave ? ((r & 1) * F + (r >> 1)) : (r < F ? 2 * r : 2 * (r - F) + 1);
+    dst[i] = src[sr * cpr + cc];
+  }
+}
+
 __global__ void blink_clock_probe_kernel(Mailbox* mb) {
   mb->clock_probe = global_timer_ns();
   __threadfence_system();
@@ -357,14 +371,31 @@ int blink_convert_weights(const blink_model_cfg* cfg, void* weights, int to_layo
   char* scratch = nullptr;
   if (cudaMalloc(&scratch, (size_t)sms * 128 * max_k * 2) != cudaSuccess) return BLINK_ENOMEM;
   const Layout lo = weight_layout(cfg);
+  const bool to_streaming = to_layout == BLINK_WEIGHTS_STREAMING;
+  const size_t gu_bytes = (size_t)2 * F * d * 2;
+  char* gu_tmp = nullptr;
+  if (cudaMalloc(&gu_tmp, gu_bytes) != cudaSuccess) { cudaFree(scratch); return BLINK_ENOMEM; }
   int rc = BLINK_OK;
+  // gate/up rows are interleaved in the streaming layout: permute each [2F][d] matrix while it is row-major
+  auto permute_gate_up = [&]() {
+    for (long long m = 0; m < L * E1 && rc == BLINK_OK; ++m) {
+      char* mat = static_cast<char*>(weights) + lo.off[3] + (size_t)m * gu_bytes;
+      if (cudaMemcpyAsync(gu_tmp, mat, gu_bytes, cudaMemcpyDeviceToDevice, 0) != cudaSuccess) rc = BLINK_ECUDA;
+      blink_interleave_rows_kernel<<<sms * 8, 256>>>(reinterpret_cast<uint4*>(mat), reinterpret_cast<const uint4*>(gu_tmp), F,
+                                                     (int)(d / 8), to_streaming);
+      if (cudaGetLastError() != cudaSuccess) rc = BLINK_ECUDA;
+    }
+  };
+  if (to_streaming) permute_gate_up();
   for (int i = 0; i < 5 && rc == BLINK_OK; ++i) {
     blink_retile_kernel<<<sms, 256>>>(static_cast<char*>(weights) + lo.off[ids[i]], rows_tot[i] / 128, (int)cols[i], scratch,
-                                      to_layout == BLINK_WEIGHTS_STREAMING);
+                                      to_streaming);
     if (cudaGetLastError() != cudaSuccess) rc = BLINK_ECUDA;
   }
+  if (!to_streaming) permute_gate_up();
   if (cudaDeviceSynchronize() != cudaSuccess) rc = BLINK_ECUDA;
   cudaFree(scratch);
+  cudaFree(gu_tmp);
   return rc;
 }
 
@@ -650,6 +681,10 @@ int blink_create(const blink_model_cfg* model, const blink_sched_cfg* sched, con
     }
     TRY(dev_alloc(x, &p, MB * c.d * esz)); c.xs = p;
     TRY(dev_alloc(x, &c.rowss_a, TM)); TRY(dev_alloc(x, &c.rowss_b, TM)); TRY(dev_alloc(x, &c.tile_cnt, (size_t)TILE_CNT_SLOTS));
+    // one stamp per (256-row token pass, gate/up weight tile); the SwiGLU phase lists the units in shared memory
+    const size_t gu_units = ((TM + 255) / 256) * (size_t)((c.F + 63) / 64);
+    c.gu_direct = c.w_streaming && c.gemm_tc && c.E == 0 && !c.fused && gu_units <= 32768;
+    TRY(dev_alloc(x, &c.gu_done, gu_units));
     TRY(dev_alloc(x, &c.logits, MB * c.V));
     TRY(dev_alloc(x, &c.rope_cos, (size_t)c.max_pos * (c.hd / 2), false));
     TRY(dev_alloc(x, &c.rope_sin, (size_t)c.max_pos * (c.hd / 2), false));

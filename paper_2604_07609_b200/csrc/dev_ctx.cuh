@@ -199,6 +199,8 @@ struct DevCtx {
   float* rowss_b;      // [Tmax] the same after the down GEMM (input of the next layer's first norm / the final norm)
   int32_t* tile_cnt;   // [TILE_CNT_SLOTS] k-blocks delivered per output tile of the running GEMM; self-resetting
   int fused;           // 1: RoPE + KV write and SwiGLU run in the epilogues of the QKV and gate/up GEMMs
+  int gu_direct;       // 1: gate/up tiles whose sums are complete in one accumulator are written as activations by the GEMM
+  int32_t* gu_done;    // [token passes][gate/up weight tiles] stamp (iteration * L + layer + 1) of the last such write
   int fused_norm;      // 1: the O and down epilogues add up sum(x^2) per row and the norms are element-wise
   float* logits;  // [MB][V]
   float *rope_cos, *rope_sin;  // [max_pos][hd/2]

@@ -491,10 +491,10 @@ __device__ __noinline__ void fixup_rope_kv(const DevCtx& c, int layer, int nt, i
 
 // gate tile j and up tile j of rows [t0, t1) of `gu` (row pitch 2F): act = silu(gate) * up; both cleared.
 template <typename WT>
-__device__ __noinline__ void fixup_silu(float* gu, WT* act, int F, int j, int t0, int t1) {
+__device__ __noinline__ void fixup_silu(float* gu, WT* act, int F, int f0, int width, int t0, int t1) {
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-  const int f = j * 128 + lane * 4;
-  if (f >= F) return;
+  const int f = f0 + lane * 4;
+  if (lane * 4 >= width || f >= F) return;
   for (int tb = t0 + w; tb < t1; tb += FIX_WARPS * FIX_U) {
     float4 g[FIX_U], u4[FIX_U];
 #pragma unroll
@@ -679,6 +679,15 @@ constexpr int ATTN_SMEM_FLOATS(int HD, int NREP) { return NREP * HD + 2 * 8 * NR
 // SILU_U items in flight before it stores.  A function of its own: inlined into the loop kernel
 // the buffers of loaded values end up in local memory.
 template <typename WT>
+__device__ __forceinline__ void silu_store(float* gu, WT* out, int t, int j, int F, const float4& g, const float4& u, bool clear) {
+  store4<WT>(out + (size_t)t * F + j, g.x / (1.0f + __expf(-g.x)) * u.x, g.y / (1.0f + __expf(-g.y)) * u.y,
+             g.z / (1.0f + __expf(-g.z)) * u.z, g.w / (1.0f + __expf(-g.w)) * u.w);
+  if (clear) {   // consumed: the next split-K gate/up GEMM adds partial sums into a cleared buffer
+    __stcg(reinterpret_cast<float4*>(gu + (size_t)t * 2 * F + j), make_float4(0.f, 0.f, 0.f, 0.f));
+    __stcg(reinterpret_cast<float4*>(gu + (size_t)t * 2 * F + F + j), make_float4(0.f, 0.f, 0.f, 0.f));
+  }
+}
+template <typename WT>
 __device__ __noinline__ void silu_mul_rows(float* __restrict__ gu, WT* __restrict__ out, int T, int F, bool clear) {
   constexpr int SILU_U = 4;
   const int F4 = F / 4;
@@ -697,22 +706,89 @@ __device__ __noinline__ void silu_mul_rows(float* __restrict__ gu, WT* __restric
     for (int k = 0; k < SILU_U; ++k) {
       const int idx = base + k * stride;
       if (idx < total) {
-        const int t = idx / F4, j = (idx - t * F4) * 4;
-        store4<WT>(out + (size_t)t * F + j, g[k].x / (1.0f + __expf(-g[k].x)) * u[k].x,
-                   g[k].y / (1.0f + __expf(-g[k].y)) * u[k].y, g[k].z / (1.0f + __expf(-g[k].z)) * u[k].z,
-                   g[k].w / (1.0f + __expf(-g[k].w)) * u[k].w);
-        if (clear) {   // consumed: the next split-K gate/up GEMM adds partial sums into a cleared buffer
-          __stcg(reinterpret_cast<float4*>(gu + (size_t)t * 2 * F + j), make_float4(0.f, 0.f, 0.f, 0.f));
-          __stcg(reinterpret_cast<float4*>(gu + (size_t)t * 2 * F + F + j), make_float4(0.f, 0.f, 0.f, 0.f));
-        }
+        const int t = idx / F4;
+        silu_store<WT>(gu, out, t, (idx - t * F4) * 4, F, g[k], u[k], clear);
       }
     }
   }
 }
+// The same over the (token pass, gate/up weight tile) units that the GEMM has not already written as
+// activations (a unit is up to 256 rows x 64 features; the GEMM stamps the units it wrote).  Every CTA
+// compacts the pending units into shared memory once, then all threads of the grid share their items evenly.
+static __device__ __noinline__ int silu_pending_units(const int* done, int stamp, int n_units, int* list) {
+  __shared__ int s_warp[FWD_THREADS / 32];
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  int count = 0;   // uniform over the CTA
+  for (int b0 = 0; b0 < n_units; b0 += FWD_THREADS) {
+    const int unit = b0 + threadIdx.x;
+    const bool pend = unit < n_units && __ldcg(done + unit) != stamp;   // written by other SMs: not through L1
+    const unsigned m = __ballot_sync(0xffffffffu, pend);
+    if (lane == 0) s_warp[w] = __popc(m);
+    __syncthreads();
+    int off = count, tot = 0;
+#pragma unroll
+    for (int i = 0; i < FWD_THREADS / 32; ++i) {
+      if (i < w) off += s_warp[i];
+      tot += s_warp[i];
+    }
+    if (pend) list[off + __popc(m & ((1u << lane) - 1u))] = unit;
+    count += tot;
+    __syncthreads();
+  }
+  return count;
+}
+// A CTA takes a quarter of a pending unit at a time: 64 rows x 64 features, four items per thread.  The
+// loads are asynchronous copies into a staging area in shared memory (each thread reads back only what it
+// copied itself), so four items are in flight per thread without holding registers for them: a body that
+// needs many registers here changes the register allocation of the other phase functions of the loop
+// kernel, to their cost.
+constexpr int SILU_STAGE_OFF = 32768 * 4;   // bytes: the staging area follows the list of pending units
 template <typename WT>
-static __device__ __noinline__ void phase_silu_mul(const DevCtx& c) {
+__device__ __noinline__ void silu_mul_pending(float* __restrict__ gu, WT* __restrict__ out, int T, int F, const int* list, int count) {
+  const int tiles = F >> 6;
+  const int r_in = threadIdx.x >> 4, col = (threadIdx.x & 15) << 2;
+  const char* stage = reinterpret_cast<const char*>(list) + SILU_STAGE_OFF + threadIdx.x * 16;   // [8][FWD_THREADS] x 16 bytes
+  const uint32_t stage_s = (uint32_t)__cvta_generic_to_shared(stage);
+  for (int q = blockIdx.x; q < count * 4; q += gridDim.x) {
+    const int unit = list[q >> 2];
+    const int pass = unit / tiles, tile = unit - pass * tiles;
+    const int row0 = (pass << 8) + ((q & 3) << 6) + r_in, j = (tile << 6) + col;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int t = row0 + 16 * k;
+      if (t < T) {
+        const float* src = gu + (size_t)t * 2 * F + j;
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(stage_s + (2 * k) * FWD_THREADS * 16), "l"(src) : "memory");
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(stage_s + (2 * k + 1) * FWD_THREADS * 16), "l"(src + F) : "memory");
+      }
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int t = row0 + 16 * k;
+      if (t < T) {
+        const float4 g = *reinterpret_cast<const float4*>(stage + (2 * k) * FWD_THREADS * 16);
+        const float4 u = *reinterpret_cast<const float4*>(stage + (2 * k + 1) * FWD_THREADS * 16);
+        silu_store<WT>(gu, out, t, j, F, g, u, true);
+      }
+    }
+  }
+}
+// The GEMM writes activations itself only in steps of more than one token pass: there its epilogue hides
+// behind the tensor-core work of the next tile, while at decode sizes the GEMM is bound by the weight
+// stream and the longer epilogue would show.
+__device__ __forceinline__ bool gu_direct_step(const DevCtx& c, int T) { return c.gu_direct && T > 256; }
+template <typename WT>
+static __device__ __noinline__ void phase_silu_mul(const DevCtx& c, int layer, float* smem) {
   const int T = c.E > 0 ? c.ss->cur_T * c.topE : c.ss->cur_T;   // rows of the gate/up buffer
-  if (T > 0) silu_mul_rows<WT>(c.gu, reinterpret_cast<WT*>(c.act), T, c.F, c.gemm_tc != 0);
+  if (T <= 0) return;
+  if (gu_direct_step(c, T)) {
+    int* list = reinterpret_cast<int*>(smem);
+    const int count = silu_pending_units(c.gu_done, (int)(c.ss->iter * (unsigned long long)c.L) + layer + 1, ((T + 255) >> 8) * (c.F >> 6), list);
+    silu_mul_pending<WT>(c.gu, reinterpret_cast<WT*>(c.act), T, c.F, list, count);
+  } else
+    silu_mul_rows<WT>(c.gu, reinterpret_cast<WT*>(c.act), T, c.F, c.gemm_tc != 0);
 }
 
 // ---- routed experts: group the (token, expert) pairs by expert and gather their rows ---------

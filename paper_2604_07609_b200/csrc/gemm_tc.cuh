@@ -346,6 +346,8 @@ struct TcEpiOut {
   const int* row_map;
   const float* row_scale;
   int T, N;
+  int ilv_F;               // gate/up rows interleaved in the weight tiles: row n is output column (n & 1) * F + (n >> 1)
+  __nv_bfloat16* act;      // non-null: a tile whose sums are complete goes straight to act = silu(gate) * up
 };
 // columns [c_begin, c_end) of an accumulator (token rows t_base + column) -> out; lane = weight row n
 __device__ __forceinline__ void tc_epi_columns(const TcEpiOut& e, uint32_t taddr, int n, int t_base, int c_begin, int c_end,
@@ -356,12 +358,13 @@ __device__ __forceinline__ void tc_epi_columns(const TcEpiOut& e, uint32_t taddr
     if (n < e.N) {
       const int t0 = t_base + c0;
       const int nv = min(16, e.T - t0);   // token rows of this group that exist
+      const int n_out = e.ilv_F ? (n & 1) * e.ilv_F + (n >> 1) : n;
       if (e.row_map != nullptr) {
 #pragma unroll
         for (int j = 0; j < 16; ++j)
-          if (j < nv) red_add_f32(e.out + (size_t)e.row_map[t0 + j] * e.ldo + n, e.row_scale[t0 + j] * v[j]);
+          if (j < nv) red_add_f32(e.out + (size_t)e.row_map[t0 + j] * e.ldo + n_out, e.row_scale[t0 + j] * v[j]);
       } else {
-        float* o = e.out + (size_t)t0 * e.ldo + n;
+        float* o = e.out + (size_t)t0 * e.ldo + n_out;
         if (plain) {
 #pragma unroll
           for (int j = 0; j < 16; ++j)
@@ -375,6 +378,36 @@ __device__ __forceinline__ void tc_epi_columns(const TcEpiOut& e, uint32_t taddr
     }
   }
 }
+// Gate/up tile whose K is complete in this accumulator (rows interleaved: lane 2 i holds the gate row and lane
+// 2 i + 1 the up row of feature n / 2): the pair of lanes exchanges its values and writes
+// act = silu(gate) * up in the operand type, eight of the sixteen token columns each.  Nothing goes to the
+// fp32 gate/up buffer and the SwiGLU phase skips the tile.
+__device__ __forceinline__ void tc_epi_silu(const TcEpiOut& e, uint32_t taddr, int n, int t_base, int c_begin, int c_end) {
+  const bool even = (n & 1) == 0;
+  const int f = n >> 1;
+  const int F = e.ilv_F;
+  for (int c0 = c_begin; c0 < c_end; c0 += 16) {
+    float v[16], o[16];
+    tmem_ld16(taddr + (uint32_t)c0, v);
+#pragma unroll
+    for (int j = 0; j < 16; ++j) o[j] = __shfl_xor_sync(0xffffffffu, v[j], 1);
+    if (n < e.N) {
+      const int t0 = t_base + c0;
+      const int nv = min(16, e.T - t0);
+#pragma unroll
+      for (int jj = 0; jj < 8; ++jj) {
+        const int j = even ? jj : jj + 8;
+        const float g = even ? v[jj] : o[jj + 8];
+        const float u = even ? o[jj] : v[jj + 8];
+        // approximate division (2 ulp before the rounding to bf16): the exact one is a call to a subroutine,
+        // which costs every phase of the loop kernel, not only this one
+        if (j < nv) e.act[(size_t)(t0 + j) * F + f] = __float2bfloat16_rn(__fdividef(g, 1.0f + __expf(-g)) * u);
+      }
+    }
+  }
+}
+// what the gate/up GEMM of this step and layer writes beside a tile it has turned into activations
+__device__ __forceinline__ int gu_stamp(const DevCtx& c, int layer) { return (int)(c.ss->iter * (unsigned long long)c.L) + layer + 1; }
 // First column of a CTA's last accumulator that warps 0-3 store (they have no role left by
 // then).  Below 128 columns the reduction is short and the extra waiting warps cost more.
 __device__ __forceinline__ int tc_epi_half(int n_mma) { return n_mma >= 128 ? ((n_mma / 16 + 1) / 2) * 16 : n_mma; }
@@ -522,8 +555,11 @@ static __device__ __noinline__ void tc_finish_tiles(const DevCtx& c, const GemmA
   __shared__ int s_fin[BATCH];
   __shared__ int s_nfin;
   __shared__ long long s_next;
-  const int ntiles_slot = a.fix == FIX_SILU ? g.ntiles / 2 : g.ntiles;   // gate tile j and up tile j share slot j
-  const int need = (a.fix == FIX_SILU ? 2 : 1) * g.kblocks;
+  // gate/up: with plain rows gate tile j and up tile j + ntiles / 2 share slot j; with interleaved rows one
+  // weight tile holds gate and up of 64 features
+  const bool two_tiles = a.fix == FIX_SILU && !c.w_streaming;
+  const int ntiles_slot = two_tiles ? g.ntiles / 2 : g.ntiles;
+  const int need = (two_tiles ? 2 : 1) * g.kblocks;
   long long u = g.u0;
   while (u < g.u1) {   // uniform over the CTA
     if (threadIdx.x == 0) {
@@ -553,7 +589,7 @@ static __device__ __noinline__ void tc_finish_tiles(const DevCtx& c, const GemmA
       const int tile = s_fin[i] & 0xffff, pass = s_fin[i] >> 16;
       const int t0 = pass * 256, t1 = min(a.M, t0 + 256);
       if (a.fix == FIX_ROPE_KV) fixup_rope_kv<__nv_bfloat16>(c, layer, tile, t0, t1);
-      else if (a.fix == FIX_SILU) fixup_silu<__nv_bfloat16>(a.out, reinterpret_cast<__nv_bfloat16*>(a.fix_out), a.N / 2, tile, t0, t1);
+      else if (a.fix == FIX_SILU) fixup_silu<__nv_bfloat16>(a.out, reinterpret_cast<__nv_bfloat16*>(a.fix_out), a.N / 2, two_tiles ? tile * 128 : tile * 64, two_tiles ? 128 : 64, t0, t1);
       else fixup_sumsq(a.out, a.ldo, a.N, a.fix_rowss, tile, t0, t1);
     }
     __syncthreads();
@@ -564,6 +600,10 @@ template <bool PAIR>
 static __device__ __noinline__ void phase_gemm_tc(const DevCtx& c, const GemmArgs& a, int which, int layer, float* smem_f, TcState& tc) {
   const int T = a.M, N = a.N, K = a.K;
   if (T <= 0) return;  // uniform over the grid
+  // gate/up on the streaming layout: weight rows are interleaved (gate f, up f, ...), and in a dense model
+  // a tile whose sums are complete in one accumulator goes straight to the activation rows
+  const int ilv_F = (which == GEMM_GU && c.w_streaming) ? c.F : 0;
+  __nv_bfloat16* const act_direct = (which == GEMM_GU && gu_direct_step(c, T)) ? reinterpret_cast<__nv_bfloat16*>(c.act) : nullptr;
   const TcMaps* maps = reinterpret_cast<const TcMaps*>(c.tc_maps);
   const uint32_t rank = PAIR ? cluster_ctarank() : 0u;
   const int n_tiles128 = (N + 127) / 128;
@@ -673,7 +713,7 @@ static __device__ __noinline__ void phase_gemm_tc(const DevCtx& c, const GemmArg
     }
   } else if (warp >= 4) {
     const int q = warp & 3;  // TMEM lane quarter this warp may read
-    const TcEpiOut eo{a.out, (size_t)a.ldo, a.row_map, a.row_scale, T, N};
+    const TcEpiOut eo{a.out, (size_t)a.ldo, a.row_map, a.row_scale, T, N, ilv_F, act_direct};
     const bool accumulate = a.accumulate != 0;
     int abuf = 0;
     long long u = u0;
@@ -692,7 +732,12 @@ static __device__ __noinline__ void phase_gemm_tc(const DevCtx& c, const GemmArg
       const uint32_t taddr = tc.tmem_base + (uint32_t)abuf * 256u + ((uint32_t)(q * 32) << 16);
       // the upper columns of the CTA's last accumulator are left to warps 0-3
       const int c_end = (seg_end == u1) ? tc_epi_half(n_mma) : n_mma;
-      tc_epi_columns(eo, taddr, nt * 128 + q * 32 + lane, pass * 256, 0, c_end, plain);
+      if (plain && eo.act != nullptr) {
+        tc_epi_silu(eo, taddr, nt * 128 + q * 32 + lane, pass * 256, 0, c_end);
+        if (q == 0 && lane == 0 && nt * 128 < N) c.gu_done[pass * ((N + 127) / 128) + nt] = gu_stamp(c, layer);   // read after the grid barrier
+      } else {
+        tc_epi_columns(eo, taddr, nt * 128 + q * 32 + lane, pass * 256, 0, c_end, plain);
+      }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) {
@@ -725,10 +770,11 @@ static __device__ __noinline__ void phase_gemm_tc(const DevCtx& c, const GemmArg
       // every thread waits (also when it has no columns to store) so that its parity stays in step
       if (mbar_wait_idle(c, &g_tc.acc_last, par, dead) && c_begin < n_mma) {
         tc_fence_after();
-        const TcEpiOut eo{a.out, (size_t)a.ldo, a.row_map, a.row_scale, T, N};
+        const TcEpiOut eo{a.out, (size_t)a.ldo, a.row_map, a.row_scale, T, N, ilv_F, act_direct};
         const bool plain = (kb0 == 0 && (long long)kb0 + (u1 - last_u) == kblocks) && a.accumulate == 0 && eo.row_map == nullptr;
         const uint32_t taddr = tc.tmem_base + (uint32_t)last_abuf * 256u + ((uint32_t)(warp * 32) << 16);
-        tc_epi_columns(eo, taddr, nt * 128 + warp * 32 + lane, pass * 256, c_begin, n_mma, plain);
+        if (plain && eo.act != nullptr) tc_epi_silu(eo, taddr, nt * 128 + warp * 32 + lane, pass * 256, c_begin, n_mma);
+        else tc_epi_columns(eo, taddr, nt * 128 + warp * 32 + lane, pass * 256, c_begin, n_mma, plain);
         tc_fence_before();
       }
     }

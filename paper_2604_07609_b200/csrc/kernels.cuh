@@ -73,7 +73,7 @@ __device__ __forceinline__ void run_phase(const DevCtx& c, int phase, int layer,
       }
     } break;
     case PH_SILU:
-      phase_silu_mul<WT>(c);
+      phase_silu_mul<WT>(c, layer, smem);
       break;
     case PH_DOWN: {
       if (c.E == 0) {

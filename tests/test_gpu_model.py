@@ -184,6 +184,14 @@ def test_streaming_weight_layout_round_trip_and_parity(gemm):
     for r in (0, 1, 7, 8, 77, 127):
         for c8 in range(8):
             assert torch.equal(tile[r, c8 ^ (r & 7)], rm[r, c8])
+    # gate/up: stored row 2 f is gate row f, stored row 2 f + 1 is up row f
+    off3, F = B.blink_weight_offset(model, 3), model.d_ff
+    tile = wd[off3:off3 + 16384].cpu().view(torch.bfloat16).view(128, 8, 8)
+    rm3 = w[off3:off3 + 2 * F * K * 2].view(torch.bfloat16).view(2 * F, K)
+    for r in (0, 1, 2, 9, 126, 127):
+        src = rm3[(r & 1) * F + (r >> 1), :64].reshape(8, 8)
+        for c8 in range(8):
+            assert torch.equal(tile[r, c8 ^ (r & 7)], src[c8])
     err, _, trace, toks, ora = _compare(model, sched, reqs, w, O2.round_bf16, TOL_BF16, gemm_impl=gemm,
                                         weights_layout=B.WEIGHTS_STREAMING)
     print(f"streaming layout: max-abs logit error {err:.3e}")
