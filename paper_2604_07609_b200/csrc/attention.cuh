@@ -322,7 +322,7 @@ __device__ __noinline__ void attn_decode_stream(const DevCtx& c, int layer, char
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
           if (h0 + e < NREP) {
-            const float inv = 1.0f / (e ? lt1 : lt0);
+            const float inv = __fdividef(1.0f, e ? lt1 : lt0);
 #pragma unroll
             for (int i = 0; i < HD / 16; ++i) {
               obase[(h0 + e) * HD + 16 * i + gq] = __float2bfloat16_rn(o[i][e] * inv);
@@ -371,7 +371,7 @@ __device__ __noinline__ void attn_decode_stream(const DevCtx& c, int layer, char
               num.x += f * a4.x; num.y += f * a4.y; num.z += f * a4.z; num.w += f * a4.w;
               den += f * __ldcg(r + NREP * HD + NREP + h);
             }
-            const float inv = 1.0f / den;
+            const float inv = __fdividef(1.0f, den);
             uint2 o2;
             o2.x = pack_bf2(num.x * inv, num.y * inv);
             o2.y = pack_bf2(num.z * inv, num.w * inv);
@@ -547,7 +547,7 @@ __device__ __noinline__ void attn_prefill_tile(const DevCtx& c, int layer, int i
   l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
   const int h = mrow0 / QROWS;   // 16 | QROWS, so a warp's rows belong to one head
   const int r_lo = r_base + (mrow0 + gq) % QROWS, r_hi = r_base + (mrow0 + gq + 8) % QROWS;
-  const float i_lo = 1.0f / l_lo, i_hi = 1.0f / l_hi;
+  const float i_lo = __fdividef(1.0f, l_lo), i_hi = __fdividef(1.0f, l_hi);
 #pragma unroll
   for (int nt = 0; nt < HD / 8; ++nt) {
     const size_t col = (size_t)(g * NREP + h) * HD + nt * 8 + 2 * tq;

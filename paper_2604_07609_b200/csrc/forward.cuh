@@ -121,7 +121,7 @@ __device__ __forceinline__ void norm_row_cta(const DevCtx& c, float* hrow, const
     }
   }
   ss = block_sum(ss, s_red);
-  const float inv = 1.0f / sqrtf(ss / (float)d + c.rms_eps);
+  const float inv = rsqrtf(__fdividef(ss, (float)d) + c.rms_eps);
 #pragma unroll
   for (int k = 0; k < NORM_MAXV; ++k) {
     const int i = (k * FWD_THREADS + threadIdx.x) * 4;
@@ -214,7 +214,7 @@ __device__ __noinline__ void norm_apply_rows(const float* __restrict__ h, const 
   constexpr int U = 4;   // items whose loads are in flight before the first store (one CTA per SM: latency-bound otherwise)
   const int d4 = d >> 2;
   const int total = R * d4;   // < 2^31
-  const float inv_d = 1.0f / (float)d;
+  const float inv_d = __fdividef(1.0f, (float)d);
   const int stride = gridDim.x * FWD_THREADS;
   for (int base = blockIdx.x * FWD_THREADS + threadIdx.x; base < total; base += U * stride) {
     float4 v[U], gg[U];
@@ -233,7 +233,7 @@ __device__ __noinline__ void norm_apply_rows(const float* __restrict__ h, const 
 #pragma unroll
     for (int k = 0; k < U; ++k) {
       if (base + k * stride < total) {
-        const float inv = 1.0f / sqrtf(ss[k] * inv_d + eps);
+        const float inv = rsqrtf(ss[k] * inv_d + eps);
         store4<WT>(out + (size_t)r[k] * d + j[k], v[k].x * inv * gg[k].x, v[k].y * inv * gg[k].y, v[k].z * inv * gg[k].z,
                    v[k].w * inv * gg[k].w);
       }
@@ -507,8 +507,8 @@ __device__ __noinline__ void fixup_silu(float* gu, WT* act, int F, int f0, int w
     for (int u = 0; u < FIX_U; ++u) {
       const int t = tb + u * FIX_WARPS;
       if (t >= t1) continue;
-      store4<WT>(act + (size_t)t * F + f, g[u].x / (1.0f + __expf(-g[u].x)) * u4[u].x, g[u].y / (1.0f + __expf(-g[u].y)) * u4[u].y,
-                 g[u].z / (1.0f + __expf(-g[u].z)) * u4[u].z, g[u].w / (1.0f + __expf(-g[u].w)) * u4[u].w);
+      store4<WT>(act + (size_t)t * F + f, __fdividef(g[u].x, 1.0f + __expf(-g[u].x)) * u4[u].x, __fdividef(g[u].y, 1.0f + __expf(-g[u].y)) * u4[u].y,
+                 __fdividef(g[u].z, 1.0f + __expf(-g[u].z)) * u4[u].z, __fdividef(g[u].w, 1.0f + __expf(-g[u].w)) * u4[u].w);
       __stcg(reinterpret_cast<float4*>(gu + (size_t)t * 2 * F + f), make_float4(0.f, 0.f, 0.f, 0.f));
       __stcg(reinterpret_cast<float4*>(gu + (size_t)t * 2 * F + F + f), make_float4(0.f, 0.f, 0.f, 0.f));
     }
@@ -678,10 +678,12 @@ constexpr int ATTN_SMEM_FLOATS(int HD, int NREP) { return NREP * HD + 2 * 8 * NR
 // and one CTA per SM leaves eight warps to cover that latency, so every thread has the loads of
 // SILU_U items in flight before it stores.  A function of its own: inlined into the loop kernel
 // the buffers of loaded values end up in local memory.
+// silu(g) * u with the approximate division (2 ulp, then rounded to the operand type): the exact fp32 division
+// took a quarter of the SwiGLU phase
 template <typename WT>
 __device__ __forceinline__ void silu_store(float* gu, WT* out, int t, int j, int F, const float4& g, const float4& u, bool clear) {
-  store4<WT>(out + (size_t)t * F + j, g.x / (1.0f + __expf(-g.x)) * u.x, g.y / (1.0f + __expf(-g.y)) * u.y,
-             g.z / (1.0f + __expf(-g.z)) * u.z, g.w / (1.0f + __expf(-g.w)) * u.w);
+  store4<WT>(out + (size_t)t * F + j, __fdividef(g.x, 1.0f + __expf(-g.x)) * u.x, __fdividef(g.y, 1.0f + __expf(-g.y)) * u.y,
+             __fdividef(g.z, 1.0f + __expf(-g.z)) * u.z, __fdividef(g.w, 1.0f + __expf(-g.w)) * u.w);
   if (clear) {   // consumed: the next split-K gate/up GEMM adds partial sums into a cleared buffer
     __stcg(reinterpret_cast<float4*>(gu + (size_t)t * 2 * F + j), make_float4(0.f, 0.f, 0.f, 0.f));
     __stcg(reinterpret_cast<float4*>(gu + (size_t)t * 2 * F + F + j), make_float4(0.f, 0.f, 0.f, 0.f));
