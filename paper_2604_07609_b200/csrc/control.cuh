@@ -616,7 +616,10 @@ static __device__ int schedule_step(const DevCtx& c, unsigned long long visible)
       const long long cap = n_pf > 0 ? 48 : 96;
       const long long k = (TT + cap * NW - 1) / (cap * NW) > 1 ? (TT + cap * NW - 1) / (cap * NW) : 1;
       long long S = (TT + k * NW - 1) / (k * NW);
-      if (S < 1) S = 1;
+      // at least 8 tiles per sub-range: a cut costs a partial record, a fence and a counter update (about the time of
+      // two tiles), and a unit cut into n parts is merged by one warp in n steps; with few long rows one tile per
+      // sub-range made a single 2048-token row take 120 us per layer, most of it the merge
+      if (S < 8) S = 8;
       while ((TT + S - 1) / S > c.att_sub_max) S *= 2;   // cannot happen with the sizes set at create
       c.dec_kbpre[n_dec_att] = tot_kb;
       ss->cur_ndec = n_dec_att;
