@@ -232,6 +232,40 @@ def test_decode_attention_many_rows_whole_and_split_units():
           f"{max(sum(s[4] for s in r['scheduled']) for r in trace)}")
 
 
+def test_decode_attention_few_long_rows():
+    """Two requests with contexts of 1200 and 1900 tokens: fewer tiles than warps, so every (row, kv head)
+    unit is cut into sub-ranges of the minimum size and merged from more than ten partial records."""
+    model = model_cfg(1, dtype="bf16")
+    sched = sched_cfg(1, prefill_chunk_tokens=512, max_batch=8, n_blocks=512, max_prompt=2048, max_new=6)
+    rng = np.random.default_rng(9)
+    from synth.workload import Request
+    reqs = [Request(t, 0.0, rng.integers(0, model.vocab, size=int(p)).astype(np.int32), 5)
+            for t, p in enumerate([1900, 1200])]
+    w = make_weights(model, 12, "cpu", random_gains=True)
+    err, _, trace, toks, ora = _compare(model, sched, reqs, w, O2.round_bf16, TOL_BF16)
+    print(f"2 rows, contexts 1200 and 1900: max-abs logit error {err:.3e}")
+    assert err <= TOL_BF16
+
+
+@pytest.mark.parametrize("gemm", [B.GEMM_TC, B.GEMM_TC_PAIR], ids=["single-cta", "cta-pairs"])
+def test_gate_up_epilogue_writes_activations_three_ragged_passes(gemm):
+    """Streaming layout, more than 512 rows in a step: three token passes, the last one ragged.  The
+    gate/up GEMM writes silu(gate) * up itself for the (pass, tile) units whose K it covers in one segment
+    and adds partial sums for the others; the SwiGLU phase takes exactly the others."""
+    model = model_cfg(1, d_model=512, n_q_heads=4, n_kv_heads=1, head_dim=128, d_ff=1536, vocab=4480, dtype="bf16")
+    sched = sched_cfg(1, prefill_chunk_tokens=600, max_batch=8, n_blocks=512, max_prompt=640, max_new=8)
+    rng = np.random.default_rng(23)
+    from synth.workload import Request
+    reqs = [Request(t, 0.0, rng.integers(0, model.vocab, size=int(p)).astype(np.int32), 5)
+            for t, p in enumerate([610, 33, 580, 300, 7])]
+    w = make_weights(model, 79, "cpu", random_gains=True)
+    err, _, trace, toks, ora = _compare(model, sched, reqs, w, O2.round_bf16, TOL_BF16, gemm_impl=gemm,
+                                        weights_layout=B.WEIGHTS_STREAMING)
+    rows = max(sum(s[4] for s in r["scheduled"]) for r in trace)
+    print(f"three passes, streaming layout: max-abs logit error {err:.3e}; max rows/step {rows}")
+    assert err <= TOL_BF16 and rows > 512
+
+
 # ---- top-p (nucleus) sampling ------------------------------------------------------------------------
 def test_top_p_sampler_alone_bit_exact_on_oracle_logits():
     """The nucleus sampler on given logits must pick the oracle's token, row for row: whole-vocabulary
