@@ -200,7 +200,7 @@ struct DevCtx {
   int32_t* tile_cnt;   // [TILE_CNT_SLOTS] k-blocks delivered per output tile of the running GEMM; self-resetting
   int fused;           // 1: RoPE + KV write and SwiGLU run in the epilogues of the QKV and gate/up GEMMs
   int gu_direct;       // 1: gate/up tiles whose sums are complete in one accumulator are written as activations by the GEMM
-  int32_t* gu_done;    // [token passes][gate/up weight tiles] stamp (iteration * L + layer + 1) of the last such write
+  unsigned long long* gu_done;   // [token passes][gate/up weight tiles] stamp (iteration * L + layer + 1, 64 bits: never repeats) of the last such write
   int fused_norm;      // 1: the O and down epilogues add up sum(x^2) per row and the norms are element-wise
   float* logits;  // [MB][V]
   float *rope_cos, *rope_sin;  // [max_pos][hd/2]

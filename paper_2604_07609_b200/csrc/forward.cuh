@@ -717,7 +717,7 @@ __device__ __noinline__ void silu_mul_rows(float* __restrict__ gu, WT* __restric
 // The same over the (token pass, gate/up weight tile) units that the GEMM has not already written as
 // activations (a unit is up to 256 rows x 64 features; the GEMM stamps the units it wrote).  Every CTA
 // compacts the pending units into shared memory once, then all threads of the grid share their items evenly.
-static __device__ __noinline__ int silu_pending_units(const int* done, int stamp, int n_units, int* list) {
+static __device__ __noinline__ int silu_pending_units(const unsigned long long* done, unsigned long long stamp, int n_units, int* list) {
   __shared__ int s_warp[FWD_THREADS / 32];
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   int count = 0;   // uniform over the CTA
@@ -787,7 +787,7 @@ static __device__ __noinline__ void phase_silu_mul(const DevCtx& c, int layer, f
   if (T <= 0) return;
   if (gu_direct_step(c, T)) {
     int* list = reinterpret_cast<int*>(smem);
-    const int count = silu_pending_units(c.gu_done, (int)(c.ss->iter * (unsigned long long)c.L) + layer + 1, ((T + 255) >> 8) * (c.F >> 6), list);
+    const int count = silu_pending_units(c.gu_done, c.ss->iter * (unsigned long long)c.L + (unsigned long long)layer + 1ull, ((T + 255) >> 8) * (c.F >> 6), list);
     silu_mul_pending<WT>(c.gu, reinterpret_cast<WT*>(c.act), T, c.F, list, count);
   } else
     silu_mul_rows<WT>(c.gu, reinterpret_cast<WT*>(c.act), T, c.F, c.gemm_tc != 0);

@@ -407,7 +407,7 @@ __device__ __forceinline__ void tc_epi_silu(const TcEpiOut& e, uint32_t taddr, i
   }
 }
 // what the gate/up GEMM of this step and layer writes beside a tile it has turned into activations
-__device__ __forceinline__ int gu_stamp(const DevCtx& c, int layer) { return (int)(c.ss->iter * (unsigned long long)c.L) + layer + 1; }
+__device__ __forceinline__ unsigned long long gu_stamp(const DevCtx& c, int layer) { return c.ss->iter * (unsigned long long)c.L + (unsigned long long)layer + 1ull; }
 // First column of a CTA's last accumulator that warps 0-3 store (they have no role left by
 // then).  Below 128 columns the reduction is short and the extra waiting warps cost more.
 __device__ __forceinline__ int tc_epi_half(int n_mma) { return n_mma >= 128 ? ((n_mma / 16 + 1) / 2) * 16 : n_mma; }
