@@ -322,10 +322,12 @@ def percentiles(x):
     return dict(p50=float(np.percentile(x, 50)), p99=float(np.percentile(x, 99)), mean=float(np.mean(x)))
 
 
-def realtime_run(B, m, sched, wbuf, kv, reqs, time_limit_s, use_arrivals=True, weights_layout=0):
-    """Persistent loop, requests submitted at their arrival times from host buffers, tokens
-    read back with blink_poll.  Returns throughput and latency figures."""
-    eng = B.Blink(m, sched, wbuf, kv, exec_mode=B.EXEC_PERSISTENT, stats_iters=1 << 17, idle_exit_us=2_000_000,
+def realtime_run(B, m, sched, wbuf, kv, reqs, time_limit_s, use_arrivals=True, weights_layout=0, exec_mode=None):
+    """Persistent loop (or, for the comparison arm, the host-driven loop of the same kernels), requests
+    submitted at their arrival times from host buffers, tokens read back with blink_poll.  Returns
+    throughput and latency figures."""
+    eng = B.Blink(m, sched, wbuf, kv, exec_mode=B.EXEC_PERSISTENT if exec_mode is None else exec_mode,
+                  stats_iters=1 << 17, idle_exit_us=2_000_000,
                   weights_layout=weights_layout, policy=POLICY)
     try:
         off = eng.blink_get_stats().device_clock_offset_ns
@@ -398,6 +400,8 @@ def main():
     ap.add_argument("--steps", type=int, default=30)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="blink", choices=["blink", "reference"])
+    ap.add_argument("--host-driven", default="graph", choices=["off", "graph", "launches"],
+                    help="also run the latency legs with the host-driven loop of the same kernels (comparison arm)")
     ap.add_argument("--config", type=int, default=3, help="BASELINE configuration (1..5)")
     ap.add_argument("--ramp", type=int, default=-1, help="untimed iterations that bring the batch to steady state")
     ap.add_argument("--gemm", default="auto", choices=["auto", "simt", "tc"])
@@ -690,13 +694,14 @@ def main():
                            note="all requests submitted from host memory at t=0 through blink_submit, tokens "
                                 "read with blink_poll, persistent loop; wall clock from first submit")
     # ---- real-time run at the offered load: latency, host idle and host stressed -----------------
-    def latency_leg(stressed, rate_reqs, seconds):
+    def latency_leg(stressed, rate_reqs, seconds, exec_mode=None):
         stress = Stressor() if stressed else None
         if stress:
             stress.start()
         try:
             lreqs = [q for q in rate_reqs if q.arrival_s <= seconds]
-            r = realtime_run(B, m, sched, wbuf, kv, lreqs, seconds * 3, use_arrivals=True, weights_layout=wl)
+            r = realtime_run(B, m, sched, wbuf, kv, lreqs, seconds * 3, use_arrivals=True, weights_layout=wl,
+                             exec_mode=exec_mode)
         finally:
             if stress:
                 stress.stop()
@@ -730,6 +735,28 @@ def main():
                                  ttft_host_p99=ratio(a["ttft_host_ms"]["p99"], b["ttft_host_ms"]["p99"]),
                                  tpot_host_p99=ratio(a["tpot_host_ms"]["p99"], b["tpot_host_ms"]["p99"]))
         line["latency"] = lat
+        # ---- the same kernels driven from the host, idle and stressed (Section 6.3: what interference does to a
+        # host-resident serving loop; the GPU-resident loop above is the other arm) ----
+        if args.host_driven != "off":
+            hmode = B.EXEC_HOST_GRAPH if args.host_driven == "graph" else B.EXEC_HOST_LAUNCHES
+            hl = {}
+            if args.interfere in ("both", "off"):
+                hl["isolated"] = latency_leg(False, reqs, args.latency_seconds, exec_mode=hmode)
+            if args.interfere in ("both", "on"):
+                hl["interfered"] = latency_leg(True, reqs, args.latency_seconds, exec_mode=hmode)
+            for v in hl.values():
+                v.pop("done_s", None)
+            hd = dict(driver="a host thread launches one iteration at a time (" +
+                             ("one pre-captured CUDA graph" if args.host_driven == "graph" else "one kernel launch per phase") +
+                             ") and waits for it; same device code, same requests, same offered load", **hl)
+            if "isolated" in hl and "interfered" in hl:
+                a, b = hl["isolated"], hl["interfered"]
+                ratio = lambda x, y: (y / x) if (x and y) else None
+                hd["ratios"] = dict(ttft_p99=ratio(a["ttft_ms"]["p99"], b["ttft_ms"]["p99"]),
+                                    tpot_p99=ratio(a["tpot_ms"]["p99"], b["tpot_ms"]["p99"]),
+                                    tpot_p50=ratio(a["tpot_ms"]["p50"], b["tpot_ms"]["p50"]),
+                                    throughput=ratio(a["tok_s"], b["tok_s"]))
+            line["host_driven"] = hd
     # ---- offered-load sweep (Section 6.1: 13 levels between 1 and 32 req/s; Appendix C: serviceable load) ----
     if args.rates and rank == 0 and world == 1:
         from synth.workload import RATE_LEVELS

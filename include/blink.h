@@ -73,7 +73,14 @@ enum { BLINK_WEIGHTS_ROW_MAJOR = 0, BLINK_WEIGHTS_STREAMING = 1 };
 enum {
   BLINK_EXEC_PERSISTENT = 0, /* one cooperative kernel loops on the device (product mode)           */
   BLINK_EXEC_STEPPED = 1,    /* same device code, one host launch per phase (profiling, debugging)  */
-  BLINK_EXEC_MANUAL = 2      /* the cooperative loop kernel, launched only by blink_run (measurement) */
+  BLINK_EXEC_MANUAL = 2,     /* the cooperative loop kernel, launched only by blink_run (measurement) */
+  /* Host-driven comparison arms (Section 6.1 baselines keep the host in the loop; Section 6.3 "Interference"):
+   * the same device code as STEPPED, but a thread of the library launches one iteration at a time and waits
+   * for it before it launches the next, as a host-resident serving loop does.  HOST_GRAPH launches the
+   * iteration as one pre-captured CUDA graph, HOST_LAUNCHES as one kernel launch per phase.  blink_submit,
+   * blink_poll and blink_cancel work as in PERSISTENT; blink_step and blink_run are refused. */
+  BLINK_EXEC_HOST_GRAPH = 3,
+  BLINK_EXEC_HOST_LAUNCHES = 4
 };
 
 /* which kernels run the dense contractions */

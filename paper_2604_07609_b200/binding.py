@@ -19,7 +19,7 @@ BLINK_OK, BLINK_EAGAIN, BLINK_EINVAL, BLINK_ESTOPPED, BLINK_EDEVICE = 0, -1, -2,
 BLINK_ETIMEDOUT, BLINK_ENOMEM, BLINK_ECUDA, BLINK_ETOOBIG = -5, -6, -7, -8
 SAMPLE_NOALLOC_MAX_ROWS = 1024
 DTYPE_BF16, DTYPE_FP32 = 0, 1
-EXEC_PERSISTENT, EXEC_STEPPED, EXEC_MANUAL = 0, 1, 2
+EXEC_PERSISTENT, EXEC_STEPPED, EXEC_MANUAL, EXEC_HOST_GRAPH, EXEC_HOST_LAUNCHES = 0, 1, 2, 3, 4
 GEMM_AUTO, GEMM_SIMT, GEMM_TC, GEMM_TC_PAIR = 0, 1, 2, 3
 WEIGHTS_ROW_MAJOR, WEIGHTS_STREAMING = 0, 1
 FUSION_AUTO, FUSION_OFF, FUSION_ON = 0, 1, 2

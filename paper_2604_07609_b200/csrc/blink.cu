@@ -174,7 +174,7 @@ struct blink_ctx {
   std::deque<int> active;
   int hint = 0;
   uint64_t next_ticket = 0;
-  int64_t launches = 0;
+  std::atomic<int64_t> launches{0};
   int64_t bytes_to_device = 0, bytes_from_device = 0;
   int64_t clock_offset = 0;
   bool final_stop = false;
@@ -186,6 +186,12 @@ struct blink_ctx {
   bool manual = false;
   bool pair = false;   // GEMMs on CTA pairs: kernels launched with clusters of two
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+  // host-driven comparison arms: a thread of the library launches one iteration at a time
+  int host_driven = 0;                 // 0, BLINK_EXEC_HOST_GRAPH or BLINK_EXEC_HOST_LAUNCHES
+  cudaGraphExec_t iter_graph = nullptr;
+  std::thread driver;
+  std::atomic<bool> driver_stop{false};
+  std::atomic<int> driver_error{0};
 };
 
 namespace {
@@ -223,6 +229,8 @@ void free_all(blink_ctx* x) {
   if (x->ev0) cudaEventDestroy(x->ev0);
   if (x->ev1) cudaEventDestroy(x->ev1);
   x->ev0 = x->ev1 = nullptr;
+  if (x->iter_graph) cudaGraphExecDestroy(x->iter_graph);
+  x->iter_graph = nullptr;
   if (x->stream) cudaStreamDestroy(x->stream);
   if (x->copy_stream) cudaStreamDestroy(x->copy_stream);
   x->stream = x->copy_stream = nullptr;
@@ -273,6 +281,7 @@ int launch_loop(blink_ctx* x) {
 
 // Re-instantiate a loop that left the GPU while work is outstanding (caller holds mu).
 int pump(blink_ctx* x) {
+  if (x->host_driven) return x->driver_error.load(std::memory_order_acquire) != 0 ? BLINK_EDEVICE : BLINK_OK;
   if (x->dc.stepped || x->manual) return BLINK_OK;
   const uint32_t st = x->mbox->loop_state;
   if (st == BLINK_LOOP_RUNNING) return BLINK_OK;
@@ -315,6 +324,48 @@ int step_once(blink_ctx* x) {
     for (int ph = PH_FNORM; ph <= PH_SAMPLE; ++ph) launch_phase(x, ph, 0);
   }
   return cudaGetLastError() == cudaSuccess ? BLINK_OK : BLINK_ECUDA;
+}
+
+// The host-resident serving loop of the comparison arms: while requests are outstanding, launch one iteration
+// and wait for it (the host is on the critical path of every token, as in the stacks of Section 6.1).
+void driver_loop(blink_ctx* x) {
+  while (!x->driver_stop.load(std::memory_order_acquire)) {
+    bool work;
+    {
+      std::lock_guard<std::mutex> g(x->mu);
+      work = !x->active.empty() && (!x->dc.start_paused || x->mbox->start != 0);
+    }
+    if (!work) {
+      std::this_thread::sleep_for(std::chrono::microseconds(50));
+      continue;
+    }
+    int rc = BLINK_OK;
+    if (x->iter_graph) {
+      if (cudaGraphLaunch(x->iter_graph, x->stream) != cudaSuccess) rc = BLINK_ECUDA;
+      x->launches += 1;
+    } else {
+      rc = step_once(x);
+    }
+    if (rc == BLINK_OK && cudaStreamSynchronize(x->stream) != cudaSuccess) rc = BLINK_ECUDA;
+    if (rc == BLINK_OK && x->mbox->device_status > 0 && x->mbox->device_status != DEV_ERR_TRACE_OVERFLOW) rc = BLINK_EDEVICE;
+    if (rc != BLINK_OK) {
+      x->driver_error.store(rc, std::memory_order_release);
+      return;
+    }
+  }
+}
+
+void driver_start(blink_ctx* x) {
+  if (!x->host_driven || x->driver.joinable() || x->driver_error.load() != 0) return;
+  x->driver_stop.store(false, std::memory_order_release);
+  x->driver = std::thread(driver_loop, x);
+}
+
+// never called with x->mu held: the driver takes it between iterations
+void driver_join(blink_ctx* x) {
+  if (!x->driver.joinable()) return;
+  x->driver_stop.store(true, std::memory_order_release);
+  x->driver.join();
 }
 
 }  // namespace
@@ -575,7 +626,9 @@ int blink_create(const blink_model_cfg* model, const blink_sched_cfg* sched, con
   c.max_pos = c.max_prompt + c.max_new;
   c.max_blocks_seq = (c.max_pos + c.bs - 1) / c.bs;
   c.control_only = sched->control_only; c.start_paused = sched->start_paused;
-  c.stepped = sched->exec_mode == BLINK_EXEC_STEPPED;
+  if (sched->exec_mode < BLINK_EXEC_PERSISTENT || sched->exec_mode > BLINK_EXEC_HOST_LAUNCHES) { delete x; return BLINK_EINVAL; }
+  x->host_driven = sched->exec_mode >= BLINK_EXEC_HOST_GRAPH ? sched->exec_mode : 0;
+  c.stepped = sched->exec_mode == BLINK_EXEC_STEPPED || x->host_driven != 0;
   x->manual = sched->exec_mode == BLINK_EXEC_MANUAL;
   c.gemm_tc = 0;
   if (!c.control_only && model->dtype == BLINK_DTYPE_BF16 && sched->gemm_impl != BLINK_GEMM_SIMT)
@@ -778,16 +831,33 @@ int blink_create(const blink_model_cfg* model, const blink_sched_cfg* sched, con
   } else {
     x->mbox->loop_state = BLINK_LOOP_NOT_STARTED;
   }
+  if (x->host_driven == BLINK_EXEC_HOST_GRAPH) {
+    // one iteration (control plane + every phase) captured once: shapes come from device metadata, so the
+    // same graph serves every step
+    cudaGraph_t g = nullptr;
+    if (cudaStreamBeginCapture(x->stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) return fail(BLINK_ECUDA);
+    const int src = step_once(x);
+    if (cudaStreamEndCapture(x->stream, &g) != cudaSuccess || src != BLINK_OK || g == nullptr) return fail(BLINK_ECUDA);
+    const cudaError_t ie = cudaGraphInstantiate(&x->iter_graph, g, 0);
+    cudaGraphDestroy(g);
+    if (ie != cudaSuccess) return fail(BLINK_ECUDA);
+    x->launches = 0;
+  }
   *out = x;
+  if (x->host_driven && !c.start_paused) driver_start(x);
   return BLINK_OK;
 }
 
 int blink_start(blink_ctx* x) {
   if (!x) return BLINK_EINVAL;
-  std::lock_guard<std::mutex> g(x->mu);
-  std::atomic_thread_fence(std::memory_order_seq_cst);
-  x->mbox->start = 1;
-  return pump(x) == BLINK_EDEVICE ? BLINK_EDEVICE : BLINK_OK;
+  {
+    std::lock_guard<std::mutex> g(x->mu);
+    std::atomic_thread_fence(std::memory_order_seq_cst);
+    x->mbox->start = 1;
+    if (!x->host_driven) return pump(x) == BLINK_EDEVICE ? BLINK_EDEVICE : BLINK_OK;
+  }
+  driver_start(x);
+  return x->driver_error.load() != 0 ? x->driver_error.load() : BLINK_OK;
 }
 
 int blink_submit(blink_ctx* x, const blink_request* r, uint64_t* ticket_out) {
@@ -907,7 +977,7 @@ int blink_cancel(blink_ctx* x, uint64_t ticket) {
 
 int blink_step(blink_ctx* x, int n_iterations) {
   if (!x || n_iterations < 0) return BLINK_EINVAL;
-  if (!x->dc.stepped) return BLINK_EINVAL;
+  if (!x->dc.stepped || x->host_driven) return BLINK_EINVAL;
   std::lock_guard<std::mutex> g(x->mu);
   for (int i = 0; i < n_iterations; ++i) {
     const int rc = step_once(x);
@@ -940,6 +1010,7 @@ int blink_run(blink_ctx* x, int64_t n_iterations, float* elapsed_ms) {
 
 int blink_stop(blink_ctx* x, int final, int timeout_ms) {
   if (!x) return BLINK_EINVAL;
+  if (x->host_driven) driver_join(x);   // leaves between iterations; blink_start brings it back
   std::lock_guard<std::mutex> g(x->mu);
   if (final) x->final_stop = true;
   if (x->dc.stepped) return cudaStreamSynchronize(x->stream) == cudaSuccess ? BLINK_OK : BLINK_ECUDA;

@@ -60,6 +60,20 @@ def test_stepped_mode_matches_persistent_mode_bitwise():
     assert_traces_equal(a[0], b[0])
 
 
+@pytest.mark.parametrize("mode", [B.EXEC_HOST_GRAPH, B.EXEC_HOST_LAUNCHES], ids=["graph-per-iteration", "launch-per-phase"])
+def test_host_driven_arms_match_persistent_mode_bitwise(mode):
+    """The comparison arms (a host thread launches one iteration at a time and waits for it) run the same
+    device code: same trace, same tokens, same logits bit for bit; blink_step is refused there."""
+    model, sched = model_cfg(1, dtype="fp32"), sched_cfg(1)
+    reqs = make_requests(1, n_requests=4)
+    w = make_weights(model, 99, "cpu", random_gains=True)
+    a = gpu_run_forced(model, sched, reqs, w, None, exec_mode=B.EXEC_PERSISTENT)
+    b = gpu_run_forced(model, sched, reqs, w, None, exec_mode=mode)
+    assert a[1] == b[1]
+    assert np.array_equal(a[2], b[2])
+    assert_traces_equal(a[0], b[0])
+
+
 def test_gqa_random_gains_chunked_prefill_small_chunk():
     """Grouped-query heads (4 q per kv head), head_dim 128, non-unit norm gains, and a chunk
     budget smaller than the prompts so prefill spans several iterations and mixes with decode."""
