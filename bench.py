@@ -756,6 +756,12 @@ def main():
                                     tpot_p99=ratio(a["tpot_ms"]["p99"], b["tpot_ms"]["p99"]),
                                     tpot_p50=ratio(a["tpot_ms"]["p50"], b["tpot_ms"]["p50"]),
                                     throughput=ratio(a["tok_s"], b["tok_s"]))
+            if not args.skip_e2e:
+                # closed loop (all requests at t = 0), the same run as `e2e`, for the throughput cost of the host in the loop
+                rh = realtime_run(B, m, sched, wbuf, kv, reqs, args.e2e_seconds, use_arrivals=False, weights_layout=wl,
+                                  exec_mode=hmode)
+                hd["e2e_tok_s"] = rh["tok_s"]
+                hd["e2e_tok_s_gpu_resident"] = line.get("e2e", {}).get("value")
             line["host_driven"] = hd
     # ---- offered-load sweep (Section 6.1: 13 levels between 1 and 32 req/s; Appendix C: serviceable load) ----
     if args.rates and rank == 0 and world == 1:
