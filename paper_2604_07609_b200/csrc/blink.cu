@@ -188,6 +188,7 @@ struct blink_ctx {
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
   // host-driven comparison arms: a thread of the library launches one iteration at a time
   int host_driven = 0;                 // 0, BLINK_EXEC_HOST_GRAPH or BLINK_EXEC_HOST_LAUNCHES
+  int device = 0;                      // the device of the context: the driver thread selects it
   cudaGraphExec_t iter_graph = nullptr;
   std::thread driver;
   std::atomic<bool> driver_stop{false};
@@ -329,6 +330,10 @@ int step_once(blink_ctx* x) {
 // The host-resident serving loop of the comparison arms: while requests are outstanding, launch one iteration
 // and wait for it (the host is on the critical path of every token, as in the stacks of Section 6.1).
 void driver_loop(blink_ctx* x) {
+  if (cudaSetDevice(x->device) != cudaSuccess) {
+    x->driver_error.store(BLINK_ECUDA, std::memory_order_release);
+    return;
+  }
   while (!x->driver_stop.load(std::memory_order_acquire)) {
     bool work;
     {
@@ -628,6 +633,7 @@ int blink_create(const blink_model_cfg* model, const blink_sched_cfg* sched, con
   c.control_only = sched->control_only; c.start_paused = sched->start_paused;
   if (sched->exec_mode < BLINK_EXEC_PERSISTENT || sched->exec_mode > BLINK_EXEC_HOST_LAUNCHES) { delete x; return BLINK_EINVAL; }
   x->host_driven = sched->exec_mode >= BLINK_EXEC_HOST_GRAPH ? sched->exec_mode : 0;
+  x->device = dev;
   c.stepped = sched->exec_mode == BLINK_EXEC_STEPPED || x->host_driven != 0;
   x->manual = sched->exec_mode == BLINK_EXEC_MANUAL;
   c.gemm_tc = 0;
