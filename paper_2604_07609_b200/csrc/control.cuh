@@ -649,7 +649,9 @@ static __device__ int schedule_step(const DevCtx& c, unsigned long long visible)
 // One pass of the control plane.  `launch_iters` counts the iterations this kernel
 // launch has started.  Sets ss->cmd to CMD_RUN (a step was composed), CMD_EXIT
 // (leave the GPU; reason in ss->exit_reason) or CMD_NONE (stepped mode, idle).
-static __device__ void control_phase(const DevCtx& c, long long& launch_iters) {
+// (a function of its own: inlined, its code shares the register allocation of the dispatcher of the loop kernel,
+// which then spills more on the path of every phase: 1-1.5 % of a decode step)
+static __device__ __noinline__ void control_phase(const DevCtx& c, long long& launch_iters) {
   SchedState* ss = c.ss;
   const int tid = threadIdx.x;
   __shared__ int s_cmd;
