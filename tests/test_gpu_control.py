@@ -23,11 +23,20 @@ def _check(model, sched, reqs, **kw):
     return trace, st, its
 
 
-@pytest.mark.parametrize("mode", [B.EXEC_PERSISTENT, B.EXEC_STEPPED], ids=["persistent", "stepped"])
+@pytest.mark.parametrize("mode", [B.EXEC_PERSISTENT, B.EXEC_STEPPED, B.EXEC_HOST_GRAPH, B.EXEC_HOST_LAUNCHES],
+                         ids=["persistent", "stepped", "host-graph", "host-launches"])
 def test_config1_trace_bit_exact(mode):
     model, sched = model_cfg(1), sched_cfg(1)
     trace, st, _ = _check(model, sched, make_requests(1), exec_mode=mode)
     assert trace[0]["W"] == 7 and len(trace[0]["admitted"]) == 8     # all visible to the first iteration
+
+
+def test_host_driven_arm_with_requests_arriving_while_it_runs():
+    """The host-driven comparison arm (a library thread launches one iteration per CUDA graph and waits for it):
+    half of the requests arrive after the start; the trace equals the oracle's replay with the logged watermarks."""
+    model, sched = model_cfg(1), sched_cfg(1)
+    trace, st, _ = _check(model, sched, make_requests(1), exec_mode=B.EXEC_HOST_GRAPH, trickle=4)
+    assert st.launches >= len(trace)        # one graph launch per iteration
 
 
 def test_tiny_pool_head_of_line_blocking():
