@@ -179,10 +179,55 @@ __device__ __forceinline__ void norm_row_cta(const DevCtx& c, float* hrow, const
   }
 }
 
+// Rows of a CTA in turn, the next row on its way (asynchronous copies into shared memory, each thread reads
+// back only what it copied itself) while the current one is summed and scaled: with several rows per CTA
+// (steps of more rows than SMs) the phase is a chain of row latencies otherwise.  The copies hold no
+// registers.  NV = d / 1024 16-byte vectors per thread.
+template <typename WT, int NV>
+static __device__ __noinline__ void norm_rows_pipelined(const DevCtx& c, const float* g, WT* out, int T, float* s_red, float* smem) {
+  constexpr int d = NV * 1024;
+  int t = blockIdx.x;
+  if (t >= T) return;
+  const char* stage = reinterpret_cast<const char*>(smem) + threadIdx.x * 16;   // [NV][FWD_THREADS] x 16 bytes
+  const uint32_t stage_s = (uint32_t)__cvta_generic_to_shared(stage);
+  const float* src = c.h + (size_t)t * d + threadIdx.x * 4;
+#pragma unroll
+  for (int k = 0; k < NV; ++k)
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(stage_s + k * FWD_THREADS * 16), "l"(src + k * FWD_THREADS * 4) : "memory");
+  asm volatile("cp.async.commit_group;" ::: "memory");
+#pragma unroll 1
+  for (; t < T; t += gridDim.x) {
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    float4 cur[NV];
+#pragma unroll
+    for (int k = 0; k < NV; ++k) cur[k] = *reinterpret_cast<const float4*>(stage + k * FWD_THREADS * 16);
+    if (t + (int)gridDim.x < T) {
+      src += (size_t)gridDim.x * d;
+#pragma unroll
+      for (int k = 0; k < NV; ++k)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(stage_s + k * FWD_THREADS * 16), "l"(src + k * FWD_THREADS * 4) : "memory");
+      asm volatile("cp.async.commit_group;" ::: "memory");
+    }
+    float ss = 0.f;
+#pragma unroll
+    for (int k = 0; k < NV; ++k) {  // fixed order, the same as norm_row_cta
+      ss = fmaf(cur[k].x, cur[k].x, ss); ss = fmaf(cur[k].y, cur[k].y, ss); ss = fmaf(cur[k].z, cur[k].z, ss); ss = fmaf(cur[k].w, cur[k].w, ss);
+    }
+    ss = block_sum(ss, s_red);
+    const float inv = rsqrtf(ss * (1.0f / (float)d) + c.rms_eps);
+    WT* orow = out + (size_t)t * d + threadIdx.x * 4;
+#pragma unroll
+    for (int k = 0; k < NV; ++k) {
+      const float4 gg = *reinterpret_cast<const float4*>(g + (k * FWD_THREADS + threadIdx.x) * 4);
+      store4<WT>(orow + k * FWD_THREADS * 4, cur[k].x * inv * gg.x, cur[k].y * inv * gg.y, cur[k].z * inv * gg.z, cur[k].w * inv * gg.w);
+    }
+  }
+}
+
 // ---- RMSNorm of the residual rows into the operand buffer; layer 0 gathers the
 // embedding first.
 template <typename WT>
-static __device__ __noinline__ void phase_norm(const DevCtx& c, int layer, int which /*0: norm1, 1: norm2*/) {
+static __device__ __noinline__ void phase_norm(const DevCtx& c, int layer, int which /*0: norm1, 1: norm2*/, float* smem) {
   __shared__ float s_red[FWD_THREADS / 32];
   const int T = c.ss->cur_T;
   const float* g = wptr_f(c, which == 0 ? 6 : 7) + (size_t)layer * c.d;
@@ -194,6 +239,11 @@ static __device__ __noinline__ void phase_norm(const DevCtx& c, int layer, int w
       c.rowss_b[i] = 0.f;
     }
   const float* wr = (which == 1 && c.E > 0) ? wptr_f(c, 5) + (size_t)layer * c.E * c.d : nullptr;
+  if (wr == nullptr && !(which == 0 && layer == 0) && T > (int)gridDim.x && (c.d == 4096 || c.d == 2048)) {
+    if (c.d == 4096) norm_rows_pipelined<WT, 4>(c, g, out, T, s_red, smem);
+    else norm_rows_pipelined<WT, 2>(c, g, out, T, s_red, smem);
+    return;
+  }
   for (int t = blockIdx.x; t < T; t += gridDim.x) {
     const WT* e = (which == 0 && layer == 0) ? wptr<WT>(c, 0) + (size_t)c.tok_id[t] * c.d : nullptr;
     norm_row_cta<WT>(c, c.h + (size_t)t * c.d, e, g, out + (size_t)t * c.d, s_red, wr, t);

@@ -29,7 +29,7 @@ __device__ __forceinline__ void run_phase(const DevCtx& c, int phase, int layer,
   switch (phase) {
     case PH_NORM1:
       if (c.fused_norm && layer > 0) phase_norm_apply<WT>(c, layer, 0, T);
-      else phase_norm<WT>(c, layer, 0);
+      else phase_norm<WT>(c, layer, 0, smem);
       break;
     case PH_QKV: {
       GemmArgs a{c.xn, c.w_base + c.w_off[1] + (size_t)layer * c.qkv_dim * c.d * esz, c.qkv, T, c.qkv_dim, c.d,
@@ -52,7 +52,7 @@ __device__ __forceinline__ void run_phase(const DevCtx& c, int phase, int layer,
     } break;
     case PH_NORM2:
       if (c.fused_norm) phase_norm_apply<WT>(c, layer, 1, T);
-      else phase_norm<WT>(c, layer, 1);
+      else phase_norm<WT>(c, layer, 1, smem);
       break;
     case PH_GU: {
       if (c.E == 0) {
