@@ -43,7 +43,7 @@ POLICY = 0   # BLINK_POLICY_* used by every engine this run creates (--policy)
 # count; the bench scales the traffic to its own steps by the ratio of algorithmic bytes.  `digest` is
 # kernel_digest() at capture time: once the kernels change the figure is stale and is reported as null.
 TRAFFIC = {
-    "C3 8B stream": dict(traffic_gb=45.50, algorithmic_gb=40.596, digest="2ace0b5037b1ceca",
+    "C3 8B stream": dict(traffic_gb=45.55, algorithmic_gb=40.596, digest="3c3e2e4e64c46518",
                          source="profiles/dram_traffic_8B_stepped.md"),
 }
 
